@@ -1,0 +1,54 @@
+"""Initial parameter values and the flat parameter order.
+
+Flat order: layers in list order; per layer (weight, [bias], gamma, beta):
+  conv    weight [c_out][k][k][c_in]      (KRSC, no bias)
+  dwconv  weight [c][k][k]
+  bn      gamma [c], beta [c]
+  linear  weight [c_out][c_in], bias [c_out]
+Conv and linear weights ~ U(-b, b), b = sqrt(6 / fan_in), fan_in = k*k*c_in/groups;
+gamma = 1, beta = 0, bias = 0.  The stream of a layer's weight is keyed by its index
+in the whole network, so a stage cut out of a network sees the same values.
+"""
+import numpy as np
+from .rng import uniform
+
+_PARAM_TID = 1000
+
+
+def param_layout(net, first, last):
+    """[(layer_index, name, shape)] in flat order."""
+    out = []
+    for i in range(first, last + 1):
+        L = net[i]
+        if L.op == "conv":
+            out.append((i, "weight", (L.c_out, L.k, L.k, L.c_in)))
+        elif L.op == "dwconv":
+            out.append((i, "weight", (L.c_out, L.k, L.k)))
+        elif L.op == "bn":
+            out.append((i, "gamma", (L.c_out,)))
+            out.append((i, "beta", (L.c_out,)))
+        elif L.op == "linear":
+            out.append((i, "weight", (L.c_out, L.c_in)))
+            out.append((i, "bias", (L.c_out,)))
+    return out
+
+
+def param_count(net, first, last):
+    return sum(int(np.prod(s)) for _, _, s in param_layout(net, first, last))
+
+
+def init_params(net, first, last, seed=0):
+    """Flat float32 parameter vector of stage [first, last]."""
+    parts = []
+    for i, name, shape in param_layout(net, first, last):
+        n = int(np.prod(shape))
+        L = net[i]
+        if name == "weight":
+            fan_in = {"conv": L.k * L.k * L.c_in, "dwconv": L.k * L.k, "linear": L.c_in}[L.op]
+            b = np.sqrt(6.0 / fan_in)
+            parts.append(((2.0 * uniform(seed, _PARAM_TID + i, n) - 1.0) * b).astype(np.float32))
+        elif name == "gamma":
+            parts.append(np.ones(n, np.float32))
+        else:
+            parts.append(np.zeros(n, np.float32))
+    return np.concatenate(parts) if parts else np.zeros(0, np.float32)
