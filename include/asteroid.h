@@ -1,0 +1,170 @@
+/*
+ * asteroid.h — C ABI of the per-stage micro-batched training step.
+ *
+ * A *stage* is a contiguous range of a network's layers; one *HPP-Round* on a stage is
+ * FP over M micro-batches of size B, BP over the same micro-batches, accumulation of the
+ * parameter gradients of all of them, and one update at the end (Asteroid, Section 3.2,
+ * "HPP Architecture and Workflow").  The calls below are exactly those steps, plus the
+ * per-layer profile that feeds the planner (Section 3.3, "DNN Model and Asteroid Profiler").
+ *
+ * Conventions
+ *  - Every call returns 0 on success or a negative AST_ERR_* code; the text of the last error
+ *    of the calling thread is available from asteroid_last_error().  Nothing throws or exits.
+ *  - Activation tensors are DEVICE pointers, NHWC, in the stage's storage type (float or
+ *    bfloat16), owned by the caller.  Parameter / state vectors passed to import/export are
+ *    HOST pointers to float.  The stage owns its arenas and frees them in destroy.
+ *  - `stream` is a cudaStream_t passed as void*.  forward/backward/accumulate/step and the loss
+ *    heads only enqueue work on it; they never synchronise.  create, destroy, import, export
+ *    and profile synchronise the device.
+ *  - The library has no CPU fallback: without a CUDA device every compute call fails.
+ *
+ * Flat parameter order (import/export): layers in list order; per layer
+ *    conv    weight [c_out][k][k][c_in]
+ *    dwconv  weight [c][k][k]
+ *    bn      gamma [c], beta [c]
+ *    linear  weight [c_out][c_in], bias [c_out]
+ */
+#ifndef ASTEROID_H
+#define ASTEROID_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct asteroid_stage asteroid_stage;
+
+enum { AST_CONV = 0, AST_DWCONV = 1, AST_BN = 2, AST_RELU6 = 3, AST_RELU = 4, AST_ADD = 5, AST_GAP = 6, AST_LINEAR = 7 };
+enum { AST_F32 = 0, AST_BF16 = 1 };
+enum {
+    AST_OK = 0,
+    AST_ERR_ARG = -1,          /* null pointer, bad range, bad size */
+    AST_ERR_UNSUPPORTED = -2,  /* a layer pattern or shape the kernels do not cover */
+    AST_ERR_ORDER = -3,        /* call sequence violates the round (see each call) */
+    AST_ERR_ALLOC = -4,        /* device allocation failed */
+    AST_ERR_CUDA = -5,         /* a CUDA runtime call failed; text in asteroid_last_error() */
+    AST_ERR_TIMEOUT = -6       /* a bounded device-side wait expired */
+};
+
+/* One layer of the network's layer sequence (Section 3.3: the model graph is topologically
+ * sorted into a sequence of layers).  `src` is the index of the layer whose output this layer
+ * reads, `add_from` (AST_ADD only) the index of the second operand; index -1 is the network
+ * input.  Inside a stage [first,last] an index equal to first-1 denotes the stage input;
+ * smaller indices are rejected.  Conv: cross-correlation, zero padding `pad`, no bias, weights
+ * [c_out][k][k][c_in].  Dwconv: k=3, pad=1, c_in==c_out.  BN: training mode, statistics over
+ * the micro-batch.  Add: out = value[src] + value[add_from]. */
+typedef struct {
+    int32_t op, c_in, c_out, k, stride, pad, src, add_from;
+} ast_layer;
+
+typedef struct {
+    int32_t dtype;            /* AST_F32, or AST_BF16 = bfloat16 activations and activation gradients,
+                                 float master weights, statistics, gradients and optimizer state */
+    int32_t slots;            /* K: micro-batches that may be resident between their FP and BP
+                                 (Section 3.2, K_p warm-up forwards); 0 means M */
+    int32_t need_input_grad;  /* 0 for the first stage of a network: BP writes no dx */
+    float bn_eps;             /* 0 means 1e-5 */
+    float bn_momentum;        /* running-statistics momentum; 0 means 0.1 */
+} ast_opts;
+
+/* Per-layer record for the planner (Section 3.3): t_f, t_b at the given batch size, output
+ * bytes a_l, weight bytes w_l; FLOPs as used by the re-planning of Section 3.4; and the three
+ * memory terms of Eq. (3). */
+typedef struct {
+    double t_f_ms, t_b_ms;       /* median device time of the kernels that execute this layer's FP / BP.
+                                    A layer fused into a neighbour's kernel reports 0 and names that
+                                    neighbour in fused_into. */
+    uint64_t a_l_bytes;          /* output activation bytes at `batch` in the storage type */
+    uint64_t w_l_bytes;          /* float32 parameter bytes */
+    uint64_t flops;              /* forward FLOPs at `batch`: 2 per multiply-accumulate of conv / linear layers */
+    uint64_t alg_bytes_f;        /* bytes the layer's FP kernels must move (each tensor once) */
+    uint64_t alg_bytes_b;        /* same for BP */
+    uint64_t mem_mod;            /* Eq. (3) Mem_MOD: parameters, accumulated and per-micro-batch gradients, derived weight copies */
+    uint64_t mem_opt;            /* Eq. (3) Mem_OPT: momentum */
+    uint64_t mem_act;            /* Eq. (3) Mem_ACT(batch): one resident micro-batch's saved tensors */
+    uint64_t mem_work;           /* BP workspace and reduction scratch (transient; not a term of Eq. (3)) */
+    int32_t fused_into;          /* layer index whose kernels execute this layer, or -1 */
+    int32_t reserved;
+} ast_layer_profile;
+
+/* Build the stage for layers [first,last] of `net` (Section 3.2: a stage model is a set of
+ * consecutive layers), for micro-batches of `micro_batch` samples of in_h x in_w x net[first].c_in,
+ * M micro-batches per round.  Parameters start at zero (gamma too): call import_state.
+ * Errors: AST_ERR_ARG (range, sizes, references below first-1), AST_ERR_UNSUPPORTED (a BN or
+ * activation that does not follow a conv/add it can fuse with, an intermediate of a fused
+ * conv-BN-activation chain read by another layer, dwconv with k!=3), AST_ERR_ALLOC. */
+int asteroid_stage_create(const ast_layer* net, int n_layers, int first, int last,
+                          int in_h, int in_w, int micro_batch, int M,
+                          const ast_opts* opts, asteroid_stage** out);
+void asteroid_stage_destroy(asteroid_stage* s);
+
+size_t asteroid_stage_param_count(const asteroid_stage* s);
+/* Elements of the stage output per micro-batch, and its (h, w, c). */
+size_t asteroid_stage_output_elems(const asteroid_stage* s, int* h, int* w, int* c);
+
+/* Load parameters (and optionally momentum; NULL keeps/clears it to zero) from HOST memory;
+ * n must equal param_count.  Also refreshes the derived weight copies the kernels read. */
+int asteroid_stage_import_state(asteroid_stage* s, const float* params, const float* momentum, size_t n);
+/* Copy state to HOST memory; any pointer may be NULL.  micro_grad is g_m of the last backward. */
+int asteroid_stage_export_state(asteroid_stage* s, float* params, float* momentum, float* grad_accum,
+                                float* micro_grad, size_t n);
+/* BatchNorm running mean / variance (momentum update once per forward, unbiased variance),
+ * concatenated over the stage's BN layers in layer order; n = sum of their channel counts. */
+int asteroid_stage_export_bn_running(asteroid_stage* s, float* mean, float* var, size_t n);
+
+/* FP of micro-batch `mb` (Section 3.2): reads x (B x in_h x in_w x c_in), writes the stage output y,
+ * and keeps in an activation slot what BP of `mb` needs (x itself is copied, the caller may reuse
+ * it).  Errors: AST_ERR_ARG (mb outside [0,M)), AST_ERR_ORDER (mb already resident, or `slots`
+ * micro-batches already resident). */
+int asteroid_stage_forward(asteroid_stage* s, int mb, const void* x, void* y, void* stream);
+/* BP of micro-batch `mb`: reads dy = dL/dy, writes dx = dL/dx (ignored when need_input_grad==0) and the
+ * parameter gradients g_mb of this micro-batch, then releases the slot.  Errors: AST_ERR_ORDER
+ * (no resident FP of mb, or the previous g not yet accumulated). */
+int asteroid_stage_backward(asteroid_stage* s, int mb, const void* dy, void* dx, void* stream);
+/* G += g_mb: accumulate the gradients of the micro-batch whose BP ran last (Section 3.2: each device
+ * accumulates gradients for all micro-batches of the mini-batch).  AST_ERR_ORDER if mb is not that one. */
+int asteroid_stage_accumulate(asteroid_stage* s, int mb, void* stream);
+/* End of the HPP-Round (Section 3.2: accumulated gradients are applied to the stage parameters):
+ * g = G/M; v = momentum*v + g; w = w - lr*v; G = 0; derived weight copies refreshed.
+ * AST_ERR_ORDER unless exactly M micro-batches were accumulated since the last step. */
+int asteroid_stage_step(asteroid_stage* s, float lr, float momentum, void* stream);
+
+/* Per-layer cost record at batch size `batch` (Section 3.3: FP/BP time of each layer for various
+ * batch sizes, output size and weight size in bytes).  Runs the stage's own kernels on zero-filled
+ * buffers of that batch size (3 warm-up + 7 timed rounds, CUDA events), synchronises.
+ * `layer` is an index in [first,last]. */
+int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_profile* out);
+
+/* Loss heads (used by the last stage and by tests).  All pointers are DEVICE pointers.
+ * MSE: *loss = mean((y-t)^2) over n elements, dy = 2 (y-t) / n. */
+int asteroid_loss_mse(const void* y, const void* target, size_t n, int dtype, void* dy, float* loss, void* stream);
+/* Softmax cross-entropy: *loss = mean_r(-log softmax(logits_r)[labels_r]),
+ * dlogits = (softmax - onehot) / rows.  rows <= 65536. */
+int asteroid_loss_softmax_xent(const void* logits, const int32_t* labels, int rows, int classes, int dtype,
+                               void* dlogits, float* loss, void* stream);
+
+/* Kernel-level trace (the paper has no counterpart; its profiler works per layer, Section 3.3).
+ * Between start and stop every kernel launch of the library is bracketed by CUDA events on its
+ * stream; stop synchronises the device and returns, per kernel kind that ran, the number of
+ * launches, the summed device time, the summed algorithmic bytes (each tensor the kernel must
+ * read or write, once) and floating-point operations.  At most `capacity` records are written,
+ * *n_out receives the count.  Tracing adds two event records per launch: do not time throughput
+ * while it is on. */
+typedef struct {
+    char name[48];
+    uint64_t launches;
+    double total_ms, alg_bytes, flops;
+} ast_kernel_stat;
+int asteroid_trace_start(void);
+int asteroid_trace_stop(ast_kernel_stat* out, int capacity, int* n_out);
+
+/* Count of kernel launches this library has enqueued in the calling process. */
+uint64_t asteroid_launch_count(void);
+const char* asteroid_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -28,8 +28,23 @@ def _layer_param_shapes(layer):
     return []
 
 
+_CONVLIKE = ("conv", "dwconv", "linear")
+_ACTS = ("relu6", "relu")
+
+
 class Stage:
-    def __init__(self, net, first, last, micro_batch, n_micro, params, eps=1e-5, bn_momentum=0.1):
+    """`store`: optional rounding function applied wherever a reduced-precision implementation
+    keeps a tensor in memory (all arithmetic stays float64).  With bfloat16 activations the
+    ReLU/ReLU6 masks are decisions taken on stored values; a comparison against such an
+    implementation is only meaningful if both sides decide on the same stored numbers.  The
+    storage points are: the output of every conv / depthwise conv / linear layer (before its
+    BatchNorm), the output of a residual add (after the ReLU that directly follows it, if any),
+    the pooled features, the stage output, and the gradient with respect to each of those
+    stored-or-recomputed unit outputs and to the stage input (rounded after every term added
+    to it).  BatchNorm and activation outputs inside a conv->BN->activation chain are never
+    stored.  store=None is the plain float64 definition."""
+
+    def __init__(self, net, first, last, micro_batch, n_micro, params, eps=1e-5, bn_momentum=0.1, store=None):
         if not (0 <= first <= last < len(net)):
             raise ValueError("bad layer range")
         self.net, self.first, self.last = net, first, last
@@ -52,6 +67,33 @@ class Stage:
             raise ValueError("parameter vector has %d values, stage needs %d" % (flat.size, off))
         self.saved = {}          # micro-batch -> {layer index: output}, caches
         self.n_accumulated = 0
+        self.store = store
+
+    def _chains_into_next(self, i):
+        """True if layer i+1 continues layer i's chain (conv->BN, conv/BN->activation, add->ReLU),
+        i.e. the output of layer i is an unstored intermediate."""
+        if i < self.first or i >= self.last:
+            return False
+        a, b = self.net[i], self.net[i + 1]
+        if b.src != i:
+            return False
+        if a.op in _CONVLIKE:
+            return b.op == "bn" or b.op in _ACTS
+        if a.op == "bn":
+            return b.op in _ACTS and i - 1 >= self.first and self.net[i - 1].op in _CONVLIKE and a.src == i - 1
+        if a.op == "add":
+            return b.op == "relu"
+        return False
+
+    def _stored_forward(self, i):
+        op = self.net[i].op
+        if i == self.last or op in _CONVLIKE or op == "gap":
+            return True
+        if op == "add":
+            return not self._chains_into_next(i)
+        if op == "relu":
+            return i - 1 >= self.first and self.net[i - 1].op == "add" and self.net[i].src == i - 1
+        return False
 
     # ---- flat views -------------------------------------------------------------------
     def _flat(self, d):
@@ -101,6 +143,8 @@ class Stage:
                                           self.p[(i, "bias")]).reshape(a.shape[0], 1, 1, -1)
             else:
                 raise ValueError(ly.op)
+            if self.store is not None and self._stored_forward(i):
+                val[i] = self.store(val[i])
         self.saved[mb] = (val, cache)
         return val[self.last]
 
@@ -113,6 +157,8 @@ class Stage:
 
         def give(idx, d):
             grad[idx] = grad[idx] + d if idx in grad else d
+            if self.store is not None and not self._chains_into_next(idx):
+                grad[idx] = self.store(grad[idx])
 
         for i in range(self.last, self.first - 1, -1):
             ly = net[i]

@@ -1,0 +1,489 @@
+// BatchNorm statistics / backward reductions, elementwise pieces (residual add, activation
+// masks, materialisation of a stage output), global average pooling, gradient accumulation,
+// the SGD-momentum update and the two loss heads.  All are bandwidth-bound passes over
+// [pixels][channels] tensors; reductions are two-stage and deterministic (no float atomics).
+#include "kernels.h"
+
+namespace ast {
+namespace {
+
+// ------------------------------------------------------------------ per-channel reductions
+// A block owns `cw` channel groups (V channels each) and a contiguous pixel range; thread
+// (row, jl) walks the range with stride `rows`.  OP::acc adds one pixel's contribution to the
+// thread's NACC*V accumulators.  Rows are combined through shared memory, blocks through
+// partial[block_y][acc][c], summed in fixed order (in double) by the finishing kernel.
+struct StatsOp {
+    static constexpr int NACC = 2;
+    const void* z;
+    template <typename T, int V> __device__ __forceinline__ void acc(size_t e, int c0, const float* pivot, float (*a)[V]) const {
+        float v[V];
+        ld_raw_w<T, V>(z, e, v);
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            float d = v[q] - pivot[q];
+            a[0][q] += d;
+            a[1][q] = fmaf(d, d, a[1][q]);
+        }
+    }
+    template <typename T, int V> __device__ __forceinline__ void pivot(int c0, float* pv) const { ld_raw_w<T, V>(z, (size_t)c0, pv); }
+};
+
+struct BwdOp {
+    static constexpr int NACC = 2;
+    GradSrc g;            // k1 = nullptr here: yields dpre
+    const float* mean;
+    const float* rstd;
+    template <typename T, int V> __device__ __forceinline__ void acc(size_t e, int c0, const float* pivot, float (*a)[V]) const {
+        float d[V];
+        ld_grad_w<T, V>(g, e, c0, d);
+        if (mean) {
+            float z[V];
+            ld_raw_w<T, V>(g.z, e, z);
+#pragma unroll
+            for (int q = 0; q < V; ++q) {
+                a[0][q] += d[q];
+                a[1][q] = fmaf(d[q], (z[q] - __ldg(mean + c0 + q)) * __ldg(rstd + c0 + q), a[1][q]);
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < V; ++q) a[0][q] += d[q];
+        }
+    }
+    template <typename T, int V> __device__ __forceinline__ void pivot(int, float*) const {}
+};
+
+template <typename T, int V, typename OP>
+__global__ void __launch_bounds__(256) chan_reduce_kernel(OP op, size_t pixels, int c, int cw, int rows, size_t pix_per_block,
+                                                          float* __restrict__ partial) {
+    extern __shared__ float red[];
+    const int cg = c / V;
+    const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
+    const int j = blockIdx.x * cw + jl;
+    const bool active = row < rows && j < cg;
+    const int c0 = j * V;
+    float a[OP::NACC][V];
+#pragma unroll
+    for (int t = 0; t < OP::NACC; ++t)
+#pragma unroll
+        for (int q = 0; q < V; ++q) a[t][q] = 0.f;
+    if (active) {
+        float pv[V];
+#pragma unroll
+        for (int q = 0; q < V; ++q) pv[q] = 0.f;
+        op.template pivot<T, V>(c0, pv);
+        size_t pbeg = (size_t)blockIdx.y * pix_per_block, pend = min(pixels, pbeg + pix_per_block);
+        for (size_t p = pbeg + row; p < pend; p += rows) op.template acc<T, V>(p * c + c0, c0, pv, a);
+    }
+    const int width = cw * V;
+    for (int t = 0; t < OP::NACC; ++t) {
+        if (row < rows) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) red[row * width + jl * V + q] = a[t][q];
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < width; e += blockDim.x) {
+            int ch = blockIdx.x * width + e;
+            if (ch < c) {
+                float s = 0.f;
+                for (int r2 = 0; r2 < rows; ++r2) s += red[r2 * width + e];
+                partial[((size_t)blockIdx.y * OP::NACC + t) * c + ch] = s;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+struct ReducePlan {
+    int V, cw, rows, gx;
+    size_t by, ppb, smem;
+};
+
+ReducePlan plan_reduce(int dtype, size_t pixels, int c, int nacc, size_t scratch_floats) {
+    ReducePlan p;
+    int vmax = dtype == 0 ? 4 : 8;
+    p.V = (c % vmax == 0) ? vmax : 1;
+    int cg = c / p.V;
+    p.cw = cg < 32 ? cg : 32;
+    p.rows = 256 / p.cw;
+    p.gx = (cg + p.cw - 1) / p.cw;
+    size_t by = (4 * 148 + p.gx - 1) / p.gx;
+    size_t max_by = (pixels + (size_t)p.rows * 4 - 1) / ((size_t)p.rows * 4);
+    if (by > max_by) by = max_by;
+    size_t cap = scratch_floats / ((size_t)nacc * c);
+    if (by > cap) by = cap;
+    if (by < 1) by = 1;
+    p.ppb = (pixels + by - 1) / by;
+    p.by = (pixels + p.ppb - 1) / p.ppb;
+    p.smem = (size_t)p.rows * p.cw * p.V * sizeof(float);
+    return p;
+}
+
+double esz(int dtype) { return dtype == 0 ? 4.0 : 2.0; }
+
+template <typename OP>
+void launch_reduce(int dtype, const ReducePlan& p, const OP& op, size_t pixels, int c, float* partial, int kind, double bytes, cudaStream_t st) {
+    LaunchScope ls(kind, bytes + 8.0 * c * p.by, 4.0 * pixels * c, st);
+    dim3 grid(p.gx, (unsigned)p.by);
+    if (dtype == 0) {
+        if (p.V == 1) chan_reduce_kernel<float, 1, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        else chan_reduce_kernel<float, 4, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
+    } else {
+        if (p.V == 1) chan_reduce_kernel<__nv_bfloat16, 1, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        else chan_reduce_kernel<__nv_bfloat16, 8, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
+    }
+}
+
+template <typename T>
+__global__ void bn_stats_finish(const float* __restrict__ partial, int blocks, int c, const T* __restrict__ z, double count,
+                                const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float momentum, BnFwdOut o) {
+    int ch = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ch >= c) return;
+    double s1 = 0.0, s2 = 0.0;
+    for (int b = 0; b < blocks; ++b) {
+        s1 += partial[((size_t)b * 2 + 0) * c + ch];
+        s2 += partial[((size_t)b * 2 + 1) * c + ch];
+    }
+    double pivot = to_f<T>(z[ch]);
+    double m1 = s1 / count;
+    double mean = pivot + m1;
+    double var = s2 / count - m1 * m1;
+    if (var < 0.0) var = 0.0;
+    double rstd = 1.0 / sqrt(var + (double)eps);
+    double sc = (double)gamma[ch] * rstd;
+    o.mean[ch] = (float)mean;
+    o.rstd[ch] = (float)rstd;
+    o.scale[ch] = (float)sc;
+    o.shift[ch] = (float)((double)beta[ch] - mean * sc);
+    double unbiased = count > 1.0 ? var * count / (count - 1.0) : var;
+    o.run_mean[ch] = (float)((1.0 - momentum) * o.run_mean[ch] + momentum * mean);
+    o.run_var[ch] = (float)((1.0 - momentum) * o.run_var[ch] + momentum * unbiased);
+}
+
+__global__ void bn_bwd_finish(const float* __restrict__ partial, int blocks, int c, double count, const float* __restrict__ mean,
+                              const float* __restrict__ rstd, const float* __restrict__ gamma, BnBwdOut o) {
+    int ch = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ch >= c) return;
+    double s1 = 0.0, s2 = 0.0;
+    for (int b = 0; b < blocks; ++b) {
+        s1 += partial[((size_t)b * 2 + 0) * c + ch];
+        s2 += partial[((size_t)b * 2 + 1) * c + ch];
+    }
+    o.dbeta[ch] = (float)s1;
+    if (o.dgamma) {
+        o.dgamma[ch] = (float)s2;
+        double r = rstd[ch], m = mean[ch];
+        double k1 = (double)gamma[ch] * r;
+        o.k1[ch] = (float)k1;
+        o.k2[ch] = (float)(k1 * (-s1 + s2 * m * r) / count);
+        o.k3[ch] = (float)(-k1 * s2 * r / count);
+    }
+}
+
+// ------------------------------------------------------------------ elementwise
+template <typename T, int V>
+__global__ void __launch_bounds__(256) ew_add_kernel(ValSrc a, ValSrc b, int act, size_t groups, int c, T* __restrict__ out, T* __restrict__ out2) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= groups) return;
+    size_t e = i * V;
+    int c0 = (int)(e % c);
+    float x[V], y[V];
+    ld_val_w<T, V>(a, e, c0, x);
+    if (b.p) {
+        ld_val_w<T, V>(b, e, c0, y);
+#pragma unroll
+        for (int q = 0; q < V; ++q) x[q] += y[q];
+    }
+#pragma unroll
+    for (int q = 0; q < V; ++q) x[q] = apply_act(x[q], act);
+    st_raw_w<T, V>(out, e, x);
+    if (out2) st_raw_w<T, V>(out2, e, x);
+}
+
+// mode 0: dst = d * [out_val > 0];  mode 1: dst = a + b
+template <typename T, int V>
+__global__ void __launch_bounds__(256) ew_flat_kernel(int mode, const T* __restrict__ a, const T* __restrict__ b, size_t groups, T* __restrict__ dst) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= groups) return;
+    float x[V], y[V];
+    ld_raw_w<T, V>(a, i * V, x);
+    ld_raw_w<T, V>(b, i * V, y);
+#pragma unroll
+    for (int q = 0; q < V; ++q) x[q] = mode == 0 ? (y[q] > 0.f ? x[q] : 0.f) : x[q] + y[q];
+    st_raw_w<T, V>(dst, i * V, x);
+}
+
+template <typename T> __global__ void gap_fwd_kernel(ValSrc x, int n, int hw, int c, T* __restrict__ out) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n * c) return;
+    int ch = i % c, s = i / c;
+    float acc = 0.f;
+    for (int p = 0; p < hw; ++p) acc += ld_val<T>(x, ((size_t)s * hw + p) * c + ch, ch);
+    out[i] = from_f<T>(acc / (float)hw);
+}
+
+template <typename T> __global__ void gap_bwd_kernel(const T* __restrict__ da, int n, int hw, int c, const T* addend, T* dx) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)n * hw * c) return;
+    int ch = (int)(i % c);
+    int s = (int)(i / ((size_t)hw * c));
+    float v = to_f<T>(da[(size_t)s * c + ch]) / (float)hw;
+    if (addend) v += to_f<T>(addend[i]);
+    dx[i] = from_f<T>(v);
+}
+
+// ------------------------------------------------------------------ parameters
+__global__ void accumulate_kernel(float* __restrict__ G, const float* __restrict__ g, size_t n4, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n4) {
+        float4 a = reinterpret_cast<float4*>(G)[i];
+        float4 b = reinterpret_cast<const float4*>(g)[i];
+        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        reinterpret_cast<float4*>(G)[i] = a;
+    } else {
+        size_t e = n4 * 4 + (i - n4);
+        if (e < n) G[e] += g[e];
+    }
+}
+
+__device__ __forceinline__ void sgd1(float& w, float& v, float& G, float inv_m, float lr, float mu) {
+    float g = G * inv_m;
+    v = fmaf(mu, v, g);
+    w = fmaf(-lr, v, w);
+    G = 0.f;
+}
+
+__global__ void sgd_step_kernel(float* __restrict__ w, float* __restrict__ v, float* __restrict__ G, size_t n4, size_t n, float inv_m, float lr,
+                                float mu) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n4) {
+        float4 a = reinterpret_cast<float4*>(w)[i], b = reinterpret_cast<float4*>(v)[i], c = reinterpret_cast<float4*>(G)[i];
+        sgd1(a.x, b.x, c.x, inv_m, lr, mu);
+        sgd1(a.y, b.y, c.y, inv_m, lr, mu);
+        sgd1(a.z, b.z, c.z, inv_m, lr, mu);
+        sgd1(a.w, b.w, c.w, inv_m, lr, mu);
+        reinterpret_cast<float4*>(w)[i] = a;
+        reinterpret_cast<float4*>(v)[i] = b;
+        reinterpret_cast<float4*>(G)[i] = c;
+    } else {
+        size_t e = n4 * 4 + (i - n4);
+        if (e < n) sgd1(w[e], v[e], G[e], inv_m, lr, mu);
+    }
+}
+
+__global__ void refresh_kernel(const float* __restrict__ w, const int32_t* __restrict__ perm, float* __restrict__ d, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) d[i] = w[perm[i]];
+}
+
+// ------------------------------------------------------------------ losses
+constexpr int LOSS_MAX_BLOCKS = 1024;
+
+__device__ __forceinline__ float block_sum(float v, float* sh) {
+    v = warp_sum(v);
+    int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) sh[wid] = v;
+    __syncthreads();
+    float r = 0.f;
+    if (wid == 0) {
+        r = lane < (blockDim.x >> 5) ? sh[lane] : 0.f;
+        r = warp_sum(r);
+    }
+    __syncthreads();
+    return r;   // valid in warp 0
+}
+
+__device__ __forceinline__ float block_max(float v, float* sh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) sh[wid] = v;
+    __syncthreads();
+    float r = sh[0];
+    for (int i = 1; i < (blockDim.x >> 5); ++i) r = fmaxf(r, sh[i]);
+    __syncthreads();
+    return r;
+}
+
+// The block that takes the last ticket sums the per-block partials in index order.
+__device__ void finish_loss(float part, float* scratch, unsigned* ticket, int nparts, float scale, float* loss, float* sh) {
+    __shared__ bool last;
+    if (threadIdx.x == 0) {
+        scratch[blockIdx.x] = part;
+        __threadfence();
+        unsigned t = atomicAdd(ticket, 1u);
+        last = (t == (unsigned)nparts - 1);
+    }
+    __syncthreads();
+    if (last) {
+        __threadfence();
+        float s = 0.f;
+        for (int i = threadIdx.x; i < nparts; i += blockDim.x) s += *((volatile float*)scratch + i);
+        s = block_sum(s, sh);
+        if (threadIdx.x == 0) {
+            *loss = s * scale;
+            *ticket = 0;
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) mse_kernel(const T* __restrict__ y, const T* __restrict__ t, size_t n, T* __restrict__ dy, float* loss,
+                                                  float* scratch, unsigned* ticket) {
+    __shared__ float sh[32];
+    float acc = 0.f;
+    const float k = 2.f / (float)n;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float d = to_f<T>(y[i]) - to_f<T>(t[i]);
+        acc = fmaf(d, d, acc);
+        dy[i] = from_f<T>(d * k);
+    }
+    float part = block_sum(acc, sh);
+    finish_loss(part, scratch, ticket, gridDim.x, 1.f / (float)n, loss, sh);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) xent_kernel(const T* __restrict__ logits, const int32_t* __restrict__ labels, int rows, int classes,
+                                                   T* __restrict__ dl, float* loss, float* scratch, unsigned* ticket) {
+    __shared__ float sh[32];
+    const int r = blockIdx.x;
+    const T* lg = logits + (size_t)r * classes;
+    float mx = -INFINITY;
+    for (int j = threadIdx.x; j < classes; j += blockDim.x) mx = fmaxf(mx, to_f<T>(lg[j]));
+    mx = block_max(mx, sh);
+    float se = 0.f;
+    for (int j = threadIdx.x; j < classes; j += blockDim.x) se += expf(to_f<T>(lg[j]) - mx);
+    se = block_sum(se, sh);
+    __shared__ float se_all;
+    if (threadIdx.x == 0) se_all = se;
+    __syncthreads();
+    se = se_all;
+    const int lab = labels[r];
+    const float inv_rows = 1.f / (float)rows;
+    for (int j = threadIdx.x; j < classes; j += blockDim.x) {
+        float p = expf(to_f<T>(lg[j]) - mx) / se;
+        dl[(size_t)r * classes + j] = from_f<T>((p - (j == lab ? 1.f : 0.f)) * inv_rows);
+    }
+    float part = logf(se) - (to_f<T>(lg[lab]) - mx);
+    finish_loss(part, scratch, ticket, rows, inv_rows, loss, sh);
+}
+
+}  // namespace
+
+// =================================================================== launchers
+void bn_stats(int dtype, const void* z, size_t pixels, int c, const float* gamma, const float* beta, float eps, float momentum, float* scratch,
+              size_t scratch_floats, const BnFwdOut& o, cudaStream_t st) {
+    ReducePlan p = plan_reduce(dtype, pixels, c, 2, scratch_floats);
+    StatsOp op{z};
+    launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_STATS, (double)pixels * c * esz(dtype), st);
+    LaunchScope ls(K_BN_STATS_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
+    if (dtype == 0)
+        bn_stats_finish<float><<<(c + 127) / 128, 128, 0, st>>>(scratch, (int)p.by, c, (const float*)z, (double)pixels, gamma, beta, eps, momentum, o);
+    else
+        bn_stats_finish<__nv_bfloat16><<<(c + 127) / 128, 128, 0, st>>>(scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
+                                                                       momentum, o);
+}
+
+void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int c, const float* scale, const float* shift, int act,
+                   const float* mean, const float* rstd, const float* gamma, float* scratch, size_t scratch_floats, const BnBwdOut& o,
+                   cudaStream_t st) {
+    ReducePlan p = plan_reduce(dtype, pixels, c, 2, scratch_floats);
+    BwdOp op{GradSrc{dy, z, scale, shift, nullptr, nullptr, nullptr, act}, mean, rstd};
+    launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_BWD_REDUCE, (double)pixels * c * esz(dtype) * ((act != ACT_NONE || mean) ? 2.0 : 1.0), st);
+    LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
+    bn_bwd_finish<<<(c + 127) / 128, 128, 0, st>>>(scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
+}
+
+template <typename T, int V> static void ew_add_launch(const ValSrc& a, const ValSrc& b, int act, size_t n, int c, void* out, void* out2, cudaStream_t st) {
+    size_t groups = n / V;
+    LaunchScope ls(K_EW_ADD, (double)n * sizeof(T) * (1 + (b.p ? 1 : 0) + 1 + (out2 ? 1 : 0)), (double)n, st);
+    ew_add_kernel<T, V><<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(a, b, act, groups, c, (T*)out, (T*)out2);
+}
+
+void ew_add(int dtype, const ValSrc& a, const ValSrc& b, int act, size_t pixels, int c, void* out, void* out2, cudaStream_t st) {
+    size_t n = pixels * c;
+    if (dtype == 0) {
+        if (c % 4 == 0) ew_add_launch<float, 4>(a, b, act, n, c, out, out2, st);
+        else ew_add_launch<float, 1>(a, b, act, n, c, out, out2, st);
+    } else {
+        if (c % 8 == 0) ew_add_launch<__nv_bfloat16, 8>(a, b, act, n, c, out, out2, st);
+        else ew_add_launch<__nv_bfloat16, 1>(a, b, act, n, c, out, out2, st);
+    }
+}
+
+void ew_apply(int dtype, const ValSrc& a, size_t pixels, int c, void* out, cudaStream_t st) {
+    ValSrc none{nullptr, nullptr, nullptr, 0};
+    ew_add(dtype, a, none, ACT_NONE, pixels, c, out, nullptr, st);
+}
+
+template <typename T, int V> static void ew_flat_launch(int mode, const void* a, const void* b, size_t n, void* dst, cudaStream_t st) {
+    size_t groups = n / V;
+    LaunchScope ls(mode == 0 ? K_EW_MASK : K_EW_SUM, 3.0 * n * sizeof(T), (double)n, st);
+    ew_flat_kernel<T, V><<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(mode, (const T*)a, (const T*)b, groups, (T*)dst);
+}
+
+static void ew_flat(int dtype, int mode, const void* a, const void* b, size_t n, void* dst, cudaStream_t st) {
+    if (dtype == 0) {
+        if (n % 4 == 0) ew_flat_launch<float, 4>(mode, a, b, n, dst, st);
+        else ew_flat_launch<float, 1>(mode, a, b, n, dst, st);
+    } else {
+        if (n % 8 == 0) ew_flat_launch<__nv_bfloat16, 8>(mode, a, b, n, dst, st);
+        else ew_flat_launch<__nv_bfloat16, 1>(mode, a, b, n, dst, st);
+    }
+}
+
+void ew_relu_mask(int dtype, const void* d, const void* out_val, size_t n, void* dst, cudaStream_t st) { ew_flat(dtype, 0, d, out_val, n, dst, st); }
+void ew_sum(int dtype, const void* a, const void* b, size_t n, void* dst, cudaStream_t st) { ew_flat(dtype, 1, a, b, n, dst, st); }
+
+void gap_fwd(int dtype, const ValSrc& x, int n, int hw, int c, void* out, cudaStream_t st) {
+    int total = n * c;
+    LaunchScope ls(K_GAP_FWD, ((double)total * hw + total) * esz(dtype), (double)total * hw, st);
+    if (dtype == 0) gap_fwd_kernel<float><<<(total + 127) / 128, 128, 0, st>>>(x, n, hw, c, (float*)out);
+    else gap_fwd_kernel<__nv_bfloat16><<<(total + 127) / 128, 128, 0, st>>>(x, n, hw, c, (__nv_bfloat16*)out);
+}
+
+void gap_bwd(int dtype, const void* da, int n, int hw, int c, const void* addend, void* dx, cudaStream_t st) {
+    size_t total = (size_t)n * hw * c;
+    unsigned blocks = (unsigned)((total + 255) / 256);
+    LaunchScope ls(K_GAP_BWD, (double)total * esz(dtype) * (addend ? 2.0 : 1.0), (double)total, st);
+    if (dtype == 0) gap_bwd_kernel<float><<<blocks, 256, 0, st>>>((const float*)da, n, hw, c, (const float*)addend, (float*)dx);
+    else gap_bwd_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)da, n, hw, c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx);
+}
+
+void accumulate(float* G, const float* g, size_t n, cudaStream_t st) {
+    if (!n) return;
+    size_t n4 = n / 4, threads = n4 + (n - n4 * 4);
+    LaunchScope ls(K_ACCUMULATE, 12.0 * n, (double)n, st);
+    accumulate_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(G, g, n4, n);
+}
+
+void sgd_step(float* w, float* v, float* G, size_t n, float inv_m, float lr, float mu, cudaStream_t st) {
+    if (!n) return;
+    size_t n4 = n / 4, threads = n4 + (n - n4 * 4);
+    LaunchScope ls(K_SGD_STEP, 24.0 * n, 5.0 * n, st);
+    sgd_step_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(w, v, G, n4, n, inv_m, lr, mu);
+}
+
+void refresh_derived(const float* w, const int32_t* perm, float* derived, size_t n, cudaStream_t st) {
+    if (!n) return;
+    LaunchScope ls(K_REFRESH, 12.0 * n, 0.0, st);
+    refresh_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w, perm, derived, n);
+}
+
+void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, cudaStream_t st) {
+    size_t want = (n + 256 * 8 - 1) / (256 * 8);
+    int blocks = (int)(want < 1 ? 1 : (want > LOSS_MAX_BLOCKS ? LOSS_MAX_BLOCKS : want));
+    unsigned* ticket = reinterpret_cast<unsigned*>(scratch + 65536);
+    LaunchScope ls(K_LOSS_MSE, 3.0 * n * esz(dtype), 4.0 * n, st);
+    if (dtype == 0) mse_kernel<float><<<blocks, 256, 0, st>>>((const float*)y, (const float*)t, n, (float*)dy, loss, scratch, ticket);
+    else mse_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)y, (const __nv_bfloat16*)t, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
+}
+
+void loss_xent(int dtype, const void* logits, const int32_t* labels, int rows, int classes, void* dlogits, float* loss, float* scratch,
+               cudaStream_t st) {
+    unsigned* ticket = reinterpret_cast<unsigned*>(scratch + 65536);
+    LaunchScope ls(K_LOSS_XENT, 2.0 * rows * classes * esz(dtype), 6.0 * rows * classes, st);
+    if (dtype == 0) xent_kernel<float><<<rows, 256, 0, st>>>((const float*)logits, labels, rows, classes, (float*)dlogits, loss, scratch, ticket);
+    else xent_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>((const __nv_bfloat16*)logits, labels, rows, classes, (__nv_bfloat16*)dlogits, loss, scratch, ticket);
+}
+
+}  // namespace ast

@@ -1,0 +1,81 @@
+// Host-side launchers of the stage kernels.  Every launcher only enqueues work on `st`.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace ast {
+
+struct ConvGeom {
+    int n, hi, wi, ci, ho, wo, co, k, stride, pad;
+};
+
+// Kernel kinds, for launch counting and the optional per-launch event trace.
+enum KernelKind {
+    K_CONV_FWD = 0, K_CONV_BWD_DATA, K_CONV_BWD_WEIGHT, K_REDUCE_SPLITS, K_DW_FWD, K_DW_BWD_DATA, K_DW_BWD_WEIGHT,
+    K_DW_BWD_WEIGHT_FINISH, K_BN_STATS, K_BN_STATS_FINISH, K_BN_BWD_REDUCE, K_BN_BWD_FINISH, K_EW_ADD, K_EW_MASK, K_EW_SUM,
+    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_KINDS
+};
+const char* kernel_name(int kind);
+
+// Brackets one kernel launch: counts it and, while a trace is active, records a CUDA event on
+// `st` before and after it together with the bytes the kernel must move (each tensor once)
+// and its floating-point operations.
+struct LaunchScope {
+    LaunchScope(int kind, double alg_bytes, double flops, cudaStream_t st);
+    ~LaunchScope();
+    int slot;
+    cudaStream_t st;
+};
+uint64_t launches();
+
+// ---- dense convolution as implicit GEMM (plain FFMA tiles; float and bfloat16 storage) ----
+// z[n,ho,wo,ko] = sum_{r,s,c} x[n,ho*st-pad+r,wo*st-pad+s,c] * w[ko][r][s][c]  (+ bias[ko])
+void conv_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w, const float* bias, void* z, cudaStream_t st);
+// dx[n,hi,wi,c] = sum_{r,s,ko} dz[n,(hi+pad-r)/st,(wi+pad-s)/st,ko] * wt[c][r][s][ko]  (+ addend)
+void conv_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* wt, const void* addend, void* dx, cudaStream_t st);
+// gw[ko][r][s][c] = sum_{n,ho,wo} dz[n,ho,wo,ko] * x[n,ho*st-pad+r,wo*st-pad+s,c]; split over pixels, partials in scratch
+void conv_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats,
+                     float* gw, cudaStream_t st);
+
+// ---- depthwise 3x3 (weights tap-major: w9c[r*3+s][c]) ----
+void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, cudaStream_t st);
+void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w9c, const void* addend, void* dx, cudaStream_t st);
+// gw[c][r][s]
+void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats,
+                   float* gw, cudaStream_t st);
+
+// ---- BatchNorm statistics and backward reductions over a [pixels][c] tensor ----
+struct BnFwdOut {
+    float *mean, *rstd, *scale, *shift, *run_mean, *run_var;
+};
+void bn_stats(int dtype, const void* z, size_t pixels, int c, const float* gamma, const float* beta, float eps, float momentum,
+              float* scratch, size_t scratch_floats, const BnFwdOut& o, cudaStream_t st);
+struct BnBwdOut {
+    float *dgamma, *dbeta, *k1, *k2, *k3;   // dgamma/k* null: only dbeta = sum of dpre (bias gradient)
+};
+void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int c, const float* scale, const float* shift, int act,
+                   const float* mean, const float* rstd, const float* gamma, float* scratch, size_t scratch_floats,
+                   const BnBwdOut& o, cudaStream_t st);
+
+// ---- elementwise over [pixels][c] ----
+void ew_add(int dtype, const ValSrc& a, const ValSrc& b, int act, size_t pixels, int c, void* out, void* out2, cudaStream_t st);
+void ew_apply(int dtype, const ValSrc& a, size_t pixels, int c, void* out, cudaStream_t st);
+void ew_relu_mask(int dtype, const void* d, const void* out_val, size_t n, void* dst, cudaStream_t st);
+void ew_sum(int dtype, const void* a, const void* b, size_t n, void* dst, cudaStream_t st);
+void gap_fwd(int dtype, const ValSrc& x, int n, int hw, int c, void* out, cudaStream_t st);
+void gap_bwd(int dtype, const void* da, int n, int hw, int c, const void* addend, void* dx, cudaStream_t st);
+
+// ---- parameters ----
+void accumulate(float* G, const float* g, size_t n, cudaStream_t st);
+void sgd_step(float* w, float* v, float* G, size_t n, float inv_m, float lr, float mu, cudaStream_t st);
+void refresh_derived(const float* w, const int32_t* perm, float* derived, size_t n, cudaStream_t st);
+
+// ---- losses (scratch: >= 1024 floats + 1 counter word) ----
+void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, cudaStream_t st);
+void loss_xent(int dtype, const void* logits, const int32_t* labels, int rows, int classes, void* dlogits, float* loss,
+               float* scratch, cudaStream_t st);
+
+}  // namespace ast

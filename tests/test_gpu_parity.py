@@ -1,0 +1,97 @@
+"""Parity of the CUDA library with the float64 oracle, through the C ABI, on seeded inputs.
+
+Tolerances (max|gpu-ref| / max|ref| per tensor): 1e-4 for float32 storage, 2e-2 for bfloat16
+storage with float32 accumulation.  With bfloat16 storage the ReLU/ReLU6 masks are decisions
+taken on stored (rounded) values, so the oracle takes them on the same values: it rounds at the
+library's storage points and keeps all arithmetic in float64."""
+import numpy as np
+import pytest
+
+import stage_inputs as si
+from harness import bf16_store, compare, gpu_round, make_inputs, oracle_round, sampled_round_check
+
+pytestmark = pytest.mark.gpu
+
+TOL = {False: 1e-4, True: 2e-2}
+
+SMALL = {
+    # name: (net, h, w, B, M, loss)
+    "block_ragged": (si.block_net(8, 3), 7, 5, 3, 2, "mse"),
+    "block_c16": (si.block_net(16, 6), 12, 12, 2, 2, "mse"),
+    "mbv2_4blocks_small": (si.stage_net_mbv2_4blocks(), 14, 14, 3, 2, "mse"),
+    "bottlenecks_small": (si.bottleneck_net(16, [(8, 32, 2, 1), (16, 64, 2, 2)]), 12, 12, 2, 2, "mse"),
+    "small_mobilenet_xent": (si.small_mobilenet(10)[0], 32, 32, 4, 2, "xent"),
+    "bnfree_block": (si.bnfree_net(8, 2), 9, 9, 2, 3, "mse"),
+}
+
+
+def run_case(net, h, w, B, M, loss, bf16, seed=0, first=0, last=None, **kw):
+    last = len(net) - 1 if last is None else last
+    xs, tg, params, _ = make_inputs(net, first, last, h, w, B, M, loss, seed, bf16)
+    outlier_frac = kw.pop("outlier_frac", 0.0)
+    deep = kw.pop("deep", False)     # bfloat16 stage of several blocks: see harness.compare
+    okw = {k: v for k, v in kw.items() if k in ("order", "rounds")}
+    ref = oracle_round(net, first, last, B, M, loss, xs, tg, params, store=bf16_store if bf16 else None, **okw)
+    pure = oracle_round(net, first, last, B, M, loss, xs, tg, params, **okw) if (bf16 and deep) else None
+    gpu = gpu_round(net, first, last, h, w, B, M, loss, xs, tg, params, bf16, **kw)
+    return compare(gpu, ref, net, first, last, TOL[bf16], need_dx=kw.get("need_dx", 1) != 0, outlier_frac=outlier_frac, pure=pure)
+
+
+@pytest.mark.parametrize("bf16", [False, True], ids=["f32", "bf16"])
+@pytest.mark.parametrize("name", list(SMALL))
+def test_small_stages(name, bf16):
+    net, h, w, B, M, loss = SMALL[name]
+    print(name, run_case(net, h, w, B, M, loss, bf16, deep=True))
+
+
+def test_config1_block_fp32():
+    """One inverted-residual block 16->96->16 at 32x32, micro-batch 8, M=4, float32, MSE."""
+    print(run_case(si.block_net(16, 6), 32, 32, 8, 4, "mse", False, outlier_frac=1e-3))
+
+
+def test_config1_two_rounds_momentum():
+    print(run_case(si.block_net(16, 6), 32, 32, 8, 4, "mse", False, rounds=2, outlier_frac=1e-3))
+
+
+def test_config2_stage_bf16_full_size():
+    """Four inverted-residual blocks at 56x56, micro-batch 32, M=8, bfloat16: the benchmarked workload
+    in the benchmark's launch configuration; the oracle evaluates micro-batches 0 and 7."""
+    print(sampled_round_check(si.stage_net_mbv2_4blocks(), 0, 34, 56, 56, 32, 8, "mse", True, [0, 7], 2e-2))
+
+
+def test_config3_mobilenetv2_bf16_full_size():
+    """Full MobileNetV2 at 224x224x3, softmax cross-entropy, M=4 micro-batches of 16; oracle on micro-batch 3."""
+    net = si.mobilenetv2_net()
+    print(sampled_round_check(net, 0, len(net) - 1, 224, 224, 16, 4, "xent", True, [3], 2e-2, need_dx=0))
+
+
+def test_config4_resnet_stage_bf16():
+    """ResNet-50 conv2_x+conv3_x at 56x56x64, M=8; micro-batch 8 instead of 32 bounds the oracle's time
+    (1.7 GMAC per sample); oracle on micro-batch 5."""
+    net = si.resnet50_c2c3_net()
+    print(sampled_round_check(net, 0, len(net) - 1, 56, 56, 8, 8, "mse", True, [5], 2e-2))
+
+
+def test_one_forward_one_backward_order_is_bit_identical():
+    net = si.block_net(16, 6)
+    M = 4
+    xs, tg, params, _ = make_inputs(net, 0, len(net) - 1, 16, 16, 4, M, "mse", 3, False)
+    a = gpu_round(net, 0, len(net) - 1, 16, 16, 4, M, "mse", xs, tg, params, False)
+    f1b = [("F", 0), ("F", 1), ("F", 2), ("B", 0), ("F", 3), ("B", 1), ("B", 2), ("B", 3)]
+    b = gpu_round(net, 0, len(net) - 1, 16, 16, 4, M, "mse", xs, tg, params, False, order=f1b, slots=3)
+    assert np.array_equal(a["G"], b["G"]) and np.array_equal(a["w"], b["w"])
+    for m in range(M):
+        assert np.array_equal(a["y"][m], b["y"][m]) and np.array_equal(a["dx"][m], b["dx"][m])
+    c = gpu_round(net, 0, len(net) - 1, 16, 16, 4, M, "mse", xs, tg, params, False)
+    assert np.array_equal(a["G"], c["G"])          # run-to-run determinism
+
+
+def test_partitioned_stages_compose():
+    """Config-5 style: a network cut at block boundaries, each stage run alone."""
+    net, units = si.small_mobilenet(10)
+    cuts = si.partition_units(net, units, 3, 32, 32)
+    shapes = si.out_shape(net, 0, len(net) - 1, 32, 32)
+    for first, last in cuts:
+        h, w, _ = shapes[first - 1] if first > 0 else (32, 32, 3)
+        loss = "xent" if last == len(net) - 1 else "mse"
+        print((first, last), run_case(net, h, w, 4, 2, loss, True, first=first, last=last, need_dx=int(first > 0), deep=True))
