@@ -133,16 +133,35 @@ void launch_reduce(int dtype, const ReducePlan& p, const OP& op, size_t pixels, 
     }
 }
 
-template <typename T>
-__global__ void bn_stats_finish(const float* __restrict__ partial, int blocks, int c, const T* __restrict__ z, double count,
-                                const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float momentum, BnFwdOut o) {
-    int ch = blockIdx.x * blockDim.x + threadIdx.x;
-    if (ch >= c) return;
-    double s1 = 0.0, s2 = 0.0;
-    for (int b = 0; b < blocks; ++b) {
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One warp per channel: lanes stride over the per-block partials (fixed assignment, fixed
+// shuffle tree: deterministic), sums in double.
+__device__ __forceinline__ void sum_partials(const float* __restrict__ partial, int blocks, int c, int ch, double& s1, double& s2) {
+    const int lane = threadIdx.x & 31;
+    s1 = 0.0;
+    s2 = 0.0;
+    for (int b = lane; b < blocks; b += 32) {
         s1 += partial[((size_t)b * 2 + 0) * c + ch];
         s2 += partial[((size_t)b * 2 + 1) * c + ch];
     }
+    s1 = warp_sum_d(s1);
+    s2 = warp_sum_d(s2);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128) bn_stats_finish(const float* __restrict__ partial, int blocks, int c, const T* __restrict__ z, double count,
+                                                       const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float momentum,
+                                                       BnFwdOut o) {
+    int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (ch >= c) return;
+    double s1, s2;
+    sum_partials(partial, blocks, c, ch, s1, s2);
+    if ((threadIdx.x & 31) != 0) return;
     double pivot = to_f<T>(z[ch]);
     double m1 = s1 / count;
     double mean = pivot + m1;
@@ -159,15 +178,14 @@ __global__ void bn_stats_finish(const float* __restrict__ partial, int blocks, i
     o.run_var[ch] = (float)((1.0 - momentum) * o.run_var[ch] + momentum * unbiased);
 }
 
-__global__ void bn_bwd_finish(const float* __restrict__ partial, int blocks, int c, double count, const float* __restrict__ mean,
-                              const float* __restrict__ rstd, const float* __restrict__ gamma, BnBwdOut o) {
-    int ch = blockIdx.x * blockDim.x + threadIdx.x;
+__global__ void __launch_bounds__(128) bn_bwd_finish(const float* __restrict__ partial, int blocks, int c, double count,
+                                                     const float* __restrict__ mean, const float* __restrict__ rstd,
+                                                     const float* __restrict__ gamma, BnBwdOut o) {
+    int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (ch >= c) return;
-    double s1 = 0.0, s2 = 0.0;
-    for (int b = 0; b < blocks; ++b) {
-        s1 += partial[((size_t)b * 2 + 0) * c + ch];
-        s2 += partial[((size_t)b * 2 + 1) * c + ch];
-    }
+    double s1, s2;
+    sum_partials(partial, blocks, c, ch, s1, s2);
+    if ((threadIdx.x & 31) != 0) return;
     o.dbeta[ch] = (float)s1;
     if (o.dgamma) {
         o.dgamma[ch] = (float)s2;
@@ -377,9 +395,9 @@ void bn_stats(int dtype, const void* z, size_t pixels, int c, const float* gamma
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_STATS, (double)pixels * c * esz(dtype), st);
     LaunchScope ls(K_BN_STATS_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
     if (dtype == 0)
-        bn_stats_finish<float><<<(c + 127) / 128, 128, 0, st>>>(scratch, (int)p.by, c, (const float*)z, (double)pixels, gamma, beta, eps, momentum, o);
+        bn_stats_finish<float><<<(c + 3) / 4, 128, 0, st>>>(scratch, (int)p.by, c, (const float*)z, (double)pixels, gamma, beta, eps, momentum, o);
     else
-        bn_stats_finish<__nv_bfloat16><<<(c + 127) / 128, 128, 0, st>>>(scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
+        bn_stats_finish<__nv_bfloat16><<<(c + 3) / 4, 128, 0, st>>>(scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
                                                                        momentum, o);
 }
 
@@ -390,7 +408,7 @@ void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int 
     BwdOp op{GradSrc{dy, z, scale, shift, nullptr, nullptr, nullptr, act}, mean, rstd};
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_BWD_REDUCE, (double)pixels * c * esz(dtype) * ((act != ACT_NONE || mean) ? 2.0 : 1.0), st);
     LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
-    bn_bwd_finish<<<(c + 127) / 128, 128, 0, st>>>(scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
+    bn_bwd_finish<<<(c + 3) / 4, 128, 0, st>>>(scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
 }
 
 template <typename T, int V> static void ew_add_launch(const ValSrc& a, const ValSrc& b, int act, size_t n, int c, void* out, void* out2, cudaStream_t st) {
