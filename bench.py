@@ -119,7 +119,7 @@ def time_oracle(batch, steps, warmup):
     from harness import bf16_store
     net, first, last = workload()
     xs, ts, params, _ = make_host_inputs(0, batch, 1)
-    st = O.Stage(net, first, last, batch, 1, params, store=bf16_store)
+    st = O.Stage(net, first, last, batch, 1, params, store=bf16_store, operand=bf16_store)
     times = []
     for it in range(warmup + steps):
         t0 = time.perf_counter()

@@ -42,9 +42,14 @@ class Stage:
     the pooled features, the stage output, and the gradient with respect to each of those
     stored-or-recomputed unit outputs and to the stage input (rounded after every term added
     to it).  BatchNorm and activation outputs inside a conv->BN->activation chain are never
-    stored.  store=None is the plain float64 definition."""
+    stored.  store=None is the plain float64 definition.
 
-    def __init__(self, net, first, last, micro_batch, n_micro, params, eps=1e-5, bn_momentum=0.1, store=None):
+    `operand`: optional rounding applied to both operands of every dense contraction (conv and
+    linear layers, in FP, in the input-gradient product and in the weight-gradient product; not the
+    depthwise conv), modelling tensor-core inputs of reduced precision with exact products and wide
+    accumulation.  operand=None keeps float64 operands."""
+
+    def __init__(self, net, first, last, micro_batch, n_micro, params, eps=1e-5, bn_momentum=0.1, store=None, operand=None):
         if not (0 <= first <= last < len(net)):
             raise ValueError("bad layer range")
         self.net, self.first, self.last = net, first, last
@@ -68,6 +73,7 @@ class Stage:
         self.saved = {}          # micro-batch -> {layer index: output}, caches
         self.n_accumulated = 0
         self.store = store
+        self.operand = operand if operand is not None else (lambda t: t)
 
     def _chains_into_next(self, i):
         """True if layer i+1 continues layer i's chain (conv->BN, conv/BN->activation, add->ReLU),
@@ -122,7 +128,7 @@ class Stage:
             ly = net[i]
             a = val[ly.src]
             if ly.op == "conv":
-                val[i] = L.conv2d_forward(a, self.p[(i, "weight")], ly.stride, ly.pad)
+                val[i] = L.conv2d_forward(self.operand(a), self.operand(self.p[(i, "weight")]), ly.stride, ly.pad)
             elif ly.op == "dwconv":
                 val[i] = L.dwconv2d_forward(a, self.p[(i, "weight")], ly.stride, ly.pad)
             elif ly.op == "bn":
@@ -139,7 +145,7 @@ class Stage:
             elif ly.op == "gap":
                 val[i] = L.gap_forward(a)
             elif ly.op == "linear":
-                val[i] = L.linear_forward(a.reshape(a.shape[0], -1), self.p[(i, "weight")],
+                val[i] = L.linear_forward(self.operand(a.reshape(a.shape[0], -1)), self.operand(self.p[(i, "weight")]),
                                           self.p[(i, "bias")]).reshape(a.shape[0], 1, 1, -1)
             else:
                 raise ValueError(ly.op)
@@ -165,7 +171,8 @@ class Stage:
             d = grad.pop(i)
             a = val[ly.src]
             if ly.op == "conv":
-                dx, g[(i, "weight")] = L.conv2d_backward(a, self.p[(i, "weight")], d, ly.stride, ly.pad)
+                dx, g[(i, "weight")] = L.conv2d_backward(self.operand(a), self.operand(self.p[(i, "weight")]), self.operand(d),
+                                                         ly.stride, ly.pad)
                 give(ly.src, dx)
             elif ly.op == "dwconv":
                 dx, g[(i, "weight")] = L.dwconv2d_backward(a, self.p[(i, "weight")], d, ly.stride, ly.pad)
@@ -182,8 +189,9 @@ class Stage:
                 give(ly.src, L.gap_backward(d, a.shape[1], a.shape[2]))
             elif ly.op == "linear":
                 a2 = a.reshape(a.shape[0], -1)
-                da, g[(i, "weight")], g[(i, "bias")] = L.linear_backward(a2, self.p[(i, "weight")],
-                                                                          d.reshape(a.shape[0], -1))
+                d2 = d.reshape(a.shape[0], -1)
+                da, g[(i, "weight")], _ = L.linear_backward(self.operand(a2), self.operand(self.p[(i, "weight")]), self.operand(d2))
+                g[(i, "bias")] = d2.sum(axis=0)
                 give(ly.src, da.reshape(a.shape))
         self.g = g
         return grad[self.first - 1]

@@ -288,9 +288,16 @@ __global__ void sgd_step_kernel(float* __restrict__ w, float* __restrict__ v, fl
     }
 }
 
-__global__ void refresh_kernel(const float* __restrict__ w, const int32_t* __restrict__ perm, float* __restrict__ d, size_t n) {
+__global__ void refresh_kernel(const float* __restrict__ w, const int32_t* __restrict__ perm, float* __restrict__ d,
+                               __nv_bfloat16* __restrict__ wb, __nv_bfloat16* __restrict__ wtb, size_t n) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) d[i] = w[perm[i]];
+    if (i >= n) return;
+    float t = w[perm[i]];
+    d[i] = t;
+    if (wb) {
+        wb[i] = __float2bfloat16_rn(w[i]);
+        wtb[i] = __float2bfloat16_rn(t);
+    }
 }
 
 // ------------------------------------------------------------------ losses
@@ -481,10 +488,10 @@ void sgd_step(float* w, float* v, float* G, size_t n, float inv_m, float lr, flo
     sgd_step_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(w, v, G, n4, n, inv_m, lr, mu);
 }
 
-void refresh_derived(const float* w, const int32_t* perm, float* derived, size_t n, cudaStream_t st) {
+void refresh_derived(const float* w, const int32_t* perm, float* derived, __nv_bfloat16* wb, __nv_bfloat16* wtb, size_t n, cudaStream_t st) {
     if (!n) return;
-    LaunchScope ls(K_REFRESH, 12.0 * n, 0.0, st);
-    refresh_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w, perm, derived, n);
+    LaunchScope ls(K_REFRESH, (wb ? 20.0 : 12.0) * n, 0.0, st);
+    refresh_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w, perm, derived, wb, wtb, n);
 }
 
 void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, cudaStream_t st) {

@@ -43,6 +43,11 @@ __device__ __forceinline__ bool tap_out(const ConvGeom& g, int hi, int wi, int r
     return ho < g.ho && wo < g.wo;
 }
 
+// Operands of a dense contraction are bf16 values in bfloat16 mode (the tensor-core input
+// format), whichever kernel executes the layer; accumulation is float32.
+template <typename T> __device__ __forceinline__ float operand(float v) { return v; }
+template <> __device__ __forceinline__ float operand<__nv_bfloat16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
 template <typename T, int MODE> __global__ void __launch_bounds__(NT) igemm_kernel(const IgemmArgs a) {
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
@@ -109,8 +114,8 @@ template <typename T, int MODE> __global__ void __launch_bounds__(NT) igemm_kern
                     int nb = n0 + tid / 4;
                     if (nb < a.N) vb = __ldg(a.w + (size_t)nb * a.K + kk);
                 }
-                As[kl][tid / 4] = va;
-                Bs[kl][tid / 4] = vb;
+                As[kl][tid / 4] = operand<T>(va);
+                Bs[kl][tid / 4] = operand<T>(vb);
             }
         } else {
             int kl = tid / 16, p = k0 + kl;
@@ -132,8 +137,8 @@ template <typename T, int MODE> __global__ void __launch_bounds__(NT) igemm_kern
                     if (jb_r[j] >= 0 && tap_in(g, ph, pw, jb_r[j], jb_s[j], h2, w2))
                         vb = ld_val<T>(a.x, ((size_t)(pn * g.hi + h2) * g.wi + w2) * g.ci + jb_c[j], jb_c[j]);
                 }
-                As[kl][ml] = va;
-                Bs[kl][ml] = vb;
+                As[kl][ml] = operand<T>(va);
+                Bs[kl][ml] = operand<T>(vb);
             }
         }
         __syncthreads();

@@ -16,7 +16,7 @@ struct ConvGeom {
 enum KernelKind {
     K_CONV_FWD = 0, K_CONV_BWD_DATA, K_CONV_BWD_WEIGHT, K_REDUCE_SPLITS, K_DW_FWD, K_DW_BWD_DATA, K_DW_BWD_WEIGHT,
     K_DW_BWD_WEIGHT_FINISH, K_BN_STATS, K_BN_STATS_FINISH, K_BN_BWD_REDUCE, K_BN_BWD_FINISH, K_EW_ADD, K_EW_MASK, K_EW_SUM,
-    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_KINDS
+    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_KINDS
 };
 const char* kernel_name(int kind);
 
@@ -39,6 +39,12 @@ void conv_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float*
 // gw[ko][r][s][c] = sum_{n,ho,wo} dz[n,ho,wo,ko] * x[n,ho*st-pad+r,wo*st-pad+s,c]; split over pixels, partials in scratch
 void conv_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats,
                      float* gw, cudaStream_t st);
+
+// ---- pointwise conv on tcgen05 tensor cores (bf16 storage, channel counts multiples of 8) ----
+bool pw_tc_supported(int dtype, const ConvGeom& g, bool bwd_data);
+// wb: bf16 weights [co][ci]; wtb: bf16 transposed weights [ci][co]; err: device error word
+void pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const float* bias, void* z, int* err, cudaStream_t st);
+void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st);
 
 // ---- depthwise 3x3 (weights tap-major: w9c[r*3+s][c]) ----
 void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, cudaStream_t st);
@@ -71,7 +77,8 @@ void gap_bwd(int dtype, const void* da, int n, int hw, int c, const void* addend
 // ---- parameters ----
 void accumulate(float* G, const float* g, size_t n, cudaStream_t st);
 void sgd_step(float* w, float* v, float* G, size_t n, float inv_m, float lr, float mu, cudaStream_t st);
-void refresh_derived(const float* w, const int32_t* perm, float* derived, size_t n, cudaStream_t st);
+// derived[i] = w[perm[i]]; wb[i] = bf16(w[i]); wtb[i] = bf16(w[perm[i]])  (wb/wtb may be null)
+void refresh_derived(const float* w, const int32_t* perm, float* derived, __nv_bfloat16* wb, __nv_bfloat16* wtb, size_t n, cudaStream_t st);
 
 // ---- losses (scratch: >= 1024 floats + 1 counter word) ----
 void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, cudaStream_t st);

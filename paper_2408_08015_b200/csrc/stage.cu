@@ -79,6 +79,8 @@ struct asteroid_stage {
     // device arenas
     float *w = nullptr, *v = nullptr, *G = nullptr, *g = nullptr, *derived = nullptr, *run = nullptr, *coef = nullptr, *scratch = nullptr;
     int32_t* perm = nullptr;
+    __nv_bfloat16 *wb = nullptr, *wtb = nullptr;   // bf16 copies of the weights and of the derived (transposed) weights
+    int* err = nullptr;                            // device error word (bounded waits)
     char *slot_mem = nullptr, *grad_mem = nullptr;
     size_t slot_bytes = 0, slot_stat_off = 0, grad_bytes = 0, scratch_floats = 0;
     size_t bytes_mod = 0, bytes_opt = 0, bytes_work = 0;
@@ -293,6 +295,7 @@ static void free_stage(asteroid_stage* s) {
     for (auto e : s->tm.ev) cudaEventDestroy(e);
     cudaFree(s->w); cudaFree(s->v); cudaFree(s->G); cudaFree(s->g); cudaFree(s->derived); cudaFree(s->run);
     cudaFree(s->coef); cudaFree(s->scratch); cudaFree(s->perm); cudaFree(s->slot_mem); cudaFree(s->grad_mem);
+    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err);
     delete s;
 }
 
@@ -355,7 +358,9 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
         void* obuf = sv.base + o.buf_off;
         tick(s, ui, 0, st);
         if (u.kind == U_CONV) {
-            conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, u.b_off >= 0 ? s->w + u.b_off : nullptr, obuf, st);
+            const float* bias = u.b_off >= 0 ? s->w + u.b_off : nullptr;
+            if (pw_tc_supported(dt, u.g, false)) pw_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, bias, obuf, s->err, st);
+            else conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, bias, obuf, st);
         } else if (u.kind == U_DW) {
             dw_fwd(dt, u.g, val_src(s, sv, u.in), s->derived + u.w_off, obuf, st);
         } else if (u.kind == U_ADD) {
@@ -437,7 +442,8 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             if (want_in) {
                 GradState& gi = gs[u.in];
                 const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
-                if (u.kind == U_CONV) conv_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
+                if (u.kind == U_CONV && pw_tc_supported(dt, u.g, true)) pw_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
+                else if (u.kind == U_CONV) conv_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 else dw_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 gi.state = G_OWNED;
                 gi.ptr = own(u.in);
@@ -493,6 +499,11 @@ static int create_impl(const ast_layer* net, int n_layers, int first, int last, 
     if ((rc = dev_alloc(&s->derived, np * 4, &mod))) return rc;
     if ((rc = dev_alloc(&s->perm, np * 4, &mod))) return rc;
     if ((rc = dev_alloc(&s->run, s->n_run * 4, &mod))) return rc;
+    if (s->dtype == AST_BF16) {
+        if ((rc = dev_alloc(&s->wb, np * 2, &mod))) return rc;
+        if ((rc = dev_alloc(&s->wtb, np * 2, &mod))) return rc;
+    }
+    if ((rc = dev_alloc(&s->err, 256, &work))) return rc;
     if ((rc = dev_alloc(&s->v, np * 4, &opt))) return rc;
     if ((rc = dev_alloc(&s->slot_mem, s->slot_bytes * s->slots, &act))) return rc;
     if ((rc = dev_alloc(&s->grad_mem, s->grad_bytes, &work))) return rc;
@@ -563,7 +574,7 @@ int asteroid_stage_import_state(asteroid_stage* s, const float* params, const fl
         if (momentum) CU(cudaMemcpy(s->v, momentum, n * 4, cudaMemcpyHostToDevice));
         else CU(cudaMemset(s->v, 0, n * 4));
         CU(cudaMemset(s->G, 0, n * 4));
-        refresh_derived(s->w, s->perm, s->derived, n, 0);
+        refresh_derived(s->w, s->perm, s->derived, s->wb, s->wtb, n, 0);
     }
     int rc = reset_bn_running(s);
     if (rc) return rc;
@@ -577,6 +588,12 @@ int asteroid_stage_export_state(asteroid_stage* s, float* params, float* momentu
     if (!s) return fail(AST_ERR_ARG, "null argument");
     if (n != s->n_params) return fail(AST_ERR_ARG, "state has %zu values, the stage has %zu parameters", n, s->n_params);
     CU(cudaDeviceSynchronize());
+    int errw = 0;
+    CU(cudaMemcpy(&errw, s->err, sizeof errw, cudaMemcpyDeviceToHost));
+    if (errw) {
+        CU(cudaMemset(s->err, 0, sizeof errw));
+        return fail(AST_ERR_TIMEOUT, "a bounded device-side wait expired in a tensor-core kernel; results of this round are invalid");
+    }
     if (n) {
         if (params) CU(cudaMemcpy(params, s->w, n * 4, cudaMemcpyDeviceToHost));
         if (momentum) CU(cudaMemcpy(momentum, s->v, n * 4, cudaMemcpyDeviceToHost));
@@ -651,7 +668,7 @@ int asteroid_stage_step(asteroid_stage* s, float lr, float momentum, void* strea
     if (s->n_acc != s->M) return fail(AST_ERR_ORDER, "step after %d of %d micro-batches accumulated", s->n_acc, s->M);
     cudaStream_t st = (cudaStream_t)stream;
     sgd_step(s->w, s->v, s->G, s->n_params, 1.f / (float)s->M, lr, momentum, st);
-    refresh_derived(s->w, s->perm, s->derived, s->n_params, st);
+    refresh_derived(s->w, s->perm, s->derived, s->wb, s->wtb, s->n_params, st);
     CU(cudaGetLastError());
     s->n_acc = 0;
     return AST_OK;
@@ -707,6 +724,10 @@ int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_pr
         if (s->n_params) {
             CU(cudaMemcpy(t->w, s->w, s->n_params * 4, cudaMemcpyDeviceToDevice));
             CU(cudaMemcpy(t->derived, s->derived, s->n_params * 4, cudaMemcpyDeviceToDevice));
+            if (s->wb) {
+                CU(cudaMemcpy(t->wb, s->wb, s->n_params * 2, cudaMemcpyDeviceToDevice));
+                CU(cudaMemcpy(t->wtb, s->wtb, s->n_params * 2, cudaMemcpyDeviceToDevice));
+            }
         }
         const Val &vi = t->vals[0], &vo = t->vals.back();
         char *x = nullptr, *y = nullptr, *dy = nullptr, *dx = nullptr;

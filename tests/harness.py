@@ -23,14 +23,15 @@ def default_order(M):
 
 
 def bf16_store(a):
-    """Rounding applied at storage points when mirroring bfloat16 activation storage."""
+    """Rounding applied at storage points, and to the operands of dense contractions, when mirroring
+    bfloat16 activation storage with bfloat16 tensor-core inputs."""
     return si.round_to_bf16(np.asarray(a, np.float32)).astype(np.float64)
 
 
 def oracle_round(net, first, last, B, M, loss, xs, tg, params, lr=0.01, mu=0.9, order=None, momentum0=None, rounds=1,
                  store=None):
     import oracle as O
-    st = O.Stage(net, first, last, B, M, params, store=store)
+    st = O.Stage(net, first, last, B, M, params, store=store, operand=store)
     if momentum0 is not None:
         off = 0
         for k in st.v:
