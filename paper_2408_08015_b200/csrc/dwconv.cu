@@ -1,53 +1,180 @@
-// Depthwise 3x3 convolution, NHWC, 16-byte channel vectors: forward, backward-data and
-// backward-weight.  All three are bandwidth-bound; the producer's BatchNorm+activation
-// (forward) and the BatchNorm-backward transform of the incoming gradient (backward) are
-// applied while loading, so no normalised tensor is ever written.
+// Depthwise 3x3 convolution, NHWC: forward, backward-data and backward-weight.
+//
+// All three are bandwidth-bound.  A thread owns V consecutive channels (one 16- or 8-byte
+// vector) and a horizontal strip of TW output pixels: the per-channel BatchNorm / activation
+// coefficients of the producer (forward) or the BatchNorm-backward coefficients (backward) are
+// loaded once into registers and applied to every vector on load, an input row is loaded once
+// and reused by the three taps and the TW outputs it feeds, and no normalised tensor or dz
+// tensor is ever written.  Lanes run along channel vectors, so a warp reads whole pixels.
 #include "kernels.h"
 
 namespace ast {
 namespace {
 
-// One thread per (pixel, channel vector).  Consecutive threads take consecutive channel
-// vectors of a pixel, then the next pixel of the row: loads are fully coalesced and the 3x3
-// neighbourhood is shared through L1.
-template <typename T> __global__ void __launch_bounds__(256) dw_fwd_kernel(ConvGeom g, ValSrc x, const float* __restrict__ w9c, T* __restrict__ z) {
-    constexpr int V = Vec<T>::N;
-    const int cv = g.ci / V;
-    size_t total = (size_t)g.n * g.ho * g.wo * cv;
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    int j = (int)(i % cv);
-    size_t p = i / cv;
-    int wo = (int)(p % g.wo);
-    size_t t = p / g.wo;
-    int ho = (int)(t % g.ho), n = (int)(t / g.ho);
-    int c0 = j * V;
-    float acc[V];
-#pragma unroll
-    for (int q = 0; q < V; ++q) acc[q] = 0.f;
-#pragma unroll
-    for (int r = 0; r < 3; ++r) {
-        int hi = ho * g.stride - 1 + r;
-        if (hi < 0 || hi >= g.hi) continue;
-#pragma unroll
-        for (int s = 0; s < 3; ++s) {
-            int wi = wo * g.stride - 1 + s;
-            if (wi < 0 || wi >= g.wi) continue;
-            float xv[V];
-            ld_val_vec<T>(x, ((size_t)(n * g.hi + hi) * g.wi + wi) * cv + j, c0, xv);
-            const float* wp = w9c + (r * 3 + s) * g.ci + c0;
-#pragma unroll
-            for (int q = 0; q < V; ++q) acc[q] = fmaf(xv[q], __ldg(wp + q), acc[q]);
-        }
+constexpr int TW = 4;
+
+// ---- V-wide raw access: (float,4) and (bf16,8) are 16-byte, (bf16,4) 8-byte ----
+template <typename T, int V> struct Raw;
+template <> struct Raw<float, 4> {
+    static __device__ __forceinline__ void ld(const void* p, size_t e, float* f) {
+        float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + e);
+        f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
     }
-    Vec<T> o;
-    o.pack(acc);
-    o.store(z, i);
+    static __device__ __forceinline__ void st(void* p, size_t e, const float* f) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(p) + e) = make_float4(f[0], f[1], f[2], f[3]);
+    }
+};
+template <> struct Raw<__nv_bfloat16, 8> {
+    static __device__ __forceinline__ void ld(const void* p, size_t e, float* f) {
+        Vec<__nv_bfloat16> v;
+        v.load(p, e >> 3);
+        v.unpack(f);
+    }
+    static __device__ __forceinline__ void st(void* p, size_t e, const float* f) {
+        Vec<__nv_bfloat16> v;
+        v.pack(f);
+        v.store(p, e >> 3);
+    }
+};
+template <> struct Raw<__nv_bfloat16, 4> {
+    static __device__ __forceinline__ void ld(const void* p, size_t e, float* f) {
+        uint2 v = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(p) + e);
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    }
+};
+
+template <int V> __device__ __forceinline__ void ld_coef(const float* p, int c0, float* out) {
+#pragma unroll
+    for (int q = 0; q < V; q += 4) {
+        float4 v = __ldg(reinterpret_cast<const float4*>(p + c0 + q));
+        out[q] = v.x; out[q + 1] = v.y; out[q + 2] = v.z; out[q + 3] = v.w;
+    }
 }
 
-template <typename T>
+// Reads a forward value: act(raw*scale + shift) with the coefficients held in registers.
+template <typename T, int V> struct ValLoader {
+    const void* p;
+    float scale[V], shift[V];
+    bool affine;
+    int act;
+    __device__ __forceinline__ ValLoader(const ValSrc& s, int c0) : p(s.p), affine(s.scale != nullptr), act(s.act) {
+        if (affine) {
+            ld_coef<V>(s.scale, c0, scale);
+            ld_coef<V>(s.shift, c0, shift);
+        }
+    }
+    __device__ __forceinline__ void load(size_t e, float* f) const {
+        Raw<T, V>::ld(p, e, f);
+        if (affine) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) f[q] = fmaf(f[q], scale[q], shift[q]);
+        }
+        if (act != ACT_NONE) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) f[q] = apply_act(f[q], act);
+        }
+    }
+};
+
+// Reads dz = k1*(dy*mask(pre)) + k2 + k3*z with the coefficients held in registers.
+template <typename T, int V> struct GradLoader {
+    const void* dy;
+    const void* z;
+    float scale[V], shift[V], k1[V], k2[V], k3[V];
+    bool affine, bn, need_z;
+    int act;
+    __device__ __forceinline__ GradLoader(const GradSrc& s, int c0)
+        : dy(s.dy), z(s.z), affine(s.scale != nullptr), bn(s.k1 != nullptr), need_z(s.act != ACT_NONE || s.k1 != nullptr), act(s.act) {
+        if (affine) {
+            ld_coef<V>(s.scale, c0, scale);
+            ld_coef<V>(s.shift, c0, shift);
+        }
+        if (bn) {
+            ld_coef<V>(s.k1, c0, k1);
+            ld_coef<V>(s.k2, c0, k2);
+            ld_coef<V>(s.k3, c0, k3);
+        }
+    }
+    __device__ __forceinline__ void load(size_t e, float* f) const {
+        Raw<T, V>::ld(dy, e, f);
+        if (!need_z) return;
+        float zz[V];
+        Raw<T, V>::ld(z, e, zz);
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            float pre = affine ? fmaf(zz[q], scale[q], shift[q]) : zz[q];
+            float d = f[q] * act_mask(pre, act);
+            f[q] = bn ? fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q])) : d;
+        }
+    }
+};
+
+// out[n,ho,wo,c] = sum_{r,s} in[n, ho*S-1+r, wo*S-1+s, c] * w[(FLIP ? 8-(3r+s) : 3r+s)][c]  (+ addend)
+// Forward: in = x (ValLoader), S = stride.  Backward-data at stride 1: in = dz (GradLoader), FLIP.
+template <typename T, int V, int S, bool FLIP, typename LOADER, typename SRC>
+__global__ void __launch_bounds__(256) dw_strip_kernel(int n_img, int hi, int wi, int ho, int wo, int c, SRC src, const float* __restrict__ w9c,
+                                                       const T* addend, T* out) {
+    constexpr int NIN = (TW - 1) * S + 3;
+    const int cv = c / V, sw = (wo + TW - 1) / TW;
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)n_img * ho * sw * cv) return;
+    const int j = (int)(idx % cv);
+    size_t sidx = idx / cv;
+    const int wo0 = (int)(sidx % sw) * TW;
+    size_t t2 = sidx / sw;
+    const int oh = (int)(t2 % ho), n = (int)(t2 / ho);
+    const int c0 = j * V;
+    LOADER ld(src, c0);
+    float acc[TW][V];
+#pragma unroll
+    for (int t = 0; t < TW; ++t)
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[t][q] = 0.f;
+    const int wi0 = wo0 * S - 1;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const int ih = oh * S - 1 + r;
+        if (ih < 0 || ih >= hi) continue;
+        float xin[NIN][V];
+        const size_t rowbase = ((size_t)n * hi + ih) * wi;
+#pragma unroll
+        for (int q2 = 0; q2 < NIN; ++q2) {
+            const int iw = wi0 + q2;
+            if (iw >= 0 && iw < wi) {
+                ld.load((rowbase + iw) * c + c0, xin[q2]);
+            } else {
+#pragma unroll
+                for (int q = 0; q < V; ++q) xin[q2][q] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            float wv[V];
+            ld_coef<V>(w9c + (FLIP ? 8 - (r * 3 + s) : r * 3 + s) * c, c0, wv);
+#pragma unroll
+            for (int t = 0; t < TW; ++t)
+#pragma unroll
+                for (int q = 0; q < V; ++q) acc[t][q] = fmaf(xin[t * S + s][q], wv[q], acc[t][q]);
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < TW; ++t) {
+        if (wo0 + t >= wo) break;
+        size_t e = (((size_t)n * ho + oh) * wo + wo0 + t) * c + c0;
+        if (addend) {
+            float ad[V];
+            Raw<T, V>::ld(addend, e, ad);
+#pragma unroll
+            for (int q = 0; q < V; ++q) acc[t][q] += ad[q];
+        }
+        Raw<T, V>::st(out, e, acc[t]);
+    }
+}
+
+// Backward-data at stride 2 (general form): one thread per input pixel and channel vector.
+template <typename T, int V>
 __global__ void __launch_bounds__(256) dw_bwd_data_kernel(ConvGeom g, GradSrc dz, const float* __restrict__ w9c, const T* addend, T* dx) {
-    constexpr int V = Vec<T>::N;
     const int cv = g.ci / V;
     size_t total = (size_t)g.n * g.hi * g.wi * cv;
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -58,11 +185,10 @@ __global__ void __launch_bounds__(256) dw_bwd_data_kernel(ConvGeom g, GradSrc dz
     size_t t = p / g.wi;
     int hi = (int)(t % g.hi), n = (int)(t / g.hi);
     int c0 = j * V;
+    GradLoader<T, V> ld(dz, c0);
     float acc[V];
     if (addend) {
-        Vec<T> a;
-        a.load(addend, i);
-        a.unpack(acc);
+        Raw<T, V>::ld(addend, p * g.ci + c0, acc);
     } else {
 #pragma unroll
         for (int q = 0; q < V; ++q) acc[q] = 0.f;
@@ -79,59 +205,78 @@ __global__ void __launch_bounds__(256) dw_bwd_data_kernel(ConvGeom g, GradSrc dz
             if (b < 0 || (g.stride == 2 && (b & 1))) continue;
             int wo = b / g.stride;
             if (wo >= g.wo) continue;
-            float dv[V];
-            ld_grad_vec<T>(dz, ((size_t)(n * g.ho + ho) * g.wo + wo) * cv + j, c0, dv);
-            const float* wp = w9c + (r * 3 + s) * g.ci + c0;
+            float dv[V], wv[V];
+            ld.load((((size_t)n * g.ho + ho) * g.wo + wo) * g.ci + c0, dv);
+            ld_coef<V>(w9c + (r * 3 + s) * g.ci, c0, wv);
 #pragma unroll
-            for (int q = 0; q < V; ++q) acc[q] = fmaf(dv[q], __ldg(wp + q), acc[q]);
+            for (int q = 0; q < V; ++q) acc[q] = fmaf(dv[q], wv[q], acc[q]);
         }
     }
-    Vec<T> o;
-    o.pack(acc);
-    o.store(dx, i);
+    Raw<T, V>::st(dx, p * g.ci + c0, acc);
 }
 
-// Weight gradient: per channel, nine sums over all output pixels.  A block owns `cw` channel
-// vectors and a contiguous range of output pixels; a thread keeps its 9*V partial sums in
-// registers, rows of the block are combined through shared memory, blocks through a partials
-// array summed in fixed order by a second kernel (deterministic, no float atomics).
-template <typename T>
-__global__ void __launch_bounds__(256) dw_bwd_weight_kernel(ConvGeom g, GradSrc dz, ValSrc x, int cw, int rows, size_t pix_per_block,
+// Weight gradient: gw[c][r][s] = sum over output pixels of dz * x(tap).  A block owns `cw`
+// channel vectors; thread (row, jl) walks output strips with stride `rows`, keeping 9*V sums
+// in registers.  Rows are combined through shared memory, blocks through a partials array
+// summed in fixed order by a second kernel (deterministic, no float atomics).
+template <typename T, int V, int S>
+__global__ void __launch_bounds__(256) dw_bwd_weight_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, int cw, int rows, size_t strips_per_block,
                                                             float* __restrict__ partial) {
-    constexpr int V = Vec<T>::N;
-    extern __shared__ float red[];      // [rows][cw*V] per tap, reused tap by tap
+    constexpr int NIN = (TW - 1) * S + 3;
+    extern __shared__ float red[];
     const int cv = g.ci / V;
     const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
     const int j = blockIdx.x * cw + jl;
     const bool active = row < rows && j < cv;
-    const int c0 = j * V;
-    size_t P = (size_t)g.n * g.ho * g.wo;
-    size_t pbeg = (size_t)blockIdx.y * pix_per_block, pend = min(P, pbeg + pix_per_block);
+    const int c0 = active ? j * V : 0;
+    const int sw = (g.wo + TW - 1) / TW;
+    const size_t n_strips = (size_t)g.n * g.ho * sw;
+    const size_t sbeg = (size_t)blockIdx.y * strips_per_block, send = min(n_strips, sbeg + strips_per_block);
     float acc[9][V];
 #pragma unroll
     for (int t = 0; t < 9; ++t)
 #pragma unroll
         for (int q = 0; q < V; ++q) acc[t][q] = 0.f;
     if (active) {
-        for (size_t p = pbeg + row; p < pend; p += rows) {
-            int wo = (int)(p % g.wo);
-            size_t t2 = p / g.wo;
-            int ho = (int)(t2 % g.ho), n = (int)(t2 / g.ho);
-            float dv[V];
-            ld_grad_vec<T>(dz, p * cv + j, c0, dv);
+        GradLoader<T, V> ldz(dzs, c0);
+        ValLoader<T, V> ldx(xs, c0);
+        for (size_t sidx = sbeg + row; sidx < send; sidx += rows) {
+            const int wo0 = (int)(sidx % sw) * TW;
+            size_t t2 = sidx / sw;
+            const int oh = (int)(t2 % g.ho), n = (int)(t2 / g.ho);
+            float dv[TW][V];
+#pragma unroll
+            for (int t = 0; t < TW; ++t) {
+                if (wo0 + t < g.wo) {
+                    ldz.load((((size_t)n * g.ho + oh) * g.wo + wo0 + t) * g.ci + c0, dv[t]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < V; ++q) dv[t][q] = 0.f;
+                }
+            }
+            const int wi0 = wo0 * S - 1;
 #pragma unroll
             for (int r = 0; r < 3; ++r) {
-                int hi = ho * g.stride - 1 + r;
-                if (hi < 0 || hi >= g.hi) continue;
+                const int ih = oh * S - 1 + r;
+                if (ih < 0 || ih >= g.hi) continue;
+                float xin[NIN][V];
+                const size_t rowbase = ((size_t)n * g.hi + ih) * g.wi;
 #pragma unroll
-                for (int s = 0; s < 3; ++s) {
-                    int wi = wo * g.stride - 1 + s;
-                    if (wi < 0 || wi >= g.wi) continue;
-                    float xv[V];
-                    ld_val_vec<T>(x, ((size_t)(n * g.hi + hi) * g.wi + wi) * cv + j, c0, xv);
+                for (int q2 = 0; q2 < NIN; ++q2) {
+                    const int iw = wi0 + q2;
+                    if (iw >= 0 && iw < g.wi) {
+                        ldx.load((rowbase + iw) * g.ci + c0, xin[q2]);
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < V; ++q) acc[r * 3 + s][q] = fmaf(dv[q], xv[q], acc[r * 3 + s][q]);
+                        for (int q = 0; q < V; ++q) xin[q2][q] = 0.f;
+                    }
                 }
+#pragma unroll
+                for (int s = 0; s < 3; ++s)
+#pragma unroll
+                    for (int t = 0; t < TW; ++t)
+#pragma unroll
+                        for (int q = 0; q < V; ++q) acc[r * 3 + s][q] = fmaf(dv[t][q], xin[t * S + s][q], acc[r * 3 + s][q]);
             }
         }
     }
@@ -143,84 +288,102 @@ __global__ void __launch_bounds__(256) dw_bwd_weight_kernel(ConvGeom g, GradSrc 
         }
         __syncthreads();
         for (int e = threadIdx.x; e < width; e += blockDim.x) {
-            int c = blockIdx.x * width + e;
-            if (c < g.ci) {
+            int ch = blockIdx.x * width + e;
+            if (ch < g.ci) {
                 float s = 0.f;
                 for (int r2 = 0; r2 < rows; ++r2) s += red[r2 * width + e];
-                partial[((size_t)blockIdx.y * 9 + t) * g.ci + c] = s;
+                partial[((size_t)blockIdx.y * 9 + t) * g.ci + ch] = s;
             }
         }
         __syncthreads();
     }
 }
 
-// gw[c][t] = sum_b partial[b][t][c]
-__global__ void dw_bwd_weight_finish(const float* __restrict__ partial, int blocks, int c_total, float* __restrict__ gw) {
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
+// gw[c][t] = sum_b partial[b][t][c]; one warp per (t, c): lanes stride over the blocks
+__global__ void __launch_bounds__(128) dw_bwd_weight_finish(const float* __restrict__ partial, int blocks, int c_total, float* __restrict__ gw) {
+    int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (i >= 9 * c_total) return;
     int t = i / c_total, c = i % c_total;
     float s = 0.f;
-    for (int b = 0; b < blocks; ++b) s += partial[((size_t)b * 9 + t) * c_total + c];
-    gw[c * 9 + t] = s;
+    for (int b = threadIdx.x & 31; b < blocks; b += 32) s += partial[((size_t)b * 9 + t) * c_total + c];
+    s = warp_sum(s);
+    if ((threadIdx.x & 31) == 0) gw[c * 9 + t] = s;
+}
+
+double esz(int dtype) { return dtype == 0 ? 4.0 : 2.0; }
+double grad_src_bytes(const GradSrc& d, double elems, int dtype) { return elems * esz(dtype) * ((d.act != ACT_NONE || d.k1) ? 2.0 : 1.0); }
+
+template <typename T, int V, int S, bool FLIP, typename LOADER, typename SRC>
+void launch_strip(int n, int hi, int wi, int ho, int wo, int c, const SRC& src, const float* w9c, const void* addend, void* out, cudaStream_t st) {
+    size_t total = (size_t)n * ho * ((wo + TW - 1) / TW) * (c / V);
+    dw_strip_kernel<T, V, S, FLIP, LOADER, SRC><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(n, hi, wi, ho, wo, c, src, w9c, (const T*)addend, (T*)out);
 }
 
 }  // namespace
 
-static double esz(int dtype) { return dtype == 0 ? 4.0 : 2.0; }
-static double grad_src_bytes(const GradSrc& d, double elems, int dtype) { return elems * esz(dtype) * ((d.act != ACT_NONE || d.k1) ? 2.0 : 1.0); }
-
 void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, cudaStream_t st) {
     double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
     LaunchScope ls(K_DW_FWD, (in_e + out_e) * esz(dtype) + 36.0 * g.ci, 18.0 * out_e, st);
+    using B = __nv_bfloat16;
     if (dtype == 0) {
-        size_t total = (size_t)g.n * g.ho * g.wo * (g.ci / 4);
-        dw_fwd_kernel<float><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, x, w9c, (float*)z);
+        if (g.stride == 1) launch_strip<float, 4, 1, false, ValLoader<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
+        else launch_strip<float, 4, 2, false, ValLoader<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     } else {
-        size_t total = (size_t)g.n * g.ho * g.wo * (g.ci / 8);
-        dw_fwd_kernel<__nv_bfloat16><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, x, w9c, (__nv_bfloat16*)z);
+        if (g.stride == 1) launch_strip<B, 8, 1, false, ValLoader<B, 8>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
+        else launch_strip<B, 8, 2, false, ValLoader<B, 8>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     }
 }
 
 void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w9c, const void* addend, void* dx, cudaStream_t st) {
     double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
     LaunchScope ls(K_DW_BWD_DATA, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) * (addend ? 2.0 : 1.0) + 36.0 * g.ci, 18.0 * out_e, st);
-    if (dtype == 0) {
+    using B = __nv_bfloat16;
+    if (g.stride == 1) {
+        // the adjoint of a stride-1 3x3 correlation is the correlation of dz with the flipped kernel
+        if (dtype == 0) launch_strip<float, 4, 1, true, GradLoader<float, 4>, GradSrc>(g.n, g.ho, g.wo, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
+        else launch_strip<B, 8, 1, true, GradLoader<B, 8>, GradSrc>(g.n, g.ho, g.wo, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
+    } else if (dtype == 0) {
         size_t total = (size_t)g.n * g.hi * g.wi * (g.ci / 4);
-        dw_bwd_data_kernel<float><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const float*)addend, (float*)dx);
+        dw_bwd_data_kernel<float, 4><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const float*)addend, (float*)dx);
     } else {
         size_t total = (size_t)g.n * g.hi * g.wi * (g.ci / 8);
-        dw_bwd_data_kernel<__nv_bfloat16><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx);
+        dw_bwd_data_kernel<B, 8><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const B*)addend, (B*)dx);
     }
 }
 
 void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw,
                    cudaStream_t st) {
-    const int V = dtype == 0 ? 4 : 8;
+    const int V = 4;
     const int cv = g.ci / V;
-    int cw = cv < 32 ? cv : 32;
+    int cw = cv < 64 ? cv : 64;
     int rows = 256 / cw;
-    size_t P = (size_t)g.n * g.ho * g.wo;
+    const int sw = (g.wo + TW - 1) / TW;
+    size_t n_strips = (size_t)g.n * g.ho * sw;
     int gx = (cv + cw - 1) / cw;
     size_t by = (4 * 148 + gx - 1) / gx;
-    size_t max_by = (P + (size_t)rows * 4 - 1) / ((size_t)rows * 4);
+    size_t max_by = (n_strips + (size_t)rows * 2 - 1) / ((size_t)rows * 2);
     if (by > max_by) by = max_by;
     size_t cap = scratch_floats / ((size_t)9 * g.ci);
     if (by > cap) by = cap;
     if (by < 1) by = 1;
-    size_t ppb = (P + by - 1) / by;
-    by = (P + ppb - 1) / ppb;
+    size_t spb = (n_strips + by - 1) / by;
+    by = (n_strips + spb - 1) / spb;
     size_t smem = (size_t)rows * cw * V * sizeof(float);
     dim3 grid(gx, (unsigned)by);
-    double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)P * g.ci;
+    double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
+    using B = __nv_bfloat16;
     {
         LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
-        if (dtype == 0)
-            dw_bwd_weight_kernel<float><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, ppb, scratch);
-        else
-            dw_bwd_weight_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, ppb, scratch);
+        if (dtype == 0) {
+            if (g.stride == 1) dw_bwd_weight_kernel<float, 4, 1><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
+            else dw_bwd_weight_kernel<float, 4, 2><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
+        } else {
+            if (g.stride == 1) dw_bwd_weight_kernel<B, 4, 1><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
+            else dw_bwd_weight_kernel<B, 4, 2><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
+        }
     }
     LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
-    dw_bwd_weight_finish<<<(9 * g.ci + 255) / 256, 256, 0, st>>>(scratch, (int)by, g.ci, gw);
+    dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
 }
 
 }  // namespace ast
