@@ -260,6 +260,174 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
     if (warp == 0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Weight gradient of a pointwise conv:  gw[k][c] = sum_p dz[p][k] * x[p][c].
+// D[128 x N] (rows = output channels k, columns = input channels c) accumulates in tensor memory
+// over the CTA's pixel range; the reduction dimension is the pixel, so both operands are read
+// exactly as they lie in global memory ([pixel][channel]) and staged MN-major: a stage holds 64
+// pixels as rows of 128 bytes (64 channels) per channel panel, 8-row groups 1024 bytes apart
+// (stride-dimension offset), panels 8192 bytes apart (leading-dimension offset), 16-byte chunks
+// XOR-swizzled with the row index.  Two stage buffers: the MMAs of one stage run while the next
+// is being loaded and transformed.  Rows/columns beyond the valid channels hold stale data and
+// only feed accumulator rows/columns that are never read; pixel rows beyond the range are zeroed.
+constexpr int WSTAGE = 64;                 // pixels per stage
+constexpr int PANEL = WSTAGE * 128;        // bytes of one 64-channel panel of a stage
+
+struct PwWArgs {
+    GradSrc dz;
+    ValSrc x;
+    float* partial;        // [splits][CO][CI]
+    int* err;
+    int P, CO, CI;         // output pixels, output channels, input channels
+    int pix_per_cta;       // multiple of WSTAGE
+    int NT;                // input channels per CTA (multiple of 16, <= 256)
+    int tmem_cols;
+    int stride, ho, wo, hi, wi;
+};
+
+__device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(PANEL >> 4) << 16;     // leading-dimension offset: next 64-channel panel
+    d |= (uint64_t)(1024 >> 4) << 32;      // stride-dimension offset: next group of 8 pixels
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+__global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t mbar_store[2];
+    __shared__ uint32_t tmem_slot;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * TM;                    // first output channel of this CTA
+    const int n0 = blockIdx.z * a.NT;                  // first input channel
+    const int ca = min(TM, a.CO - m0) >> 3;            // 16-byte chunks per pixel of the A operand
+    const int cb = min(a.NT, a.CI - n0) >> 3;
+    const int pa = (ca + 7) >> 3, pb = (cb + 7) >> 3;  // 64-channel panels
+    const int nb_panels = (a.NT + 63) >> 6;
+    const uint32_t buf_bytes = (uint32_t)(2 + nb_panels) * PANEL;
+    const int pbeg = blockIdx.y * a.pix_per_cta, pend = min(a.P, pbeg + a.pix_per_cta);
+    const uint32_t mbar0 = smem_u32(&mbar_store[0]), mbar1 = smem_u32(&mbar_store[1]);
+
+    if (tid == 0) {
+        mbar_init(mbar0, 1);
+        mbar_init(mbar1, 1);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), (uint32_t)a.tmem_cols);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    // D = f32, A = B = bf16, both MN-major (bits 15, 16)
+    const uint32_t idesc = make_idesc(a.NT) | (1u << 15) | (1u << 16);
+
+    uint32_t ph[2] = {0, 0};
+    int issued[2] = {0, 0};
+    bool ok = true, bad = false;       // `bad` is decided by a block-wide vote: uniform across threads
+    int stage = 0;
+    for (int ps = pbeg; ps < pend; ps += WSTAGE, ++stage) {
+        const int b = stage & 1;
+        uint8_t* sA = base + (size_t)b * buf_bytes;
+        uint8_t* sB = sA + 2 * PANEL;
+        if (issued[b]) {                               // the MMAs that read this buffer two stages ago
+            ok = mbar_wait(b ? mbar1 : mbar0, ph[b]);
+            ph[b] ^= 1;
+        }
+        if (!__syncthreads_and(ok ? 1 : 0)) {
+            bad = true;
+            break;
+        }
+        const int valid = min(WSTAGE, pend - ps);
+        for (int v = tid; v < WSTAGE * ca; v += NTHREADS) {
+            int kr = v / ca, j = v - kr * ca;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (kr < valid) {
+                float f[8];
+                int c0 = m0 + (j << 3);
+                ld_grad_vec<__nv_bfloat16>(a.dz, ((size_t)(ps + kr) * a.CO + c0) >> 3, c0, f);
+                q = pack8(f);
+            }
+            *reinterpret_cast<uint4*>(sA + (j >> 3) * PANEL + kr * 128 + (((j & 7) ^ (kr & 7)) << 4)) = q;
+        }
+        for (int v = tid; v < WSTAGE * cb; v += NTHREADS) {
+            int kr = v / cb, j = v - kr * cb;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (kr < valid) {
+                float f[8];
+                int c0 = n0 + (j << 3);
+                size_t pin = ps + kr;
+                if (a.stride > 1) {
+                    int p = ps + kr;
+                    int wo = p % a.wo, t = p / a.wo;
+                    int ho = t % a.ho, n = t / a.ho;
+                    pin = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
+                }
+                ld_val_vec<__nv_bfloat16>(a.x, (pin * a.CI + c0) >> 3, c0, f);
+                q = pack8(f);
+            }
+            *reinterpret_cast<uint4*>(sB + (j >> 3) * PANEL + kr * 128 + (((j & 7) ^ (kr & 7)) << 4)) = q;
+        }
+        fence_async_smem();
+        __syncthreads();
+        if (tid == 0) {
+            fence_after_sync();
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+#pragma unroll
+            for (int s = 0; s < WSTAGE / 16; ++s)      // 16 pixels = two 8-row groups per MMA
+                umma_bf16(tmem, make_desc_mn(a0 + s * 2048), make_desc_mn(b0 + s * 2048), idesc, (stage > 0 || s > 0) ? 1u : 0u);
+            umma_commit(b ? mbar1 : mbar0);
+        }
+        issued[b] = 1;
+    }
+    // drain: the last commit covers every earlier MMA of the issuing thread
+    if (!bad && stage > 0) {
+        const int lb = (stage - 1) & 1;
+        ok = mbar_wait(lb ? mbar1 : mbar0, ph[lb]);
+        if (!__syncthreads_and(ok ? 1 : 0)) bad = true;
+    }
+    fence_after_sync();
+    __syncthreads();
+    if (bad) {
+        if (tid == 0) atomicExch(a.err, 1);
+    } else {
+        const int q = warp & 3, half = warp >> 2;
+        const int row = q * 32 + lane, k = m0 + row;
+        float* dst = a.partial + ((size_t)blockIdx.y * a.CO + (size_t)(k < a.CO ? k : 0)) * a.CI;
+        for (int g = half; g < (a.NT >> 3); g += 2) {
+            float v[8];
+            if (stage > 0) {
+                tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g << 3), v);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = 0.f;
+            }
+            int c = n0 + (g << 3);
+            if (k < a.CO && c < a.CI) {
+                *reinterpret_cast<float4*>(dst + c) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4*>(dst + c + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            }
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+    (void)pa; (void)pb;
+}
+
+__global__ void reduce_splits_tc(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float s = 0.f;
+    for (int k = 0; k < splits; ++k) s += partial[(size_t)k * n + i];
+    out[i] = s;
+}
+
 struct Tiling {
     int NT, ntiles, KC, tmem_cols;
     size_t smem;
@@ -317,6 +485,45 @@ void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* w
     double bytes = 2.0 * (double)a.P * a.K * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * (double)a.P * a.N * (addend ? 2.0 : 1.0) +
                    2.0 * a.N * a.K;
     launch<true>(a, t, K_PW_BWD_DATA_TC, bytes, st);
+}
+
+void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
+                      cudaStream_t st) {
+    PwWArgs a{};
+    a.dz = dz; a.x = x; a.partial = scratch; a.err = err;
+    a.P = g.n * g.ho * g.wo; a.CO = g.co; a.CI = g.ci;
+    a.stride = g.stride; a.ho = g.ho; a.wo = g.wo; a.hi = g.hi; a.wi = g.wi;
+    int ntiles = (a.CI + 255) / 256;
+    a.NT = ((a.CI + ntiles - 1) / ntiles + 15) / 16 * 16;
+    ntiles = (a.CI + a.NT - 1) / a.NT;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < a.NT) a.tmem_cols <<= 1;
+    int mtiles = (a.CO + TM - 1) / TM;
+    size_t out_elems = (size_t)a.CO * a.CI;
+    int splits = (2 * 148 + mtiles * ntiles - 1) / (mtiles * ntiles);
+    int max_by_pix = (a.P + 4 * WSTAGE - 1) / (4 * WSTAGE);
+    if (splits > max_by_pix) splits = max_by_pix;
+    size_t cap = scratch_floats / out_elems;
+    if ((size_t)splits > cap) splits = (int)cap;
+    if (splits < 1) splits = 1;
+    int ppc = (a.P + splits - 1) / splits;
+    ppc = (ppc + WSTAGE - 1) / WSTAGE * WSTAGE;
+    splits = (a.P + ppc - 1) / ppc;
+    a.pix_per_cta = ppc;
+    size_t smem = (size_t)2 * (2 + (a.NT + 63) / 64) * PANEL + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(pw_bwd_weight_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        attr_set = true;
+    }
+    double bytes = 2.0 * (double)a.P * a.CO * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * (double)g.n * g.hi * g.wi * a.CI +
+                   4.0 * out_elems * splits;
+    {
+        LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * a.P * a.CO * a.CI, st);
+        pw_bwd_weight_tc_kernel<<<dim3(mtiles, splits, ntiles), NTHREADS, smem, st>>>(a);
+    }
+    LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (splits + 1), (double)out_elems * splits, st);
+    reduce_splits_tc<<<(unsigned)((out_elems + 255) / 256), 256, 0, st>>>(scratch, splits, out_elems, gw);
 }
 
 }  // namespace ast
