@@ -300,7 +300,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--m-override", type=int, default=0,
+                    help="profiling captures only: run M' micro-batches per step instead of 8 (smaller device footprint); not a benchmark configuration")
     args = ap.parse_args()
+    if args.m_override > 0:
+        global M, WORKLOAD
+        M = args.m_override
+        WORKLOAD += " [profiling capture with M=%d]" % M
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -42,6 +42,11 @@ template <> struct Raw<__nv_bfloat16, 4> {
         f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
         f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
     }
+    static __device__ __forceinline__ void st(void* p, size_t e, const float* f) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]), b = __floats2bfloat162_rn(f[2], f[3]);
+        uint2 v = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p) + e) = v;
+    }
 };
 
 template <int V> __device__ __forceinline__ void ld_coef(const float* p, int c0, float* out) {
@@ -113,7 +118,7 @@ template <typename T, int V> struct GradLoader {
 // out[n,ho,wo,c] = sum_{r,s} in[n, ho*S-1+r, wo*S-1+s, c] * w[(FLIP ? 8-(3r+s) : 3r+s)][c]  (+ addend)
 // Forward: in = x (ValLoader), S = stride.  Backward-data at stride 1: in = dz (GradLoader), FLIP.
 template <typename T, int V, int S, bool FLIP, typename LOADER, typename SRC>
-__global__ void __launch_bounds__(256) dw_strip_kernel(int n_img, int hi, int wi, int ho, int wo, int c, SRC src, const float* __restrict__ w9c,
+__global__ void __launch_bounds__(128) dw_strip_kernel(int n_img, int hi, int wi, int ho, int wo, int c, SRC src, const float* __restrict__ w9c,
                                                        const T* addend, T* out) {
     constexpr int NIN = (TW - 1) * S + 3;
     const int cv = c / V, sw = (wo + TW - 1) / TW;
@@ -132,21 +137,21 @@ __global__ void __launch_bounds__(256) dw_strip_kernel(int n_img, int hi, int wi
 #pragma unroll
         for (int q = 0; q < V; ++q) acc[t][q] = 0.f;
     const int wi0 = wo0 * S - 1;
+    // Halo positions outside the image read a clamped (valid) address and are zeroed afterwards:
+    // the body stays straight-line code, so all loads of the three rows can be in flight together.
 #pragma unroll
     for (int r = 0; r < 3; ++r) {
         const int ih = oh * S - 1 + r;
-        if (ih < 0 || ih >= hi) continue;
+        const bool row_ok = ih >= 0 && ih < hi;
         float xin[NIN][V];
-        const size_t rowbase = ((size_t)n * hi + ih) * wi;
+        const size_t rowbase = ((size_t)n * hi + min(max(ih, 0), hi - 1)) * wi;
 #pragma unroll
         for (int q2 = 0; q2 < NIN; ++q2) {
             const int iw = wi0 + q2;
-            if (iw >= 0 && iw < wi) {
-                ld.load((rowbase + iw) * c + c0, xin[q2]);
-            } else {
+            const bool ok = row_ok && iw >= 0 && iw < wi;
+            ld.load((rowbase + min(max(iw, 0), wi - 1)) * c + c0, xin[q2]);
 #pragma unroll
-                for (int q = 0; q < V; ++q) xin[q2][q] = 0.f;
-            }
+            for (int q = 0; q < V; ++q) xin[q2][q] = ok ? xin[q2][q] : 0.f;
         }
 #pragma unroll
         for (int s = 0; s < 3; ++s) {
@@ -316,7 +321,7 @@ double grad_src_bytes(const GradSrc& d, double elems, int dtype) { return elems 
 template <typename T, int V, int S, bool FLIP, typename LOADER, typename SRC>
 void launch_strip(int n, int hi, int wi, int ho, int wo, int c, const SRC& src, const float* w9c, const void* addend, void* out, cudaStream_t st) {
     size_t total = (size_t)n * ho * ((wo + TW - 1) / TW) * (c / V);
-    dw_strip_kernel<T, V, S, FLIP, LOADER, SRC><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(n, hi, wi, ho, wo, c, src, w9c, (const T*)addend, (T*)out);
+    dw_strip_kernel<T, V, S, FLIP, LOADER, SRC><<<(unsigned)((total + 127) / 128), 128, 0, st>>>(n, hi, wi, ho, wo, c, src, w9c, (const T*)addend, (T*)out);
 }
 
 }  // namespace
@@ -329,8 +334,8 @@ void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, voi
         if (g.stride == 1) launch_strip<float, 4, 1, false, ValLoader<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
         else launch_strip<float, 4, 2, false, ValLoader<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     } else {
-        if (g.stride == 1) launch_strip<B, 8, 1, false, ValLoader<B, 8>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
-        else launch_strip<B, 8, 2, false, ValLoader<B, 8>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
+        if (g.stride == 1) launch_strip<B, 4, 1, false, ValLoader<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
+        else launch_strip<B, 4, 2, false, ValLoader<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     }
 }
 
@@ -341,7 +346,7 @@ void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w
     if (g.stride == 1) {
         // the adjoint of a stride-1 3x3 correlation is the correlation of dz with the flipped kernel
         if (dtype == 0) launch_strip<float, 4, 1, true, GradLoader<float, 4>, GradSrc>(g.n, g.ho, g.wo, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
-        else launch_strip<B, 8, 1, true, GradLoader<B, 8>, GradSrc>(g.n, g.ho, g.wo, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
+        else launch_strip<B, 4, 1, true, GradLoader<B, 4>, GradSrc>(g.n, g.ho, g.wo, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
     } else if (dtype == 0) {
         size_t total = (size_t)g.n * g.hi * g.wi * (g.ci / 4);
         dw_bwd_data_kernel<float, 4><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const float*)addend, (float*)dx);
