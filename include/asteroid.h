@@ -140,6 +140,19 @@ int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_pr
 /* Loss heads (used by the last stage and by tests).  All pointers are DEVICE pointers.
  * MSE: *loss = mean((y-t)^2) over n elements, dy = 2 (y-t) / n. */
 int asteroid_loss_mse(const void* y, const void* target, size_t n, int dtype, void* dy, float* loss, void* stream);
+/* The same MSE head for callers that must not allocate device memory (the paper has no counterpart;
+ * this serves hosts that run the round inside a fixed memory budget, a memory pool that forbids
+ * cudaMalloc after start-up, or a region where allocation is illegal).  asteroid_loss_mse obtains
+ * its reduction scratch with cudaMalloc on first use; this variant keeps the scratch (4.25 KB: one
+ * partial sum per block and a ticket word) in a static device array inside the library, which every
+ * GPU context that loads the library holds until the process exits.  It never calls cudaMalloc,
+ * cudaFree or any allocating routine.
+ *  - n must not exceed 67 108 864 elements (AST_ERR_ARG with a message otherwise).
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress) with
+ *    that device current; make that first call before starting any stream capture.
+ *  - All calls on a device share the one array: each call clears the ticket word on `stream` before
+ *    its kernel, and two calls whose kernels may overlap on the GPU (different streams) race. */
+int asteroid_loss_mse_noalloc(const void* y, const void* target, size_t n, int dtype, void* dy, float* loss, void* stream);
 /* Softmax cross-entropy: *loss = mean_r(-log softmax(logits_r)[labels_r]),
  * dlogits = (softmax - onehot) / rows.  rows <= 65536. */
 int asteroid_loss_softmax_xent(const void* logits, const int32_t* labels, int rows, int classes, int dtype,

@@ -13,7 +13,7 @@ EXPORTS = ["asteroid_stage_create", "asteroid_stage_destroy", "asteroid_stage_pa
            "asteroid_stage_output_elems", "asteroid_stage_import_state", "asteroid_stage_export_state",
            "asteroid_stage_export_bn_running", "asteroid_stage_forward", "asteroid_stage_backward",
            "asteroid_stage_accumulate", "asteroid_stage_step", "asteroid_stage_profile",
-           "asteroid_loss_mse", "asteroid_loss_softmax_xent", "asteroid_trace_start", "asteroid_trace_stop",
+           "asteroid_loss_mse", "asteroid_loss_mse_noalloc", "asteroid_loss_softmax_xent", "asteroid_trace_start", "asteroid_trace_stop",
            "asteroid_launch_count", "asteroid_last_error"]
 
 
@@ -72,6 +72,7 @@ def lib():
         L.asteroid_stage_step.argtypes = [vp, f, f, vp]
         L.asteroid_stage_profile.argtypes = [vp, i, i, C.POINTER(ast_layer_profile)]
         L.asteroid_loss_mse.argtypes = [vp, vp, sz, i, vp, vp, vp]
+        L.asteroid_loss_mse_noalloc.argtypes = [vp, vp, sz, i, vp, vp, vp]
         L.asteroid_loss_softmax_xent.argtypes = [vp, vp, i, i, i, vp, vp, vp]
         L.asteroid_trace_start.argtypes = []
         L.asteroid_trace_stop.argtypes = [C.POINTER(ast_kernel_stat), i, C.POINTER(i)]
@@ -162,6 +163,11 @@ def asteroid_stage_profile(h, layer, batch):
 
 def asteroid_loss_mse(y_ptr, t_ptr, n, dtype, dy_ptr, loss_ptr, stream=0):
     _check(lib().asteroid_loss_mse(y_ptr, t_ptr, n, dtype, dy_ptr, loss_ptr, stream))
+
+
+def asteroid_loss_mse_noalloc(y_ptr, t_ptr, n, dtype, dy_ptr, loss_ptr, stream=0):
+    """MSE head that performs no device allocation (static scratch inside the library; n <= 2**26)."""
+    _check(lib().asteroid_loss_mse_noalloc(y_ptr, t_ptr, n, dtype, dy_ptr, loss_ptr, stream))
 
 
 def asteroid_loss_softmax_xent(logits_ptr, labels_ptr, rows, classes, dtype, dlogits_ptr, loss_ptr, stream=0):

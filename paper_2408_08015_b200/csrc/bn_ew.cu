@@ -512,3 +512,46 @@ void loss_xent(int dtype, const void* logits, const int32_t* labels, int rows, i
 }
 
 }  // namespace ast
+
+// =================================================================== allocation-free MSE head
+namespace ast {
+namespace {
+constexpr size_t NOALLOC_MAX_ELEMS = (size_t)1 << 26;
+// Scratch of the allocation-free MSE head: one partial sum per block, then the ticket word.
+// Lives in every GPU context that loads the library, until the process exits.
+static __device__ __align__(256) float g_noalloc_scratch[LOSS_MAX_BLOCKS + 64];
+// Device address of the array per device ordinal; the array's name is only a host-side handle,
+// the address a kernel can use comes from cudaGetSymbolAddress with that device current.
+float* g_noalloc_ptr[64] = {};
+}  // namespace
+}  // namespace ast
+
+extern "C" int asteroid_loss_mse_noalloc(const void* y, const void* target, size_t n, int dtype, void* dy, float* loss, void* stream) {
+    using namespace ast;
+    if (!y || !target || !dy || !loss || n == 0) return report_error(-1, "asteroid_loss_mse_noalloc: null or empty argument");
+    if (dtype != 0 && dtype != 1) return report_error(-1, "asteroid_loss_mse_noalloc: bad dtype");
+    if (n > NOALLOC_MAX_ELEMS)
+        return report_error(-1, "asteroid_loss_mse_noalloc: n exceeds the 67108864-element limit of the allocation-free variant; use asteroid_loss_mse");
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return report_error(-5, "asteroid_loss_mse_noalloc: cudaGetDevice failed");
+    if (!g_noalloc_ptr[dev]) {
+        float* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p) return report_error(-5, "asteroid_loss_mse_noalloc: cudaGetSymbolAddress failed");
+        g_noalloc_ptr[dev] = p;
+    }
+    float* scratch = g_noalloc_ptr[dev];
+    unsigned* ticket = reinterpret_cast<unsigned*>(scratch + LOSS_MAX_BLOCKS);
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the previous call left: the ticket must start at zero
+    if (cudaMemsetAsync(ticket, 0, sizeof(unsigned), st) != cudaSuccess) return report_error(-5, "asteroid_loss_mse_noalloc: cudaMemsetAsync failed");
+    size_t want = (n + 256 * 8 - 1) / (256 * 8);
+    int blocks = (int)(want < 1 ? 1 : (want > LOSS_MAX_BLOCKS ? LOSS_MAX_BLOCKS : want));
+    {
+        LaunchScope ls(K_LOSS_MSE, 3.0 * n * (dtype == 0 ? 4.0 : 2.0), 4.0 * n, st);
+        if (dtype == 0) mse_kernel<float><<<blocks, 256, 0, st>>>((const float*)y, (const float*)target, n, (float*)dy, loss, scratch, ticket);
+        else mse_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)y, (const __nv_bfloat16*)target, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
+    }
+    if (cudaGetLastError() != cudaSuccess) return report_error(-5, "asteroid_loss_mse_noalloc: kernel launch failed");
+    return 0;
+}

@@ -30,6 +30,8 @@ struct LaunchScope {
     cudaStream_t st;
 };
 uint64_t launches();
+// records `msg` as the calling thread's last error and returns `code`
+int report_error(int code, const char* msg);
 
 // ---- dense convolution as implicit GEMM (plain FFMA tiles; float and bfloat16 storage) ----
 // z[n,ho,wo,ko] = sum_{r,s,c} x[n,ho*st-pad+r,wo*st-pad+s,c] * w[ko][r][s][c]  (+ bias[ko])
