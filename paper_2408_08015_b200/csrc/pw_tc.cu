@@ -428,6 +428,356 @@ __global__ void reduce_splits_tc(const float* __restrict__ partial, int splits, 
     out[i] = s;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Persistent, warp-specialised form of the forward / backward-data GEMM (one CTA per SM).
+//
+//   warp 0      producer: bulk-copies (cp.async.bulk, completion on an mbarrier) the raw tile
+//               rows [pixels][K] of x (forward) or of dy and z (backward) into a ring of
+//               shared-memory stages; a tile of consecutive pixels is one contiguous byte range
+//   warp 1      MMA issuer: tcgen05.mma over the staged operand into one of two accumulators in
+//               tensor memory; tcgen05.commit releases the operand stage and publishes the tile
+//   warps 2-5   transformers: read a raw stage, apply BatchNorm+activation (or the
+//               BatchNorm-backward transform) with per-thread register-held coefficients,
+//               write bf16 into the swizzled K-major operand stage
+//   warps 6-9   epilogue: tcgen05.ld the finished accumulator, add bias / residual gradient,
+//               store bf16 to global
+//
+// Copy, transform, MMA and store of consecutive tiles overlap.  The weights stay resident in
+// shared memory.  Every wait is bounded; a wait that runs out raises a CTA-wide abort flag, every
+// role leaves its loop, outstanding bulk copies are waited for, tensor memory is freed and the
+// error word is set.
+constexpr int PIPE_THREADS = 320;
+constexpr int MAX_RAW = 8;
+
+struct PipeArgs {
+    ValSrc x;
+    GradSrc dz;
+    const __nv_bfloat16* w;     // [N][K]
+    const float* bias;
+    const void* addend;
+    __nv_bfloat16* out;
+    int* err;
+    int P, K, N, NT, tiles;
+    int tmem_cols;
+    int RS, R;                  // raw stage: RS pixels (divides 128); ring of R stages
+    int need_z;                 // backward: the transform also reads z
+    uint32_t raw_bytes;         // bytes of one raw stage (both tensors), multiple of 128
+    uint32_t a_bytes, b_bytes;  // one operand stage / the resident weights
+};
+
+__device__ __forceinline__ void mbar_arrive(uint32_t mbar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src), "r"(bytes), "r"(mbar)
+                 : "memory");
+}
+// Bounded wait that also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t mbar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(mbar, parity)) return true;
+        if (*abort_flag) return false;
+        if (i > 32) __nanosleep(32);
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]),
+          "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const PipeArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * MAX_RAW + 8];   // raw_full[R], raw_empty[R], a_full[2], a_empty[2], acc_full[2], acc_empty[2]
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_store;
+    volatile int* abort_flag = &abort_store;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = base;                               // two operand stages
+    uint8_t* sB = base + 2 * (size_t)a.a_bytes;       // resident weights
+    uint8_t* sR = sB + a.b_bytes;                     // raw ring
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int R = a.R, RS = a.RS, subs = TM / RS;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    auto raw_full = [&](int s) { return bar0 + 8u * s; };
+    auto raw_empty = [&](int s) { return bar0 + 8u * (MAX_RAW + s); };
+    auto a_full = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + s); };
+    auto a_empty = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 2 + s); };
+    auto acc_full = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 4 + s); };
+    auto acc_empty = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 6 + s); };
+
+    if (tid == 0) {
+        for (int s = 0; s < R; ++s) {
+            mbar_init(raw_full(s), 1);
+            mbar_init(raw_empty(s), 128);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(a_full(s), 128);
+            mbar_init(a_empty(s), 1);
+            mbar_init(acc_full(s), 1);
+            mbar_init(acc_empty(s), 128);
+        }
+        abort_store = 0;
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_slot), (uint32_t)a.tmem_cols);
+        tmem_relinquish();
+    }
+    const int NT = a.NT;
+    const int vpr = a.K >> 3, vpr_pad = ((a.K + 15) >> 4) << 1;
+    // resident weights: [NT][K] bf16 -> swizzled K-major blocks (rows beyond N and the K padding are zero)
+    for (int v = tid; v < NT * vpr_pad; v += PIPE_THREADS) {
+        int r = v / vpr_pad, j = v - r * vpr_pad;
+        uint4 q = make_uint4(0, 0, 0, 0);
+        if (r < a.N && j < vpr) q = __ldg(reinterpret_cast<const uint4*>(a.w + (size_t)r * a.K) + j);
+        *reinterpret_cast<uint4*>(sB + tile_off(r, j, NT)) = q;
+    }
+    fence_async_smem();
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    const int my_tiles = (a.tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const uint32_t row_bytes = (uint32_t)a.K * 2u;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            const uint8_t* src0 = reinterpret_cast<const uint8_t*>(BWD ? a.dz.dy : a.x.p);
+            const uint8_t* src1 = reinterpret_cast<const uint8_t*>(a.dz.z);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int tile = blockIdx.x + t * gridDim.x;
+                for (int sub = 0; sub < subs; ++sub, ++it) {
+                    const int s = it % R, n = it / R;
+                    if (n > 0 && !mbar_wait_abortable(raw_empty(s), (uint32_t)((n - 1) & 1), abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    const int p_first = tile * TM + sub * RS;
+                    int valid = a.P - p_first;
+                    valid = valid < 0 ? 0 : (valid > RS ? RS : valid);
+                    const uint32_t bytes = (uint32_t)valid * row_bytes;
+                    uint8_t* dst = sR + (size_t)s * a.raw_bytes;
+                    if (valid > 0) {
+                        mbar_expect_tx(raw_full(s), bytes * ((BWD && a.need_z) ? 2u : 1u));
+                        bulk_g2s(smem_u32(dst), src0 + (size_t)p_first * row_bytes, bytes, raw_full(s));
+                        if (BWD && a.need_z) bulk_g2s(smem_u32(dst + (size_t)RS * row_bytes), src1 + (size_t)p_first * row_bytes, bytes, raw_full(s));
+                    } else {
+                        mbar_arrive(raw_full(s));
+                    }
+                }
+            }
+            // never leave while a bulk copy into this CTA's shared memory may still be in flight
+            const int issued = it;
+            for (int k = (issued > R ? issued - R : 0); k < issued; ++k) mbar_wait(raw_full(k % R), (uint32_t)((k / R) & 1));
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(NT);
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+            const int steps = vpr_pad >> 1;
+            for (int t = 0; t < my_tiles; ++t) {
+                const int st = t & 1, n = t >> 1;
+                if (!mbar_wait_abortable(a_full(st), (uint32_t)(n & 1), abort_flag)) break;
+                if (n > 0 && !mbar_wait_abortable(acc_empty(st), (uint32_t)((n - 1) & 1), abort_flag)) break;
+                fence_after_sync();
+                const uint32_t d = tmem + (uint32_t)(st * NT);
+                for (int k = 0; k < steps; ++k) {
+                    const int kb = k >> 2, ks = k & 3;
+                    umma_bf16(d, make_desc(a0 + st * a.a_bytes + (uint32_t)kb * TM * 128u + (uint32_t)ks * 32u),
+                              make_desc(b0 + (uint32_t)kb * (uint32_t)NT * 128u + (uint32_t)ks * 32u), idesc, k > 0 ? 1u : 0u);
+                }
+                umma_commit(a_empty(st));
+                umma_commit(acc_full(st));
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ transformers
+        const int tix = tid - 64;
+        const int groups = 128 / vpr_pad;                 // row groups; thread (grp, j) owns chunk j of rows grp, grp+groups, ...
+        const int j = tix % vpr_pad, grp = tix / vpr_pad;
+        const bool active = grp < groups;
+        const bool data = j < vpr;                        // chunks beyond K are zero padding
+        const int c0 = j << 3;
+        float cs[8], ch[8], k1[8], k2[8], k3[8];
+        bool affine = false, bn = false;
+        int act = ACT_NONE;
+        if (active && data) {
+            const float* scale = BWD ? a.dz.scale : a.x.scale;
+            const float* shift = BWD ? a.dz.shift : a.x.shift;
+            act = BWD ? a.dz.act : a.x.act;
+            affine = scale != nullptr;
+            if (affine) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    cs[q] = __ldg(scale + c0 + q);
+                    ch[q] = __ldg(shift + c0 + q);
+                }
+            }
+            if (BWD && a.dz.k1) {
+                bn = true;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    k1[q] = __ldg(a.dz.k1 + c0 + q);
+                    k2[q] = __ldg(a.dz.k2 + c0 + q);
+                    k3[q] = __ldg(a.dz.k3 + c0 + q);
+                }
+            }
+        }
+        int it = 0;
+        bool ok = true;
+        for (int t = 0; t < my_tiles && ok; ++t) {
+            const int tile = blockIdx.x + t * gridDim.x;
+            const int st = t & 1, n = t >> 1;
+            if (n > 0 && !mbar_wait_abortable(a_empty(st), (uint32_t)((n - 1) & 1), abort_flag)) break;
+            uint8_t* dstA = sA + (size_t)st * a.a_bytes;
+            for (int sub = 0; sub < subs; ++sub, ++it) {
+                const int s = it % R;
+                if (!mbar_wait_abortable(raw_full(s), (uint32_t)((it / R) & 1), abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                const uint8_t* raw = sR + (size_t)s * a.raw_bytes;
+                if (active) {
+                    for (int rl = grp; rl < RS; rl += groups) {
+                        const int r = sub * RS + rl;
+                        uint4 q4 = make_uint4(0, 0, 0, 0);
+                        if (data && tile * TM + r < a.P) {
+                            float f[8];
+                            Vec<__nv_bfloat16> v;
+                            v.raw = *reinterpret_cast<const uint4*>(raw + (size_t)rl * row_bytes + (j << 4));
+                            v.unpack(f);
+                            if (!BWD) {
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) f[q] = apply_act(affine ? fmaf(f[q], cs[q], ch[q]) : f[q], act);
+                            } else if (a.need_z) {
+                                float zz[8];
+                                v.raw = *reinterpret_cast<const uint4*>(raw + (size_t)RS * row_bytes + (size_t)rl * row_bytes + (j << 4));
+                                v.unpack(zz);
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) {
+                                    float pre = affine ? fmaf(zz[q], cs[q], ch[q]) : zz[q];
+                                    float d = f[q] * act_mask(pre, act);
+                                    f[q] = bn ? fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q])) : d;
+                                }
+                            }
+                            q4 = pack8(f);
+                        }
+                        *reinterpret_cast<uint4*>(dstA + tile_off(r, j, TM)) = q4;
+                    }
+                }
+                mbar_arrive(raw_empty(s));
+            }
+            if (!ok) break;
+            fence_async_smem();
+            mbar_arrive(a_full(st));
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;                            // TMEM lane quarter this warp may read
+        const int row = q * 32 + lane;
+        for (int t = 0; t < my_tiles; ++t) {
+            const int tile = blockIdx.x + t * gridDim.x;
+            const int st = t & 1, n = t >> 1;
+            if (!mbar_wait_abortable(acc_full(st), (uint32_t)(n & 1), abort_flag)) break;
+            fence_after_sync();
+            const int p = tile * TM + row;
+            for (int g = 0; g < (NT >> 4); ++g) {
+                float v[16];
+                tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(st * NT + (g << 4)), v);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int nn = (g << 4) + (hh << 3);
+                    if (p < a.P && nn < a.N) {
+                        float* vv = v + (hh << 3);
+                        const size_t e = (size_t)p * a.N + nn;
+                        if (!BWD && a.bias) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) vv[i] += __ldg(a.bias + nn + i);
+                        }
+                        if (BWD && a.addend) {
+                            float ad[8];
+                            Vec<__nv_bfloat16> av;
+                            av.load(a.addend, e >> 3);
+                            av.unpack(ad);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) vv[i] += ad[i];
+                        }
+                        *reinterpret_cast<uint4*>(a.out + e) = pack8(vv);
+                    }
+                }
+            }
+            fence_before_sync();
+            mbar_arrive(acc_empty(st));
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && abort_store) atomicExch(a.err, 1);
+    if (warp == 1) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+}
+
+// Chooses the pipeline's shared-memory split; returns false if the shape does not fit (large K
+// or N), in which case the one-tile-per-CTA kernel is used.
+bool plan_pipe(PipeArgs& a, size_t* smem) {
+    if (a.N > 256 || a.K > 256) return false;
+    a.NT = (a.N + 15) / 16 * 16;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < 2 * a.NT) a.tmem_cols <<= 1;
+    if (a.tmem_cols > 512) return false;
+    const int nkb = (a.K + KB - 1) / KB;
+    a.a_bytes = (uint32_t)nkb * TM * 128u;
+    a.b_bytes = (uint32_t)nkb * (uint32_t)a.NT * 128u;
+    const size_t budget = 220 * 1024 - 1024;
+    const size_t fixed = 2 * (size_t)a.a_bytes + a.b_bytes;
+    if (fixed >= budget) return false;
+    const int tensors = a.need_z ? 2 : 1;
+    for (int rs = 128; rs >= 32; rs >>= 1) {
+        size_t rb = ((size_t)rs * a.K * 2 * tensors + 127) / 128 * 128;
+        size_t r = (budget - fixed) / rb;
+        if (r >= 2 || (r >= 1 && rs == 32)) {
+            // at least two stages in flight, at most MAX_RAW and no more than three tiles' worth
+            size_t cap = (size_t)3 * (TM / rs);
+            if (r > cap) r = cap;
+            if (r > MAX_RAW) r = MAX_RAW;
+            a.RS = rs;
+            a.R = (int)r;
+            a.raw_bytes = (uint32_t)rb;
+            *smem = fixed + r * rb + 1024;
+            return a.R >= 2;
+        }
+    }
+    return false;
+}
+
+template <bool BWD> void launch_pipe(const PipeArgs& a, size_t smem, int kind, double bytes, cudaStream_t st) {
+    static bool attr_set = false;
+    static int n_sm = 0;
+    if (!attr_set) {
+        cudaFuncSetAttribute(pw_pipe_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        attr_set = true;
+    }
+    LaunchScope ls(kind, bytes, 2.0 * a.P * a.N * a.K, st);
+    int grid = a.tiles < n_sm ? a.tiles : n_sm;
+    pw_pipe_kernel<BWD><<<grid, PIPE_THREADS, smem, st>>>(a);
+}
+
 struct Tiling {
     int NT, ntiles, KC, tmem_cols;
     size_t smem;
@@ -471,8 +821,18 @@ void pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, cons
     a.x = x; a.w = wb; a.bias = bias; a.out = (__nv_bfloat16*)z; a.err = err;
     a.P = g.n * g.ho * g.wo; a.K = g.ci; a.N = g.co;
     a.stride = g.stride; a.ho = g.ho; a.wo = g.wo; a.hi = g.hi; a.wi = g.wi;
-    Tiling t = pick_tiling(a.K, a.N);
     double bytes = 2.0 * ((double)a.P * a.K + (double)a.P * a.N) + 2.0 * a.N * a.K;
+    if (g.stride == 1) {
+        PipeArgs pa{};
+        pa.x = x; pa.w = wb; pa.bias = bias; pa.out = (__nv_bfloat16*)z; pa.err = err;
+        pa.P = a.P; pa.K = a.K; pa.N = a.N; pa.tiles = (a.P + TM - 1) / TM; pa.need_z = 0;
+        size_t smem = 0;
+        if (plan_pipe(pa, &smem)) {
+            launch_pipe<false>(pa, smem, K_PW_FWD_TC, bytes, st);
+            return;
+        }
+    }
+    Tiling t = pick_tiling(a.K, a.N);
     launch<false>(a, t, K_PW_FWD_TC, bytes, st);
 }
 
@@ -481,9 +841,19 @@ void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* w
     a.dz = dz; a.w = wtb; a.addend = addend; a.out = (__nv_bfloat16*)dx; a.err = err;
     a.P = g.n * g.ho * g.wo; a.K = g.co; a.N = g.ci;
     a.stride = 1;
-    Tiling t = pick_tiling(a.K, a.N);
     double bytes = 2.0 * (double)a.P * a.K * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * (double)a.P * a.N * (addend ? 2.0 : 1.0) +
                    2.0 * a.N * a.K;
+    {
+        PipeArgs pa{};
+        pa.dz = dz; pa.w = wtb; pa.addend = addend; pa.out = (__nv_bfloat16*)dx; pa.err = err;
+        pa.P = a.P; pa.K = a.K; pa.N = a.N; pa.tiles = (a.P + TM - 1) / TM; pa.need_z = (dz.act != ACT_NONE || dz.k1) ? 1 : 0;
+        size_t smem = 0;
+        if (plan_pipe(pa, &smem)) {
+            launch_pipe<true>(pa, smem, K_PW_BWD_DATA_TC, bytes, st);
+            return;
+        }
+    }
+    Tiling t = pick_tiling(a.K, a.N);
     launch<true>(a, t, K_PW_BWD_DATA_TC, bytes, st);
 }
 
