@@ -13,43 +13,53 @@ namespace {
 // thread's NACC*V accumulators.  Rows are combined through shared memory, blocks through
 // partial[block_y][acc][c], summed in fixed order (in double) by the finishing kernel.
 struct StatsOp {
-    static constexpr int NACC = 2;
+    static constexpr int NACC = 2, NCTX = 1;     // context: the pivot (first pixel's value of each channel)
     const void* z;
-    template <typename T, int V> __device__ __forceinline__ void acc(size_t e, int c0, const float* pivot, float (*a)[V]) const {
+    template <typename T, int V> __device__ __forceinline__ void init(int c0, float (*ctx)[V]) const { ld_raw_w<T, V>(z, (size_t)c0, ctx[0]); }
+    template <typename T, int V> __device__ __forceinline__ void acc(size_t e, const float (*ctx)[V], float (*a)[V]) const {
         float v[V];
         ld_raw_w<T, V>(z, e, v);
 #pragma unroll
         for (int q = 0; q < V; ++q) {
-            float d = v[q] - pivot[q];
+            float d = v[q] - ctx[0][q];
             a[0][q] += d;
             a[1][q] = fmaf(d, d, a[1][q]);
         }
     }
-    template <typename T, int V> __device__ __forceinline__ void pivot(int c0, float* pv) const { ld_raw_w<T, V>(z, (size_t)c0, pv); }
 };
 
+// sums of dpre = dy*mask(pre) and of dpre*xhat; the per-channel coefficients live in registers
 struct BwdOp {
-    static constexpr int NACC = 2;
-    GradSrc g;            // k1 = nullptr here: yields dpre
+    static constexpr int NACC = 2, NCTX = 4;     // context: scale, shift, mean, rstd
+    GradSrc g;            // k1 unused here
     const float* mean;
     const float* rstd;
-    template <typename T, int V> __device__ __forceinline__ void acc(size_t e, int c0, const float* pivot, float (*a)[V]) const {
+    template <typename T, int V> __device__ __forceinline__ void init(int c0, float (*ctx)[V]) const {
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            ctx[0][q] = g.scale ? __ldg(g.scale + c0 + q) : 1.f;
+            ctx[1][q] = g.scale ? __ldg(g.shift + c0 + q) : 0.f;
+            ctx[2][q] = mean ? __ldg(mean + c0 + q) : 0.f;
+            ctx[3][q] = mean ? __ldg(rstd + c0 + q) : 0.f;
+        }
+    }
+    template <typename T, int V> __device__ __forceinline__ void acc(size_t e, const float (*ctx)[V], float (*a)[V]) const {
         float d[V];
-        ld_grad_w<T, V>(g, e, c0, d);
-        if (mean) {
+        ld_raw_w<T, V>(g.dy, e, d);
+        if (g.act != ACT_NONE || mean) {
             float z[V];
             ld_raw_w<T, V>(g.z, e, z);
 #pragma unroll
             for (int q = 0; q < V; ++q) {
-                a[0][q] += d[q];
-                a[1][q] = fmaf(d[q], (z[q] - __ldg(mean + c0 + q)) * __ldg(rstd + c0 + q), a[1][q]);
+                float dm = d[q] * act_mask(fmaf(z[q], ctx[0][q], ctx[1][q]), g.act);
+                a[0][q] += dm;
+                a[1][q] = fmaf(dm, (z[q] - ctx[2][q]) * ctx[3][q], a[1][q]);
             }
         } else {
 #pragma unroll
             for (int q = 0; q < V; ++q) a[0][q] += d[q];
         }
     }
-    template <typename T, int V> __device__ __forceinline__ void pivot(int, float*) const {}
 };
 
 template <typename T, int V, typename OP>
@@ -67,12 +77,11 @@ __global__ void __launch_bounds__(256) chan_reduce_kernel(OP op, size_t pixels, 
 #pragma unroll
         for (int q = 0; q < V; ++q) a[t][q] = 0.f;
     if (active) {
-        float pv[V];
-#pragma unroll
-        for (int q = 0; q < V; ++q) pv[q] = 0.f;
-        op.template pivot<T, V>(c0, pv);
+        float ctx[OP::NCTX][V];
+        op.template init<T, V>(c0, ctx);
         size_t pbeg = (size_t)blockIdx.y * pix_per_block, pend = min(pixels, pbeg + pix_per_block);
-        for (size_t p = pbeg + row; p < pend; p += rows) op.template acc<T, V>(p * c + c0, c0, pv, a);
+#pragma unroll 4
+        for (size_t p = pbeg + row; p < pend; p += rows) op.template acc<T, V>(p * c + c0, ctx, a);
     }
     const int width = cw * V;
     for (int t = 0; t < OP::NACC; ++t) {
@@ -133,35 +142,54 @@ void launch_reduce(int dtype, const ReducePlan& p, const OP& op, size_t pixels, 
     }
 }
 
-__device__ __forceinline__ double warp_sum_d(double v) {
+// A block of 1024 threads finishes 32 channels: thread (bg, cl) sums the partials of blocks bg, bg+32, ...
+// of channel cl (32 consecutive channels per load: coalesced), the eight sub-sums are combined in
+// fixed order through shared memory, in double (the thirty-two sub-sums in index order).  Returns true in the thread that owns the channel.
+__device__ __forceinline__ bool sum_partials(const float* __restrict__ partial, int blocks, int c, int& ch, double& s1, double& s2) {
+    __shared__ double sh[2][32][32];
+    const int cl = threadIdx.x & 31, bg = threadIdx.x >> 5;
+    ch = blockIdx.x * 32 + cl;
+    double a1 = 0.0, a2 = 0.0;
+    if (ch < c) {
+        // eight partials per round are loaded before any is added: the loads overlap, the order of
+        // the additions stays fixed
+        for (int b0 = bg; b0 < blocks; b0 += 32 * 8) {
+            float v1[8], v2[8];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-// One warp per channel: lanes stride over the per-block partials (fixed assignment, fixed
-// shuffle tree: deterministic), sums in double.
-__device__ __forceinline__ void sum_partials(const float* __restrict__ partial, int blocks, int c, int ch, double& s1, double& s2) {
-    const int lane = threadIdx.x & 31;
+            for (int u = 0; u < 8; ++u) {
+                const int b = b0 + 32 * u;
+                const bool ok = b < blocks;
+                v1[u] = ok ? partial[((size_t)b * 2 + 0) * c + ch] : 0.f;
+                v2[u] = ok ? partial[((size_t)b * 2 + 1) * c + ch] : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                a1 += v1[u];
+                a2 += v2[u];
+            }
+        }
+    }
+    sh[0][bg][cl] = a1;
+    sh[1][bg][cl] = a2;
+    __syncthreads();
+    if (bg != 0 || ch >= c) return false;
     s1 = 0.0;
     s2 = 0.0;
-    for (int b = lane; b < blocks; b += 32) {
-        s1 += partial[((size_t)b * 2 + 0) * c + ch];
-        s2 += partial[((size_t)b * 2 + 1) * c + ch];
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+        s1 += sh[0][k][cl];
+        s2 += sh[1][k][cl];
     }
-    s1 = warp_sum_d(s1);
-    s2 = warp_sum_d(s2);
+    return true;
 }
 
 template <typename T>
-__global__ void __launch_bounds__(128) bn_stats_finish(const float* __restrict__ partial, int blocks, int c, const T* __restrict__ z, double count,
+__global__ void __launch_bounds__(1024) bn_stats_finish(const float* __restrict__ partial, int blocks, int c, const T* __restrict__ z, double count,
                                                        const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float momentum,
                                                        BnFwdOut o) {
-    int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (ch >= c) return;
+    int ch;
     double s1, s2;
-    sum_partials(partial, blocks, c, ch, s1, s2);
-    if ((threadIdx.x & 31) != 0) return;
+    if (!sum_partials(partial, blocks, c, ch, s1, s2)) return;
     double pivot = to_f<T>(z[ch]);
     double m1 = s1 / count;
     double mean = pivot + m1;
@@ -178,14 +206,12 @@ __global__ void __launch_bounds__(128) bn_stats_finish(const float* __restrict__
     o.run_var[ch] = (float)((1.0 - momentum) * o.run_var[ch] + momentum * unbiased);
 }
 
-__global__ void __launch_bounds__(128) bn_bwd_finish(const float* __restrict__ partial, int blocks, int c, double count,
+__global__ void __launch_bounds__(1024) bn_bwd_finish(const float* __restrict__ partial, int blocks, int c, double count,
                                                      const float* __restrict__ mean, const float* __restrict__ rstd,
                                                      const float* __restrict__ gamma, BnBwdOut o) {
-    int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (ch >= c) return;
+    int ch;
     double s1, s2;
-    sum_partials(partial, blocks, c, ch, s1, s2);
-    if ((threadIdx.x & 31) != 0) return;
+    if (!sum_partials(partial, blocks, c, ch, s1, s2)) return;
     o.dbeta[ch] = (float)s1;
     if (o.dgamma) {
         o.dgamma[ch] = (float)s2;
@@ -402,9 +428,9 @@ void bn_stats(int dtype, const void* z, size_t pixels, int c, const float* gamma
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_STATS, (double)pixels * c * esz(dtype), st);
     LaunchScope ls(K_BN_STATS_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
     if (dtype == 0)
-        bn_stats_finish<float><<<(c + 3) / 4, 128, 0, st>>>(scratch, (int)p.by, c, (const float*)z, (double)pixels, gamma, beta, eps, momentum, o);
+        bn_stats_finish<float><<<(c + 31) / 32, 1024, 0, st>>>(scratch, (int)p.by, c, (const float*)z, (double)pixels, gamma, beta, eps, momentum, o);
     else
-        bn_stats_finish<__nv_bfloat16><<<(c + 3) / 4, 128, 0, st>>>(scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
+        bn_stats_finish<__nv_bfloat16><<<(c + 31) / 32, 1024, 0, st>>>(scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
                                                                        momentum, o);
 }
 
@@ -415,7 +441,7 @@ void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int 
     BwdOp op{GradSrc{dy, z, scale, shift, nullptr, nullptr, nullptr, act}, mean, rstd};
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_BWD_REDUCE, (double)pixels * c * esz(dtype) * ((act != ACT_NONE || mean) ? 2.0 : 1.0), st);
     LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
-    bn_bwd_finish<<<(c + 3) / 4, 128, 0, st>>>(scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
+    bn_bwd_finish<<<(c + 31) / 32, 1024, 0, st>>>(scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
 }
 
 template <typename T, int V> static void ew_add_launch(const ValSrc& a, const ValSrc& b, int act, size_t n, int c, void* out, void* out2, cudaStream_t st) {

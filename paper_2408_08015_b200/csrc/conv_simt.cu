@@ -181,7 +181,13 @@ __global__ void reduce_splits_kernel(const float* __restrict__ partial, int spli
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float s = 0.f;
-    for (int k = 0; k < splits; ++k) s += partial[(size_t)k * n + i];
+    for (int k0 = 0; k0 < splits; k0 += 8) {      // eight loads in flight, additions in index order
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = (k0 + u < splits) ? partial[(size_t)(k0 + u) * n + i] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += v[u];
+    }
     out[i] = s;
 }
 

@@ -508,7 +508,13 @@ __global__ void __launch_bounds__(128) dw_bwd_weight_finish(const float* __restr
     if (i >= 9 * c_total) return;
     int t = i / c_total, c = i % c_total;
     float s = 0.f;
-    for (int b = threadIdx.x & 31; b < blocks; b += 32) s += partial[((size_t)b * 9 + t) * c_total + c];
+    for (int b0 = threadIdx.x & 31; b0 < blocks; b0 += 32 * 8) {   // eight loads in flight, fixed addition order
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = (b0 + 32 * u < blocks) ? partial[((size_t)(b0 + 32 * u) * 9 + t) * c_total + c] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += v[u];
+    }
     s = warp_sum(s);
     if ((threadIdx.x & 31) == 0) gw[c * 9 + t] = s;
 }
