@@ -187,36 +187,45 @@ template <typename T>
 __global__ void __launch_bounds__(1024) bn_stats_finish(const float* __restrict__ partial, int blocks, int c, const T* __restrict__ z, double count,
                                                        const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float momentum,
                                                        BnFwdOut o) {
+    // the owner thread's per-channel inputs are requested before the partials so that all of the
+    // kernel's global loads overlap
+    const int chp = blockIdx.x * 32 + (threadIdx.x & 31);
+    const bool owner = (threadIdx.x >> 5) == 0 && chp < c;
+    const float pv = owner ? to_f<T>(z[chp]) : 0.f, gm = owner ? gamma[chp] : 0.f, bt = owner ? beta[chp] : 0.f;
+    const float rm = owner ? o.run_mean[chp] : 0.f, rv = owner ? o.run_var[chp] : 0.f;
     int ch;
     double s1, s2;
     if (!sum_partials(partial, blocks, c, ch, s1, s2)) return;
-    double pivot = to_f<T>(z[ch]);
+    double pivot = pv;
     double m1 = s1 / count;
     double mean = pivot + m1;
     double var = s2 / count - m1 * m1;
     if (var < 0.0) var = 0.0;
     double rstd = 1.0 / sqrt(var + (double)eps);
-    double sc = (double)gamma[ch] * rstd;
+    double sc = (double)gm * rstd;
     o.mean[ch] = (float)mean;
     o.rstd[ch] = (float)rstd;
     o.scale[ch] = (float)sc;
-    o.shift[ch] = (float)((double)beta[ch] - mean * sc);
+    o.shift[ch] = (float)((double)bt - mean * sc);
     double unbiased = count > 1.0 ? var * count / (count - 1.0) : var;
-    o.run_mean[ch] = (float)((1.0 - momentum) * o.run_mean[ch] + momentum * mean);
-    o.run_var[ch] = (float)((1.0 - momentum) * o.run_var[ch] + momentum * unbiased);
+    o.run_mean[ch] = (float)((1.0 - momentum) * rm + momentum * mean);
+    o.run_var[ch] = (float)((1.0 - momentum) * rv + momentum * unbiased);
 }
 
 __global__ void __launch_bounds__(1024) bn_bwd_finish(const float* __restrict__ partial, int blocks, int c, double count,
                                                      const float* __restrict__ mean, const float* __restrict__ rstd,
                                                      const float* __restrict__ gamma, BnBwdOut o) {
+    const int chp = blockIdx.x * 32 + (threadIdx.x & 31);
+    const bool owner = (threadIdx.x >> 5) == 0 && chp < c && o.dgamma != nullptr;
+    const float pr = owner ? rstd[chp] : 0.f, pm = owner ? mean[chp] : 0.f, pg = owner ? gamma[chp] : 0.f;
     int ch;
     double s1, s2;
     if (!sum_partials(partial, blocks, c, ch, s1, s2)) return;
     o.dbeta[ch] = (float)s1;
     if (o.dgamma) {
         o.dgamma[ch] = (float)s2;
-        double r = rstd[ch], m = mean[ch];
-        double k1 = (double)gamma[ch] * r;
+        double r = pr, m = pm;
+        double k1 = (double)pg * r;
         o.k1[ch] = (float)k1;
         o.k2[ch] = (float)(k1 * (-s1 + s2 * m * r) / count);
         o.k3[ch] = (float)(-k1 * s2 * r / count);

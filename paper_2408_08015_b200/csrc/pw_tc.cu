@@ -784,6 +784,299 @@ template <bool BWD> void launch_pipe(const PipeArgs& a, size_t smem, int kind, d
     pw_pipe_kernel<BWD><<<grid, PIPE_THREADS, smem, st>>>(a);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Pipelined weight gradient (one CTA per pixel range, all output channels in one CTA).
+//
+//   warp 0      producer: per 64-pixel stage, bulk-copies the raw rows of dy, z and x
+//   warp 1      MMA issuer: for every (128-row, N-tile) pair one tcgen05.mma per 16 pixels into
+//               its own tensor-memory columns, accumulating over the CTA's whole pixel range
+//   warps 2-9   transformers: dz = BatchNorm/activation backward of (dy, z), x = BatchNorm +
+//               activation of the producer's raw output, both written bf16 MN-major; after the
+//               last stage the same warps read the accumulators and write the CTA's partial
+// The partials of all CTAs are then summed in index order by reduce_splits_2d.
+constexpr int WG_THREADS = 320;
+
+struct WgArgs {
+    GradSrc dz;
+    ValSrc x;
+    float* partial;       // [ctas][CO][CI]
+    float* gw;            // [CO][CI] (written by the split-sum kernel that follows)
+    int* err;
+    int P, CO, CI;
+    int pix_per_cta;      // multiple of WSTAGE
+    int mtiles, ntiles, NT, tmem_cols;
+    int pa, pb;           // 64-channel panels of the two operands per stage (pa even)
+    int need_z, R;
+    uint32_t raw_bytes, op_bytes;
+};
+
+__global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * MAX_RAW + 5];    // raw_full[R], raw_empty[R], op_full[2], op_empty[2], done
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_store;
+    volatile int* abort_flag = &abort_store;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sOp = base;                                   // two operand stages: [A panels][B panels]
+    uint8_t* sR = base + 2 * (size_t)a.op_bytes;           // raw ring
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int R = a.R;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    auto raw_full = [&](int s) { return bar0 + 8u * s; };
+    auto raw_empty = [&](int s) { return bar0 + 8u * (MAX_RAW + s); };
+    auto op_full = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + s); };
+    auto op_empty = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 2 + s); };
+    const uint32_t done_bar = bar0 + 8u * (2 * MAX_RAW + 4);
+    if (tid == 0) {
+        for (int s = 0; s < R; ++s) {
+            mbar_init(raw_full(s), 1);
+            mbar_init(raw_empty(s), 256);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(op_full(s), 256);
+            mbar_init(op_empty(s), 1);
+        }
+        mbar_init(done_bar, 1);
+        abort_store = 0;
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_slot), (uint32_t)a.tmem_cols);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    const int pbeg = blockIdx.x * a.pix_per_cta, pend = min(a.P, pbeg + a.pix_per_cta);
+    const int stages = (pend - pbeg + WSTAGE - 1) / WSTAGE;
+    const uint32_t rowA = (uint32_t)a.CO * 2u, rowB = (uint32_t)a.CI * 2u;
+    const uint32_t offZ = WSTAGE * rowA, offX = offZ * (a.need_z ? 2u : 1u);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint8_t* gdy = reinterpret_cast<const uint8_t*>(a.dz.dy);
+            const uint8_t* gz = reinterpret_cast<const uint8_t*>(a.dz.z);
+            const uint8_t* gx = reinterpret_cast<const uint8_t*>(a.x.p);
+            int it = 0;
+            for (; it < stages; ++it) {
+                const int s = it % R, n = it / R;
+                if (n > 0 && !mbar_wait_abortable(raw_empty(s), (uint32_t)((n - 1) & 1), abort_flag)) break;
+                const int p0 = pbeg + it * WSTAGE;
+                const uint32_t valid = (uint32_t)min(WSTAGE, pend - p0);
+                uint8_t* dst = sR + (size_t)s * a.raw_bytes;
+                mbar_expect_tx(raw_full(s), valid * (rowA * (a.need_z ? 2u : 1u) + rowB));
+                bulk_g2s(smem_u32(dst), gdy + (size_t)p0 * rowA, valid * rowA, raw_full(s));
+                if (a.need_z) bulk_g2s(smem_u32(dst + offZ), gz + (size_t)p0 * rowA, valid * rowA, raw_full(s));
+                bulk_g2s(smem_u32(dst + offX), gx + (size_t)p0 * rowB, valid * rowB, raw_full(s));
+            }
+            for (int k = (it > R ? it - R : 0); k < it; ++k) mbar_wait(raw_full(k % R), (uint32_t)((k / R) & 1));
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(a.NT) | (1u << 15) | (1u << 16);
+            bool ok = true;
+            for (int it = 0; it < stages && ok; ++it) {
+                const int st = it & 1, n = it >> 1;
+                if (!mbar_wait_abortable(op_full(st), (uint32_t)(n & 1), abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                fence_after_sync();
+                const uint32_t a0 = smem_u32(sOp + (size_t)st * a.op_bytes), b0 = a0 + (uint32_t)a.pa * PANEL;
+                for (int mt = 0; mt < a.mtiles; ++mt)
+                    for (int nt = 0; nt < a.ntiles; ++nt) {
+                        const uint32_t d = tmem + (uint32_t)((mt * a.ntiles + nt) * a.NT);
+#pragma unroll
+                        for (int k = 0; k < WSTAGE / 16; ++k)
+                            umma_bf16(d, make_desc_mn(a0 + (uint32_t)mt * 2u * PANEL + k * 2048), make_desc_mn(b0 + (uint32_t)nt * (uint32_t)(a.NT >> 6) * PANEL + k * 2048),
+                                      idesc, (it > 0 || k > 0) ? 1u : 0u);
+                    }
+                umma_commit(op_empty(st));
+            }
+            if (ok) umma_commit(done_bar);
+        }
+    } else {
+        // ---------------------------------------------------------------- transformers, then epilogue
+        const int tix = tid - 64;
+        const int ca = a.CO >> 3, cb = a.CI >> 3, ct = ca + cb;
+        const int groups = 256 / ct;
+        const int j = tix % ct, grp = tix / ct;
+        const bool active = grp < groups;
+        const bool isA = j < ca;
+        const int jc = isA ? j : j - ca;
+        const int c0 = jc << 3;
+        float cs[8], ch[8], k1[8], k2[8], k3[8];
+        bool affine = false, bn = false;
+        int act = ACT_NONE;
+        if (active) {
+            const float* scale = isA ? a.dz.scale : a.x.scale;
+            const float* shift = isA ? a.dz.shift : a.x.shift;
+            act = isA ? a.dz.act : a.x.act;
+            affine = scale != nullptr;
+            if (affine) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    cs[q] = __ldg(scale + c0 + q);
+                    ch[q] = __ldg(shift + c0 + q);
+                }
+            }
+            if (isA && a.dz.k1) {
+                bn = true;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    k1[q] = __ldg(a.dz.k1 + c0 + q);
+                    k2[q] = __ldg(a.dz.k2 + c0 + q);
+                    k3[q] = __ldg(a.dz.k3 + c0 + q);
+                }
+            }
+        }
+        bool ok = true;
+        for (int it = 0; it < stages; ++it) {
+            const int st = it & 1, n = it >> 1, s = it % R;
+            if (n > 0 && !mbar_wait_abortable(op_empty(st), (uint32_t)((n - 1) & 1), abort_flag)) {
+                ok = false;
+                break;
+            }
+            if (!mbar_wait_abortable(raw_full(s), (uint32_t)((it / R) & 1), abort_flag)) {
+                ok = false;
+                break;
+            }
+            const uint8_t* raw = sR + (size_t)s * a.raw_bytes;
+            uint8_t* dst = sOp + (size_t)st * a.op_bytes + (isA ? 0u : (uint32_t)a.pa * PANEL) + (uint32_t)(jc >> 3) * PANEL;
+            const int valid = min(WSTAGE, pend - (pbeg + it * WSTAGE));
+            if (active) {
+                for (int kr = grp; kr < WSTAGE; kr += groups) {
+                    uint4 q4 = make_uint4(0, 0, 0, 0);
+                    if (kr < valid) {
+                        float f[8];
+                        Vec<__nv_bfloat16> v;
+                        if (isA) {
+                            v.raw = *reinterpret_cast<const uint4*>(raw + (size_t)kr * rowA + (jc << 4));
+                            v.unpack(f);
+                            if (a.need_z) {
+                                float zz[8];
+                                v.raw = *reinterpret_cast<const uint4*>(raw + offZ + (size_t)kr * rowA + (jc << 4));
+                                v.unpack(zz);
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) {
+                                    float pre = affine ? fmaf(zz[q], cs[q], ch[q]) : zz[q];
+                                    float d = f[q] * act_mask(pre, act);
+                                    f[q] = bn ? fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q])) : d;
+                                }
+                            }
+                        } else {
+                            v.raw = *reinterpret_cast<const uint4*>(raw + offX + (size_t)kr * rowB + (jc << 4));
+                            v.unpack(f);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) f[q] = apply_act(affine ? fmaf(f[q], cs[q], ch[q]) : f[q], act);
+                        }
+                        q4 = pack8(f);
+                    }
+                    *reinterpret_cast<uint4*>(dst + kr * 128 + (((jc & 7) ^ (kr & 7)) << 4)) = q4;
+                }
+            }
+            mbar_arrive(raw_empty(s));
+            fence_async_smem();
+            mbar_arrive(op_full(st));
+        }
+        if (ok && stages > 0) ok = mbar_wait_abortable(done_bar, 0u, abort_flag);
+        if (ok) {
+            fence_after_sync();
+            const int q = warp & 3, half = (warp - 2) >> 2;    // two warps share each lane quarter
+            float* pbase = a.partial + (size_t)blockIdx.x * a.CO * a.CI;
+            for (int mt = 0; mt < a.mtiles; ++mt) {
+                const int k = mt * TM + q * 32 + lane;
+                for (int nt = 0; nt < a.ntiles; ++nt)
+                    for (int g = half; g < (a.NT >> 4); g += 2) {
+                        float v[16];
+                        if (stages > 0) {
+                            tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)((mt * a.ntiles + nt) * a.NT + (g << 4)), v);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                        }
+                        const int c = nt * a.NT + (g << 4);
+                        if (k < a.CO) {
+#pragma unroll
+                            for (int hh = 0; hh < 4; ++hh)
+                                if (c + hh * 4 < a.CI)
+                                    *reinterpret_cast<float4*>(pbase + (size_t)k * a.CI + c + hh * 4) = make_float4(v[hh * 4], v[hh * 4 + 1], v[hh * 4 + 2], v[hh * 4 + 3]);
+                        }
+                    }
+            }
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && abort_store) atomicExch(a.err, 1);
+    if (warp == 1) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+}
+
+// out[i] = sum_k partial[k][i], k in index order.  A block of 1024 threads owns 32 outputs:
+// thread (kg, il) adds the partials kg, kg+32, ... of output il (32 consecutive outputs per
+// load: coalesced; all of a thread's loads are issued before the additions), the 32 sub-sums
+// are combined in fixed order through shared memory.
+__global__ void __launch_bounds__(1024) reduce_splits_2d(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
+    __shared__ float sh[32][33];
+    const int il = threadIdx.x & 31, kg = threadIdx.x >> 5;
+    const size_t i = (size_t)blockIdx.x * 32 + il;
+    float acc = 0.f;
+    if (i < n) {
+        for (int k0 = kg; k0 < splits; k0 += 32 * 8) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = (k0 + 32 * u < splits) ? partial[(size_t)(k0 + 32 * u) * n + i] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc += v[u];
+        }
+    }
+    sh[kg][il] = acc;
+    __syncthreads();
+    if (kg == 0 && i < n) {
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) s += sh[k][il];
+        out[i] = s;
+    }
+}
+
+bool plan_wgrad(WgArgs& a, size_t* smem, size_t scratch_floats, int n_sm) {
+    if (a.CO > 512 || a.CI > 512 || (a.CO + a.CI) / 8 > 256) return false;
+    a.ntiles = (a.CI + 255) / 256;
+    a.NT = ((a.CI + a.ntiles - 1) / a.ntiles + 63) / 64 * 64;      // whole panels per N tile
+    if (a.ntiles == 1) a.NT = (a.CI + 15) / 16 * 16;
+    a.mtiles = (a.CO + TM - 1) / TM;
+    int cols = a.mtiles * a.ntiles * a.NT;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < cols) a.tmem_cols <<= 1;
+    if (a.tmem_cols > 512) return false;
+    a.pa = a.mtiles * 2;
+    a.pb = a.ntiles == 1 ? (a.NT + 63) / 64 : a.ntiles * (a.NT / 64);
+    a.op_bytes = (uint32_t)(a.pa + a.pb) * PANEL;
+    size_t rb = (size_t)WSTAGE * (a.CO * 2 * (a.need_z ? 2 : 1) + a.CI * 2);
+    rb = (rb + 127) / 128 * 128;
+    a.raw_bytes = (uint32_t)rb;
+    const size_t budget = 220 * 1024 - 1024;
+    const size_t fixed = 2 * (size_t)a.op_bytes;
+    if (fixed + 2 * rb > budget) return false;
+    size_t r = (budget - fixed) / rb;
+    if (r > 4) r = 4;
+    a.R = (int)r;
+    *smem = fixed + r * rb + 1024;
+    size_t out_elems = (size_t)a.CO * a.CI;
+    int ctas = n_sm;
+    int max_by_pix = (a.P + 2 * WSTAGE - 1) / (2 * WSTAGE);
+    if (ctas > max_by_pix) ctas = max_by_pix;
+    size_t cap = scratch_floats / out_elems;
+    if ((size_t)ctas > cap) ctas = (int)cap;
+    if (ctas < 1) return false;
+    int ppc = (a.P + ctas - 1) / ctas;
+    ppc = (ppc + WSTAGE - 1) / WSTAGE * WSTAGE;
+    a.pix_per_cta = ppc;
+    return true;
+}
+
 struct Tiling {
     int NT, ntiles, KC, tmem_cols;
     size_t smem;
@@ -865,6 +1158,34 @@ void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* w
 
 void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                       cudaStream_t st) {
+    if (g.stride == 1) {
+        static int n_sm = 0;
+        static bool attr = false;
+        if (!attr) {
+            cudaFuncSetAttribute(pw_wgrad_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+            int dev = 0;
+            cudaGetDevice(&dev);
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+            attr = true;
+        }
+        WgArgs wa{};
+        wa.dz = dz; wa.x = x; wa.partial = scratch; wa.gw = gw; wa.err = err;
+        wa.P = g.n * g.ho * g.wo; wa.CO = g.co; wa.CI = g.ci;
+        wa.need_z = (dz.act != ACT_NONE || dz.k1) ? 1 : 0;
+        size_t smem = 0;
+        if (plan_wgrad(wa, &smem, scratch_floats, n_sm)) {
+            int ctas = (wa.P + wa.pix_per_cta - 1) / wa.pix_per_cta;
+            double bytes = 2.0 * (double)wa.P * wa.CO * (wa.need_z ? 2.0 : 1.0) + 2.0 * (double)wa.P * wa.CI + 4.0 * wa.CO * wa.CI * (2.0 * ctas + 1);
+            {
+                LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * wa.P * wa.CO * wa.CI, st);
+                pw_wgrad_pipe_kernel<<<ctas, WG_THREADS, smem, st>>>(wa);
+            }
+            size_t out_elems = (size_t)wa.CO * wa.CI;
+            LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);
+            reduce_splits_2d<<<(unsigned)((out_elems + 31) / 32), 1024, 0, st>>>(scratch, ctas, out_elems, gw);
+            return;
+        }
+    }
     PwWArgs a{};
     a.dz = dz; a.x = x; a.partial = scratch; a.err = err;
     a.P = g.n * g.ho * g.wo; a.CO = g.co; a.CI = g.ci;
