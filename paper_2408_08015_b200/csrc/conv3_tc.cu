@@ -1,0 +1,216 @@
+// Dense 3x3 convolution (stride 1, pad 1) as an implicit GEMM on tcgen05: forward and
+// backward-data.
+//
+// Pixels of one image are addressed in *padded, flattened* coordinates f = hp*(W+2) + wp.  In
+// these coordinates tap (r,s) of output position f reads position f + (r-1)*(W+2) + (s-1): a
+// constant row offset.  A CTA owns 128 consecutive positions; it stages the 128 + 2(W+2) + 2
+// positions they touch ONCE (producer BatchNorm + activation, or the BatchNorm-backward
+// transform, applied on the way; padding positions are zeros) as K-major rows of 64 channels,
+// and every tap's A operand is the same buffer seen through a descriptor whose start address is
+// moved by the tap's row offset.  Per tap the weights [N][C] are streamed into one of two
+// shared-memory stages while the previous tap's MMAs run; the 9*C/16 MMAs accumulate into one
+// tensor-memory tile.  Positions that are padding produce values that are never stored.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+#include "tc_common.cuh"
+
+namespace ast {
+namespace {
+
+using namespace tc;
+constexpr int C3_THREADS = 256;
+
+struct C3Args {
+    ValSrc x;                  // forward operand
+    GradSrc dz;                // backward operand
+    const __nv_bfloat16* w;    // forward: [N][9][C] (N = c_out, C = c_in); backward: [N][9][C] with N = c_in, C = c_out
+    const void* addend;        // backward only, may be null
+    __nv_bfloat16* out;        // [n][H][W][N]
+    int* err;
+    int n_img, H, W, C, N;     // C: reduction channels (multiple of 64), N: output channels (multiple of 16, <= 256)
+    int tiles_per_img, rows_pad, tmem_cols;
+    int flip;                  // backward: tap t uses weight tap 8 - t
+};
+
+// K-major, 128-byte swizzle, start address anywhere on a 128-byte row of a 1024-byte aligned
+// buffer.  The swizzle is a function of the shared-memory address bits (16-byte chunk index XOR
+// address bits 7..9), and the rows were written with the same function of their address, so a
+// start address moved by whole rows needs no correction: the base-offset field stays 0.
+__device__ __forceinline__ uint64_t make_desc_row(uint32_t smem_addr) { return make_desc(smem_addr); }
+
+template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kernel(const C3Args a) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2];
+    __shared__ uint32_t tmem_slot;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Wp = a.W + 2;
+    const int kbs = a.C >> 6;                               // 64-channel blocks
+    const uint32_t a_block = (uint32_t)a.rows_pad * 128u;   // bytes of one channel block of the staged rows
+    const uint32_t b_stage = (uint32_t)kbs * (uint32_t)a.N * 128u;
+    uint8_t* sA = base;
+    uint8_t* sB = base + (size_t)kbs * a_block;
+    const int img = blockIdx.x / a.tiles_per_img, tile = blockIdx.x - img * a.tiles_per_img;
+    const int f0 = Wp + 1 + tile * TM;                      // first output position of this CTA
+    const int fs0 = f0 - Wp - 1;                            // first staged position
+    const int rows = TM + 2 * Wp + 2;
+    const uint32_t bar0 = smem_u32(&bars[0]), bar1 = smem_u32(&bars[1]);
+
+    if (tid == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar1, 1);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), (uint32_t)a.tmem_cols);
+        tmem_relinquish();
+    }
+    // ---- stage the input rows once: position -> (hp, wp); interior positions are pixels ----
+    {
+        const int vpr = a.C >> 3;
+        for (int v = tid; v < rows * vpr; v += C3_THREADS) {
+            const int r = v / vpr, j = v - r * vpr;
+            const int f = fs0 + r;
+            const int hp = f / Wp, wp = f - hp * Wp;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (f >= 0 && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W) {
+                float fv[8];
+                const int c0 = j << 3;
+                const size_t e = (((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.C + c0;
+                if (BWD) ld_grad_vec<__nv_bfloat16>(a.dz, e >> 3, c0, fv);
+                else ld_val_vec<__nv_bfloat16>(a.x, e >> 3, c0, fv);
+                q = pack8(fv);
+            }
+            *reinterpret_cast<uint4*>(sA + (size_t)(j >> 3) * a_block + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+        }
+    }
+    fence_async_smem();
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t idesc = make_idesc(a.N);
+
+    // ---- nine taps: stream the tap's weights into stage t&1, then its C/16 MMAs ----
+    uint32_t ph[2] = {0, 0};
+    bool bad = false;
+    const int vpr = a.C >> 3;
+    for (int t = 0; t < 9; ++t) {
+        const int st = t & 1;
+        if (t >= 2) {                                   // the MMAs of tap t-2 read this weight stage
+            bool ok = mbar_wait(st ? bar1 : bar0, ph[st]);
+            ph[st] ^= 1;
+            if (!__syncthreads_and(ok ? 1 : 0)) {
+                bad = true;
+                break;
+            }
+        }
+        const int wt = a.flip ? 8 - t : t;
+        uint8_t* dstB = sB + (size_t)st * b_stage;
+        for (int v = tid; v < a.N * vpr; v += C3_THREADS) {
+            const int n = v / vpr, j = v - n * vpr;
+            uint4 q = __ldg(reinterpret_cast<const uint4*>(a.w + ((size_t)n * 9 + wt) * a.C) + j);
+            *reinterpret_cast<uint4*>(dstB + tile_off(n, j, a.N)) = q;
+        }
+        fence_async_smem();
+        __syncthreads();
+        if (tid == 0) {
+            fence_after_sync();
+            const int r = t / 3, s = t - r * 3;
+            const uint32_t a0 = smem_u32(sA) + (uint32_t)(r * Wp + s) * 128u;
+            const uint32_t b0 = smem_u32(dstB);
+            for (int k = 0; k < (a.C >> 4); ++k) {
+                const int kb = k >> 2, ks = k & 3;
+                umma_bf16(tmem, make_desc_row(a0 + (uint32_t)kb * a_block + (uint32_t)ks * 32u),
+                          make_desc(b0 + (uint32_t)kb * (uint32_t)a.N * 128u + (uint32_t)ks * 32u), idesc, (t > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(st ? bar1 : bar0);
+        }
+    }
+    if (!bad) {                                         // the last commit (tap 8, stage 0) covers every MMA
+        bool ok = mbar_wait(bar0, ph[0]);
+        if (!__syncthreads_and(ok ? 1 : 0)) bad = true;
+    }
+    fence_after_sync();
+    __syncthreads();
+    if (bad) {
+        if (tid == 0) atomicExch(a.err, 1);
+    } else {
+        const int q = warp & 3, half = warp >> 2;
+        const int f = f0 + q * 32 + lane;
+        const int hp = f / Wp, wp = f - hp * Wp;
+        const bool pix = hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+        const size_t e0 = (((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.N;
+        for (int g = half; g < (a.N >> 4); g += 2) {
+            float v[16];
+            tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g << 4), v);
+            if (pix) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    float* vv = v + (hh << 3);
+                    const size_t e = e0 + (g << 4) + (hh << 3);
+                    if (BWD && a.addend) {
+                        float ad[8];
+                        Vec<__nv_bfloat16> av;
+                        av.load(a.addend, e >> 3);
+                        av.unpack(ad);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) vv[i] += ad[i];
+                    }
+                    *reinterpret_cast<uint4*>(a.out + e) = pack8(vv);
+                }
+            }
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+}
+
+template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, cudaStream_t st) {
+    const int Wp = a.W + 2;
+    const int centers = (a.H - 1) * Wp + a.W;           // positions Wp+1 .. H*Wp+W
+    a.tiles_per_img = (centers + TM - 1) / TM;
+    a.rows_pad = (TM + 2 * Wp + 2 + 7) / 8 * 8;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < a.N) a.tmem_cols <<= 1;
+    const int kbs = a.C / 64;
+    size_t smem = (size_t)kbs * a.rows_pad * 128 + 2 * (size_t)kbs * a.N * 128 + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(conv3_tc_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        attr_set = true;
+    }
+    LaunchScope ls(kind, bytes, 2.0 * 9.0 * a.n_img * a.H * a.W * (double)a.C * a.N, st);
+    conv3_tc_kernel<BWD><<<a.n_img * a.tiles_per_img, C3_THREADS, smem, st>>>(a);
+}
+
+}  // namespace
+
+bool conv3_tc_supported(int dtype, const ConvGeom& g) {
+    if (!(dtype == 1 && g.k == 3 && g.stride == 1 && g.pad == 1)) return false;
+    if (g.ci % 64 || g.co % 64 || g.ci > 256 || g.co > 256) return false;
+    const int Wp = g.wi + 2;
+    const int rows_pad = (TM + 2 * Wp + 2 + 7) / 8 * 8;
+    const int cmax = g.ci > g.co ? g.ci : g.co;
+    return (size_t)(cmax / 64) * rows_pad * 128 + 2 * (size_t)(cmax / 64) * cmax * 128 + 1024 <= 200 * 1024;
+}
+
+void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st) {
+    C3Args a{};
+    a.x = x; a.w = wb; a.out = (__nv_bfloat16*)z; a.err = err;
+    a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.C = g.ci; a.N = g.co; a.flip = 0;
+    double px = (double)g.n * g.hi * g.wi;
+    launch_c3<false>(a, K_CONV3_FWD_TC, 2.0 * px * (g.ci + g.co) + 2.0 * 9 * g.ci * g.co, st);
+}
+
+void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st) {
+    C3Args a{};
+    a.dz = dz; a.w = wtb; a.addend = addend; a.out = (__nv_bfloat16*)dx; a.err = err;
+    a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.C = g.co; a.N = g.ci; a.flip = 1;
+    double px = (double)g.n * g.hi * g.wi;
+    launch_c3<true>(a, K_CONV3_BWD_DATA_TC,
+                    2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci * (addend ? 2.0 : 1.0) + 2.0 * 9 * g.ci * g.co, st);
+}
+
+}  // namespace ast

@@ -362,6 +362,7 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
         if (u.kind == U_CONV) {
             const float* bias = u.b_off >= 0 ? s->w + u.b_off : nullptr;
             if (pw_tc_supported(dt, u.g, false)) pw_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, bias, obuf, s->err, st);
+            else if (conv3_tc_supported(dt, u.g)) conv3_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, obuf, s->err, st);
             else conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, bias, obuf, st);
         } else if (u.kind == U_DW) {
             dw_fwd(dt, u.g, val_src(s, sv, u.in), s->derived + u.w_off, obuf, st);
@@ -447,6 +448,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                 GradState& gi = gs[u.in];
                 const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
                 if (u.kind == U_CONV && pw_tc_supported(dt, u.g, true)) pw_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
+                else if (u.kind == U_CONV && conv3_tc_supported(dt, u.g)) conv3_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
                 else if (u.kind == U_CONV) conv_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 else dw_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 gi.state = G_OWNED;

@@ -22,6 +22,8 @@ SMALL = {
     "bottlenecks_small": (si.bottleneck_net(16, [(8, 32, 2, 1), (16, 64, 2, 2)]), 12, 12, 2, 2, "mse"),
     "small_mobilenet_xent": (si.small_mobilenet(10)[0], 32, 32, 4, 2, "xent"),
     "bnfree_block": (si.bnfree_net(8, 2), 9, 9, 2, 3, "mse"),
+    "bottleneck_c64": (si.bottleneck_net(64, [(64, 128, 1, 1)]), 10, 9, 2, 2, "mse"),
+    "bottleneck_c128": (si.bottleneck_net(128, [(128, 128, 2, 1)]), 7, 12, 2, 1, "mse"),
 }
 
 
