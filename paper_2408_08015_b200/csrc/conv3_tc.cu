@@ -185,6 +185,176 @@ template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, cudaStream
     conv3_tc_kernel<BWD><<<a.n_img * a.tiles_per_img, C3_THREADS, smem, st>>>(a);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Weight gradient of the 3x3 conv:  gw[k][t][c] = sum_f dz[f][k] * x[f + off_t][c]  over the
+// padded-flattened positions f of all images (dz and x are zero at padding positions).
+// The reduction index is the position, so both operands are MN-major exactly as staged:
+// rows = positions, 128 bytes = 64 channels.  x is staged with its halo once per tile and tap t
+// reads it through a start address moved by off_t rows; each tap owns its own accumulator
+// columns in tensor memory.  A CTA walks a range of tiles and a group of taps (9*c_in columns
+// do not fit the 512 columns), accumulates in tensor memory, and writes one partial in the
+// gradient's own layout; the partials are summed in index order by a second kernel.
+struct W3Args {
+    GradSrc dz;
+    ValSrc x;
+    float* partial;            // [ctas][CO][9][CI], only this CTA's taps are written
+    int* err;
+    int n_img, H, W, CI, CO;
+    int tiles_per_img, total_tiles, tiles_per_cta, rows_pad, taps_per_group, tmem_cols;
+};
+
+__device__ __forceinline__ uint64_t make_desc_mn_lbo(uint32_t smem_addr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+__global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args a) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bar_store;
+    __shared__ uint32_t tmem_slot;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Wp = a.W + 2;
+    const int kbi = a.CI >> 6, kbo = (a.CO + 63) >> 6;
+    const uint32_t x_block = (uint32_t)a.rows_pad * 128u;
+    const uint32_t dz_block = TM * 128u;
+    uint8_t* sDZ = base;                                   // two 64-channel panels (rows beyond c_out are never read back)
+    uint8_t* sX = base + 2 * dz_block;
+    const int rows = TM + 2 * Wp + 2;
+    const uint32_t bar = smem_u32(&bar_store);
+    const int t_first = blockIdx.y * a.taps_per_group;
+    const int t_count = min(a.taps_per_group, 9 - t_first);
+    if (tid == 0) mbar_init(bar, 1);
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), (uint32_t)a.tmem_cols);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t idesc = make_idesc(a.CI) | (1u << 15) | (1u << 16);
+    const int tile_beg = blockIdx.x * a.tiles_per_cta, tile_end = min(a.total_tiles, tile_beg + a.tiles_per_cta);
+    uint32_t phase = 0;
+    bool bad = false;
+    for (int tl = tile_beg; tl < tile_end; ++tl) {
+        const int img = tl / a.tiles_per_img, tile = tl - img * a.tiles_per_img;
+        const int f0 = Wp + 1 + tile * TM, fs0 = f0 - Wp - 1;
+        // x with halo
+        const int vx = a.CI >> 3;
+        for (int v = tid; v < rows * vx; v += C3_THREADS) {
+            const int r = v / vx, j = v - r * vx;
+            const int f = fs0 + r;
+            const int hp = f / Wp, wp = f - hp * Wp;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (f >= 0 && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W) {
+                float fv[8];
+                const int c0 = j << 3;
+                ld_val_vec<__nv_bfloat16>(a.x, ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CI + c0) >> 3, c0, fv);
+                q = pack8(fv);
+            }
+            *reinterpret_cast<uint4*>(sX + (size_t)(j >> 3) * x_block + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+        }
+        // dz at the 128 centre positions
+        const int vz = a.CO >> 3;
+        for (int v = tid; v < TM * vz; v += C3_THREADS) {
+            const int r = v / vz, j = v - r * vz;
+            const int f = f0 + r;
+            const int hp = f / Wp, wp = f - hp * Wp;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W) {
+                float fv[8];
+                const int c0 = j << 3;
+                ld_grad_vec<__nv_bfloat16>(a.dz, ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CO + c0) >> 3, c0, fv);
+                q = pack8(fv);
+            }
+            *reinterpret_cast<uint4*>(sDZ + (size_t)(j >> 3) * dz_block + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+        }
+        fence_async_smem();
+        __syncthreads();
+        if (tid == 0) {
+            fence_after_sync();
+            const uint32_t z0 = smem_u32(sDZ), x0 = smem_u32(sX);
+            for (int tt = 0; tt < t_count; ++tt) {
+                const int t = t_first + tt, r = t / 3, s = t - r * 3;
+                const uint32_t xs = x0 + (uint32_t)(r * Wp + s) * 128u;
+                const uint32_t d = tmem + (uint32_t)(tt * a.CI);
+#pragma unroll
+                for (int k = 0; k < TM / 16; ++k)
+                    umma_bf16(d, make_desc_mn_lbo(z0 + k * 2048, dz_block), make_desc_mn_lbo(xs + k * 2048, x_block), idesc,
+                              (tl > tile_beg || k > 0) ? 1u : 0u);
+            }
+            umma_commit(bar);
+        }
+        bool ok = mbar_wait(bar, phase);      // shared memory is rewritten by the next tile
+        phase ^= 1;
+        if (!__syncthreads_and(ok ? 1 : 0)) {
+            bad = true;
+            break;
+        }
+    }
+    fence_after_sync();
+    __syncthreads();
+    if (bad) {
+        if (tid == 0) atomicExch(a.err, 1);
+    } else {
+        const int q = warp & 3, half = warp >> 2;
+        const int k = q * 32 + lane;
+        float* pb = a.partial + (size_t)blockIdx.x * a.CO * 9 * a.CI;
+        for (int tt = 0; tt < t_count; ++tt) {
+            const int t = t_first + tt;
+            for (int g = half; g < (a.CI >> 4); g += 2) {
+                float v[16];
+                if (tile_end > tile_beg) {
+                    tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(tt * a.CI + (g << 4)), v);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                }
+                if (k < a.CO) {
+                    float* dst = pb + ((size_t)k * 9 + t) * a.CI + (g << 4);
+#pragma unroll
+                    for (int hh = 0; hh < 4; ++hh) *reinterpret_cast<float4*>(dst + hh * 4) = make_float4(v[hh * 4], v[hh * 4 + 1], v[hh * 4 + 2], v[hh * 4 + 3]);
+                }
+            }
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+    (void)kbi; (void)kbo;
+}
+
+__global__ void __launch_bounds__(1024) reduce_splits_c3(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
+    __shared__ float sh[32][33];
+    const int il = threadIdx.x & 31, kg = threadIdx.x >> 5;
+    const size_t i = (size_t)blockIdx.x * 32 + il;
+    float acc = 0.f;
+    if (i < n) {
+        for (int k0 = kg; k0 < splits; k0 += 32 * 8) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = (k0 + 32 * u < splits) ? partial[(size_t)(k0 + 32 * u) * n + i] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc += v[u];
+        }
+    }
+    sh[kg][il] = acc;
+    __syncthreads();
+    if (kg == 0 && i < n) {
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) s += sh[k][il];
+        out[i] = s;
+    }
+}
+
 }  // namespace
 
 bool conv3_tc_supported(int dtype, const ConvGeom& g) {
@@ -211,6 +381,52 @@ void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16
     double px = (double)g.n * g.hi * g.wi;
     launch_c3<true>(a, K_CONV3_BWD_DATA_TC,
                     2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci * (addend ? 2.0 : 1.0) + 2.0 * 9 * g.ci * g.co, st);
+}
+
+bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g) {
+    return conv3_tc_supported(dtype, g) && g.ci <= 128 && g.co <= 128;
+}
+
+void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
+                         cudaStream_t st) {
+    W3Args a{};
+    a.dz = dz; a.x = x; a.partial = scratch; a.err = err;
+    a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.CI = g.ci; a.CO = g.co;
+    const int Wp = a.W + 2;
+    a.tiles_per_img = ((a.H - 1) * Wp + a.W + TM - 1) / TM;
+    a.total_tiles = a.n_img * a.tiles_per_img;
+    a.rows_pad = (TM + 2 * Wp + 2 + 7) / 8 * 8;
+    a.taps_per_group = 512 / a.CI < 9 ? 512 / a.CI : 9;
+    if (a.taps_per_group > 5 && a.CI == 64) a.taps_per_group = 5;      // 5 + 4 taps: two balanced groups
+    if (a.CI == 128) a.taps_per_group = 3;
+    const int groups = (9 + a.taps_per_group - 1) / a.taps_per_group;
+    a.tmem_cols = 32;
+    while (a.tmem_cols < a.taps_per_group * a.CI) a.tmem_cols <<= 1;
+    static int n_sm = 0;
+    static bool attr = false;
+    if (!attr) {
+        cudaFuncSetAttribute(conv3_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        attr = true;
+    }
+    const size_t out_elems = (size_t)a.CO * 9 * a.CI;
+    int ctas = (2 * n_sm) / groups;
+    if (ctas > a.total_tiles) ctas = a.total_tiles;
+    if ((size_t)ctas > scratch_floats / out_elems) ctas = (int)(scratch_floats / out_elems);
+    if (ctas < 1) ctas = 1;
+    a.tiles_per_cta = (a.total_tiles + ctas - 1) / ctas;
+    ctas = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
+    size_t smem = 2 * (size_t)TM * 128 + (size_t)(a.CI / 64) * a.rows_pad * 128 + 1024;
+    double px = (double)g.n * g.hi * g.wi;
+    {
+        LaunchScope ls(K_CONV3_BWD_WEIGHT_TC, 2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci + 4.0 * out_elems * ctas,
+                       2.0 * 9.0 * px * g.ci * g.co, st);
+        conv3_wgrad_tc_kernel<<<dim3(ctas, groups), C3_THREADS, smem, st>>>(a);
+    }
+    LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);
+    reduce_splits_c3<<<(unsigned)((out_elems + 31) / 32), 1024, 0, st>>>(scratch, ctas, out_elems, gw);
 }
 
 }  // namespace ast

@@ -16,7 +16,7 @@ struct ConvGeom {
 enum KernelKind {
     K_CONV_FWD = 0, K_CONV_BWD_DATA, K_CONV_BWD_WEIGHT, K_REDUCE_SPLITS, K_DW_FWD, K_DW_BWD_DATA, K_DW_BWD_WEIGHT,
     K_DW_BWD_WEIGHT_FINISH, K_BN_STATS, K_BN_STATS_FINISH, K_BN_BWD_REDUCE, K_BN_BWD_FINISH, K_EW_ADD, K_EW_MASK, K_EW_SUM,
-    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_KINDS
+    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_CONV3_BWD_WEIGHT_TC, K_KINDS
 };
 const char* kernel_name(int kind);
 
@@ -56,6 +56,9 @@ bool conv3_tc_supported(int dtype, const ConvGeom& g);
 // wb: bf16 weights [co][3][3][ci]; wtb: bf16 derived weights [ci][3][3][co]
 void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st);
 void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st);
+bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g);
+void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
+                         cudaStream_t st);
 
 // ---- depthwise 3x3 (weights tap-major: w9c[r*3+s][c]) ----
 void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, cudaStream_t st);

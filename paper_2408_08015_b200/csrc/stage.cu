@@ -442,6 +442,8 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             ValSrc xin = val_src(s, sv, u.in);
             if (u.kind == U_CONV && pw_tc_supported(dt, u.g, false))
                 pw_bwd_weight_tc(u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, s->err, st);
+            else if (u.kind == U_CONV && conv3_wgrad_tc_supported(dt, u.g))
+                conv3_bwd_weight_tc(u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, s->err, st);
             else if (u.kind == U_CONV) conv_bwd_weight(dt, u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, st);
             else dw_bwd_weight(dt, u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, st);
             if (want_in) {
