@@ -134,12 +134,18 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
         // ---- epilogue: warp w reads lane quarter (w & 3); column groups of 8 alternate between the two warp sets ----
         const int q = warp & 3, half = warp >> 2;
         const int row = q * 32 + lane, p = p0 + row;
+        size_t pout = (size_t)p;
+        if (BWD && a.stride > 1 && p < a.P) {      // gradient of a strided 1x1 conv lands on the sampled input pixels
+            int wo = p % a.wo, t = p / a.wo;
+            int ho = t % a.ho, n = t / a.ho;
+            pout = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
+        }
         for (int g = half; g < (NT >> 3); g += 2) {
             float v[8];
             tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g << 3), v);
             int n = n0 + (g << 3);
             if (p < a.P && n < a.N) {
-                size_t e = (size_t)p * a.N + n;
+                size_t e = pout * a.N + n;
                 if (!BWD && a.bias) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) v[i] += __ldg(a.bias + n + i);
@@ -982,7 +988,7 @@ template <bool BWD> void launch(const PwArgs& a0, const Tiling& t, int kind, dou
 }  // namespace
 
 bool pw_tc_supported(int dtype, const ConvGeom& g, bool bwd_data) {
-    if (bwd_data && g.stride != 1) return false;
+    (void)bwd_data;
     return dtype == 1 && g.k == 1 && g.pad == 0 && g.ci % 8 == 0 && g.co % 8 == 0 && g.ci >= 8 && g.co >= 8;
 }
 
@@ -1010,9 +1016,20 @@ void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* w
     PwArgs a{};
     a.dz = dz; a.w = wtb; a.addend = addend; a.out = (__nv_bfloat16*)dx; a.err = err;
     a.P = g.n * g.ho * g.wo; a.K = g.co; a.N = g.ci;
-    a.stride = 1;
+    a.stride = g.stride; a.ho = g.ho; a.wo = g.wo; a.hi = g.hi; a.wi = g.wi;
     double bytes = 2.0 * (double)a.P * a.K * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * (double)a.P * a.N * (addend ? 2.0 : 1.0) +
                    2.0 * a.N * a.K;
+    if (g.stride > 1) {
+        // only the sampled pixels receive a term: the rest of dx is the addend (or zero); the kernel
+        // then accumulates in place at the sampled positions
+        const size_t full = (size_t)g.n * g.hi * g.wi * g.ci * 2;
+        if (!addend) cudaMemsetAsync(dx, 0, full, st);
+        else if (addend != dx) cudaMemcpyAsync(dx, addend, full, cudaMemcpyDeviceToDevice, st);
+        a.addend = dx;
+        Tiling t = pick_tiling(a.K, a.N);
+        launch<true>(a, t, K_PW_BWD_DATA_TC, bytes + (double)full, st);
+        return;
+    }
     {
         PipeArgs pa{};
         pa.dz = dz; pa.w = wtb; pa.addend = addend; pa.out = (__nv_bfloat16*)dx; pa.err = err;
