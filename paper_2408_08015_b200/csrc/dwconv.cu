@@ -269,31 +269,31 @@ template <typename T, int V> struct GradRoll {
     }
 };
 
-template <typename T, int V, bool FLIP, typename LOADER, typename SRC>
+template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC>
 __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, int c, int th, SRC src, const float* __restrict__ w9c,
                                                       const T* addend, T* out) {
-    constexpr int NIN = TW + 2;
+    constexpr int NIN = TWR + 2;
     extern __shared__ float wsm[];            // [9][c], tap order already flipped for the adjoint
     for (int i = threadIdx.x; i < 9 * c; i += blockDim.x) {
         int t = i / c, ch = i - t * c;
         wsm[i] = __ldg(w9c + (FLIP ? 8 - t : t) * c + ch);
     }
     __syncthreads();
-    const int cv = c / V, sw = (w + TW - 1) / TW, nrc = (h + th - 1) / th;
+    const int cv = c / V, sw = (w + TWR - 1) / TWR, nrc = (h + th - 1) / th;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)n_img * nrc * sw * cv) return;
     const int j = (int)(idx % cv);
     size_t sidx = idx / cv;
-    const int wo0 = (int)(sidx % sw) * TW;
+    const int wo0 = (int)(sidx % sw) * TWR;
     size_t t2 = sidx / sw;
     const int oh0 = (int)(t2 % nrc) * th, n = (int)(t2 / nrc);
     const int oh1 = min(h, oh0 + th);
     const int c0 = j * V;
     LOADER ld(src, c0);
     typedef typename LOADER::Raw1 Raw1;
-    float a0[TW][V], a1[TW][V];               // partial sums of output rows ih-1 and ih
+    float a0[TWR][V], a1[TWR][V];               // partial sums of output rows ih-1 and ih
 #pragma unroll
-    for (int t = 0; t < TW; ++t)
+    for (int t = 0; t < TWR; ++t)
 #pragma unroll
         for (int q = 0; q < V; ++q) a0[t][q] = a1[t][q] = 0.f;
     const int wi0 = wo0 - 1;
@@ -320,9 +320,9 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
 #pragma unroll
             for (int q2 = 0; q2 < NIN; ++q2) nxt[q2] = ld.fetch(rb + colc[q2]);
         }
-        float a2[TW][V];
+        float a2[TWR][V];
 #pragma unroll
-        for (int t = 0; t < TW; ++t)
+        for (int t = 0; t < TWR; ++t)
 #pragma unroll
             for (int q = 0; q < V; ++q) a2[t][q] = 0.f;
 #pragma unroll
@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
             *reinterpret_cast<float4*>(w1) = *reinterpret_cast<const float4*>(wsm + (1 * 3 + s) * c + c0);
             *reinterpret_cast<float4*>(w2) = *reinterpret_cast<const float4*>(wsm + (2 * 3 + s) * c + c0);
 #pragma unroll
-            for (int t = 0; t < TW; ++t)
+            for (int t = 0; t < TWR; ++t)
 #pragma unroll
                 for (int q = 0; q < V; ++q) {
                     const float xv = xin[t + s][q];
@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
         const int orow = ih - 1;
         if (orow >= oh0 && orow < oh1) {
 #pragma unroll
-            for (int t = 0; t < TW; ++t) {
+            for (int t = 0; t < TWR; ++t) {
                 if (wo0 + t < w) {
                     size_t e = (((size_t)n * h + orow) * w + wo0 + t) * c + c0;
                     if (addend) {
@@ -358,7 +358,7 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
             }
         }
 #pragma unroll
-        for (int t = 0; t < TW; ++t)
+        for (int t = 0; t < TWR; ++t)
 #pragma unroll
             for (int q = 0; q < V; ++q) {
                 a0[t][q] = a1[t][q];
@@ -367,12 +367,12 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
     }
 }
 
-template <typename T, int V, bool FLIP, typename LOADER, typename SRC>
+template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC>
 void launch_roll(int n, int h, int w, int c, const SRC& src, const float* w9c, const void* addend, void* out, cudaStream_t st) {
     int th = h >= 28 ? 8 : (h >= 14 ? 7 : h);
-    size_t total = (size_t)n * ((h + th - 1) / th) * ((w + TW - 1) / TW) * (c / V);
+    size_t total = (size_t)n * ((h + th - 1) / th) * ((w + TWR - 1) / TWR) * (c / V);
     size_t smem = (size_t)9 * c * sizeof(float);
-    dw_roll_kernel<T, V, FLIP, LOADER, SRC><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
+    dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
 }
 
 // Backward-data at stride 2 (general form): one thread per input pixel and channel vector.
@@ -535,10 +535,10 @@ void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, voi
     LaunchScope ls(K_DW_FWD, (in_e + out_e) * esz(dtype) + 36.0 * g.ci, 18.0 * out_e, st);
     using B = __nv_bfloat16;
     if (dtype == 0) {
-        if (g.stride == 1) launch_roll<float, 4, false, ValRoll<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st);
+        if (g.stride == 1) launch_roll<float, 4, 4, false, ValRoll<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st);
         else launch_strip<float, 4, 2, false, ValLoader<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     } else {
-        if (g.stride == 1) launch_roll<B, 4, false, ValRoll<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st);
+        if (g.stride == 1) launch_roll<B, 4, 4, false, ValRoll<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st);
         else launch_strip<B, 4, 2, false, ValLoader<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     }
 }
@@ -549,8 +549,8 @@ void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w
     using B = __nv_bfloat16;
     if (g.stride == 1) {
         // the adjoint of a stride-1 3x3 correlation is the correlation of dz with the flipped kernel
-        if (dtype == 0) launch_roll<float, 4, true, GradRoll<float, 4>, GradSrc>(g.n, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
-        else launch_roll<B, 4, true, GradRoll<B, 4>, GradSrc>(g.n, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
+        if (dtype == 0) launch_roll<float, 4, 4, true, GradRoll<float, 4>, GradSrc>(g.n, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
+        else launch_roll<B, 4, 2, true, GradRoll<B, 4>, GradSrc>(g.n, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
     } else if (dtype == 0) {
         size_t total = (size_t)g.n * g.hi * g.wi * (g.ci / 4);
         dw_bwd_data_kernel<float, 4><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const float*)addend, (float*)dx);
