@@ -502,6 +502,123 @@ __global__ void __launch_bounds__(256) dw_bwd_weight_kernel(ConvGeom g, GradSrc 
     }
 }
 
+
+// Rolling weight gradient for stride 1: gw[c][r][s] = sum dz[oh][wo] * x[oh-1+r][wo-1+s].
+// A thread owns V channels; a work item is a strip TWR wide and `th` rows high.  Walking down the
+// input rows ih, it holds dz rows ih-1, ih, ih+1 (zero outside the item's rows) and the x row ih:
+// tap row r pairs x row ih with dz row ih+1-r.  Each row of either tensor is loaded and decoded
+// once per item; the next rows' loads are issued before the current row's arithmetic.
+template <typename T, int V, int TWR>
+__global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, int cw, int rows, int th, size_t items_per_block,
+                                                            float* __restrict__ partial) {
+    constexpr int NIN = TWR + 2;
+    extern __shared__ float red[];
+    const int cv = g.ci / V;
+    const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
+    const int j = blockIdx.x * cw + jl;
+    const bool active = row < rows && j < cv;
+    const int c0 = active ? j * V : 0;
+    const int h = g.hi, w = g.wi, c = g.ci;
+    const int sw = (w + TWR - 1) / TWR, nrc = (h + th - 1) / th;
+    const size_t n_items = (size_t)g.n * nrc * sw;
+    const size_t ibeg = (size_t)blockIdx.y * items_per_block, iend = min(n_items, ibeg + items_per_block);
+    float acc[9][V];
+#pragma unroll
+    for (int t = 0; t < 9; ++t)
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[t][q] = 0.f;
+    if (active) {
+        GradRoll<T, V> ldz(dzs, c0);
+        ValRoll<T, V> ldx(xs, c0);
+        typedef typename GradRoll<T, V>::Raw1 RawZ;
+        typedef typename ValRoll<T, V>::Raw1 RawX;
+        for (size_t item = ibeg + row; item < iend; item += rows) {
+            const int wo0 = (int)(item % sw) * TWR;
+            size_t t2 = item / sw;
+            const int oh0 = (int)(t2 % nrc) * th, n = (int)(t2 / nrc);
+            const int oh1 = min(h, oh0 + th);
+            int xcol[NIN], zcol[TWR];
+            bool xok[NIN], zok[TWR];
+#pragma unroll
+            for (int q2 = 0; q2 < NIN; ++q2) {
+                const int wi = wo0 - 1 + q2;
+                xok[q2] = wi >= 0 && wi < w;
+                xcol[q2] = min(max(wi, 0), w - 1) * c + c0;
+            }
+#pragma unroll
+            for (int t = 0; t < TWR; ++t) {
+                zok[t] = wo0 + t < w;
+                zcol[t] = min(wo0 + t, w - 1) * c + c0;
+            }
+            float dzm[TWR][V], dz0[TWR][V], dzp[TWR][V];
+#pragma unroll
+            for (int t = 0; t < TWR; ++t)
+#pragma unroll
+                for (int q = 0; q < V; ++q) dzm[t][q] = dz0[t][q] = 0.f;
+            RawX nx[NIN];
+            RawZ nz[TWR];
+            {   // first x row (oh0-1, clamped) and first dz row (oh0)
+                const size_t rbx = ((size_t)n * h + max(oh0 - 1, 0)) * w * c, rbz = ((size_t)n * h + oh0) * w * c;
+#pragma unroll
+                for (int q2 = 0; q2 < NIN; ++q2) nx[q2] = ldx.fetch(rbx + xcol[q2]);
+#pragma unroll
+                for (int t = 0; t < TWR; ++t) nz[t] = ldz.fetch(rbz + zcol[t]);
+            }
+            for (int ih = oh0 - 1; ih <= oh1; ++ih) {
+                const bool xrow_ok = ih >= 0 && ih < h;
+                const bool zrow_ok = ih + 1 >= oh0 && ih + 1 < oh1;
+                float xin[NIN][V];
+#pragma unroll
+                for (int q2 = 0; q2 < NIN; ++q2) ldx.decode(nx[q2], xrow_ok && xok[q2], xin[q2]);
+#pragma unroll
+                for (int t = 0; t < TWR; ++t) ldz.decode(nz[t], zrow_ok && zok[t], dzp[t]);
+                if (ih < oh1) {     // next rows: x row ih+1, dz row ih+2 (addresses clamped into the image)
+                    const size_t rbx = ((size_t)n * h + min(ih + 1, h - 1)) * w * c, rbz = ((size_t)n * h + min(ih + 2, h - 1)) * w * c;
+#pragma unroll
+                    for (int q2 = 0; q2 < NIN; ++q2) nx[q2] = ldx.fetch(rbx + xcol[q2]);
+#pragma unroll
+                    for (int t = 0; t < TWR; ++t) nz[t] = ldz.fetch(rbz + zcol[t]);
+                }
+#pragma unroll
+                for (int s = 0; s < 3; ++s)
+#pragma unroll
+                    for (int t = 0; t < TWR; ++t)
+#pragma unroll
+                        for (int q = 0; q < V; ++q) {
+                            const float xv = xin[t + s][q];
+                            acc[0 * 3 + s][q] = fmaf(dzp[t][q], xv, acc[0 * 3 + s][q]);
+                            acc[1 * 3 + s][q] = fmaf(dz0[t][q], xv, acc[1 * 3 + s][q]);
+                            acc[2 * 3 + s][q] = fmaf(dzm[t][q], xv, acc[2 * 3 + s][q]);
+                        }
+#pragma unroll
+                for (int t = 0; t < TWR; ++t)
+#pragma unroll
+                    for (int q = 0; q < V; ++q) {
+                        dzm[t][q] = dz0[t][q];
+                        dz0[t][q] = dzp[t][q];
+                    }
+            }
+        }
+    }
+    const int width = cw * V;
+    for (int t = 0; t < 9; ++t) {
+        if (row < rows) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) red[row * width + jl * V + q] = acc[t][q];
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < width; e += blockDim.x) {
+            int ch = blockIdx.x * width + e;
+            if (ch < g.ci) {
+                float s = 0.f;
+                for (int r2 = 0; r2 < rows; ++r2) s += red[r2 * width + e];
+                partial[((size_t)blockIdx.y * 9 + t) * g.ci + ch] = s;
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // gw[c][t] = sum_b partial[b][t][c]; one warp per (t, c): lanes stride over the blocks
 __global__ void __launch_bounds__(128) dw_bwd_weight_finish(const float* __restrict__ partial, int blocks, int c_total, float* __restrict__ gw) {
     int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -562,6 +679,37 @@ void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w
 
 void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw,
                    cudaStream_t st) {
+    if (g.stride == 1) {
+        constexpr int TWR = 2;
+        const int V = 4;
+        const int cv = g.ci / V;
+        const int parts = (cv + 47) / 48;              // channel-vector columns per block: an even split, at most 48
+        int cw = (cv + parts - 1) / parts;
+        int rows = 128 / cw;
+        const int th = g.hi >= 28 ? 8 : (g.hi >= 14 ? 7 : g.hi);
+        const int sw = (g.wi + TWR - 1) / TWR, nrc = (g.hi + th - 1) / th;
+        size_t n_items = (size_t)g.n * nrc * sw;
+        int gx = (cv + cw - 1) / cw;
+        size_t by = (8 * 148 + gx - 1) / gx;
+        size_t max_by = (n_items + (size_t)rows - 1) / (size_t)rows;
+        if (by > max_by) by = max_by;
+        size_t cap = scratch_floats / ((size_t)9 * g.ci);
+        if (by > cap) by = cap;
+        if (by < 1) by = 1;
+        size_t ipb = (n_items + by - 1) / by;
+        by = (n_items + ipb - 1) / ipb;
+        size_t smem = (size_t)rows * cw * V * sizeof(float);
+        dim3 grid(gx, (unsigned)by);
+        double in_e = (double)g.n * g.hi * g.wi * g.ci;
+        {
+            LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, in_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * in_e, st);
+            if (dtype == 0) dw_wgrad_roll_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+            else dw_wgrad_roll_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+        }
+        LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
+        dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
+        return;
+    }
     const int V = 4;
     const int cv = g.ci / V;
     int cw = cv < 64 ? cv : 64;
