@@ -115,7 +115,7 @@ ReducePlan plan_reduce(int dtype, size_t pixels, int c, int nacc, size_t scratch
     p.cw = cg < 32 ? cg : 32;
     p.rows = 256 / p.cw;
     p.gx = (cg + p.cw - 1) / p.cw;
-    size_t by = (4 * 148 + p.gx - 1) / p.gx;
+    size_t by = (2 * 148 + p.gx - 1) / p.gx;
     size_t max_by = (pixels + (size_t)p.rows * 4 - 1) / ((size_t)p.rows * 4);
     if (by > max_by) by = max_by;
     size_t cap = scratch_floats / ((size_t)nacc * c);
