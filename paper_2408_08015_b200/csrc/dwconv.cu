@@ -13,7 +13,7 @@ namespace {
 
 constexpr int TW = 4;
 
-// ---- V-wide raw access: (float,4) and (bf16,8) are 16-byte, (bf16,4) 8-byte ----
+// ---- V-wide raw access: (float,4) is 16-byte, (bf16,4) 8-byte ----
 template <typename T, int V> struct Raw;
 template <> struct Raw<float, 4> {
     static __device__ __forceinline__ void ld(const void* p, size_t e, float* f) {
@@ -22,18 +22,6 @@ template <> struct Raw<float, 4> {
     }
     static __device__ __forceinline__ void st(void* p, size_t e, const float* f) {
         *reinterpret_cast<float4*>(reinterpret_cast<float*>(p) + e) = make_float4(f[0], f[1], f[2], f[3]);
-    }
-};
-template <> struct Raw<__nv_bfloat16, 8> {
-    static __device__ __forceinline__ void ld(const void* p, size_t e, float* f) {
-        Vec<__nv_bfloat16> v;
-        v.load(p, e >> 3);
-        v.unpack(f);
-    }
-    static __device__ __forceinline__ void st(void* p, size_t e, const float* f) {
-        Vec<__nv_bfloat16> v;
-        v.pack(f);
-        v.store(p, e >> 3);
     }
 };
 template <> struct Raw<__nv_bfloat16, 4> {
@@ -375,133 +363,6 @@ void launch_roll(int n, int h, int w, int c, const SRC& src, const float* w9c, c
     dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
 }
 
-// Backward-data at stride 2 (general form): one thread per input pixel and channel vector.
-template <typename T, int V>
-__global__ void __launch_bounds__(256) dw_bwd_data_kernel(ConvGeom g, GradSrc dz, const float* __restrict__ w9c, const T* addend, T* dx) {
-    const int cv = g.ci / V;
-    size_t total = (size_t)g.n * g.hi * g.wi * cv;
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    int j = (int)(i % cv);
-    size_t p = i / cv;
-    int wi = (int)(p % g.wi);
-    size_t t = p / g.wi;
-    int hi = (int)(t % g.hi), n = (int)(t / g.hi);
-    int c0 = j * V;
-    GradLoader<T, V> ld(dz, c0);
-    float acc[V];
-    if (addend) {
-        Raw<T, V>::ld(addend, p * g.ci + c0, acc);
-    } else {
-#pragma unroll
-        for (int q = 0; q < V; ++q) acc[q] = 0.f;
-    }
-#pragma unroll
-    for (int r = 0; r < 3; ++r) {
-        int a = hi + 1 - r;
-        if (a < 0 || (g.stride == 2 && (a & 1))) continue;
-        int ho = a / g.stride;
-        if (ho >= g.ho) continue;
-#pragma unroll
-        for (int s = 0; s < 3; ++s) {
-            int b = wi + 1 - s;
-            if (b < 0 || (g.stride == 2 && (b & 1))) continue;
-            int wo = b / g.stride;
-            if (wo >= g.wo) continue;
-            float dv[V], wv[V];
-            ld.load((((size_t)n * g.ho + ho) * g.wo + wo) * g.ci + c0, dv);
-            ld_coef<V>(w9c + (r * 3 + s) * g.ci, c0, wv);
-#pragma unroll
-            for (int q = 0; q < V; ++q) acc[q] = fmaf(dv[q], wv[q], acc[q]);
-        }
-    }
-    Raw<T, V>::st(dx, p * g.ci + c0, acc);
-}
-
-// Weight gradient: gw[c][r][s] = sum over output pixels of dz * x(tap).  A block owns `cw`
-// channel vectors; thread (row, jl) walks output strips with stride `rows`, keeping 9*V sums
-// in registers.  Rows are combined through shared memory, blocks through a partials array
-// summed in fixed order by a second kernel (deterministic, no float atomics).
-template <typename T, int V, int S>
-__global__ void __launch_bounds__(256) dw_bwd_weight_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, int cw, int rows, size_t strips_per_block,
-                                                            float* __restrict__ partial) {
-    constexpr int NIN = (TW - 1) * S + 3;
-    extern __shared__ float red[];
-    const int cv = g.ci / V;
-    const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
-    const int j = blockIdx.x * cw + jl;
-    const bool active = row < rows && j < cv;
-    const int c0 = active ? j * V : 0;
-    const int sw = (g.wo + TW - 1) / TW;
-    const size_t n_strips = (size_t)g.n * g.ho * sw;
-    const size_t sbeg = (size_t)blockIdx.y * strips_per_block, send = min(n_strips, sbeg + strips_per_block);
-    float acc[9][V];
-#pragma unroll
-    for (int t = 0; t < 9; ++t)
-#pragma unroll
-        for (int q = 0; q < V; ++q) acc[t][q] = 0.f;
-    if (active) {
-        GradLoader<T, V> ldz(dzs, c0);
-        ValLoader<T, V> ldx(xs, c0);
-        for (size_t sidx = sbeg + row; sidx < send; sidx += rows) {
-            const int wo0 = (int)(sidx % sw) * TW;
-            size_t t2 = sidx / sw;
-            const int oh = (int)(t2 % g.ho), n = (int)(t2 / g.ho);
-            float dv[TW][V];
-#pragma unroll
-            for (int t = 0; t < TW; ++t) {
-                if (wo0 + t < g.wo) {
-                    ldz.load((((size_t)n * g.ho + oh) * g.wo + wo0 + t) * g.ci + c0, dv[t]);
-                } else {
-#pragma unroll
-                    for (int q = 0; q < V; ++q) dv[t][q] = 0.f;
-                }
-            }
-            const int wi0 = wo0 * S - 1;
-#pragma unroll
-            for (int r = 0; r < 3; ++r) {
-                const int ih = oh * S - 1 + r;
-                if (ih < 0 || ih >= g.hi) continue;
-                float xin[NIN][V];
-                const size_t rowbase = ((size_t)n * g.hi + ih) * g.wi;
-#pragma unroll
-                for (int q2 = 0; q2 < NIN; ++q2) {
-                    const int iw = wi0 + q2;
-                    if (iw >= 0 && iw < g.wi) {
-                        ldx.load((rowbase + iw) * g.ci + c0, xin[q2]);
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < V; ++q) xin[q2][q] = 0.f;
-                    }
-                }
-#pragma unroll
-                for (int s = 0; s < 3; ++s)
-#pragma unroll
-                    for (int t = 0; t < TW; ++t)
-#pragma unroll
-                        for (int q = 0; q < V; ++q) acc[r * 3 + s][q] = fmaf(dv[t][q], xin[t * S + s][q], acc[r * 3 + s][q]);
-            }
-        }
-    }
-    const int width = cw * V;
-    for (int t = 0; t < 9; ++t) {
-        if (row < rows) {
-#pragma unroll
-            for (int q = 0; q < V; ++q) red[row * width + jl * V + q] = acc[t][q];
-        }
-        __syncthreads();
-        for (int e = threadIdx.x; e < width; e += blockDim.x) {
-            int ch = blockIdx.x * width + e;
-            if (ch < g.ci) {
-                float s = 0.f;
-                for (int r2 = 0; r2 < rows; ++r2) s += red[r2 * width + e];
-                partial[((size_t)blockIdx.y * 9 + t) * g.ci + ch] = s;
-            }
-        }
-        __syncthreads();
-    }
-}
-
 
 // Rolling weight gradient for stride 1: gw[c][r][s] = sum dz[oh][wo] * x[oh-1+r][wo-1+s].
 // A thread owns V channels; a work item is a strip TWR wide and `th` rows high.  Walking down the
@@ -619,6 +480,231 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Stride-2 backward kernels, rolling over the rows of dz.
+// Forward: z(ho,wo) = sum_{r,s} x(2ho-1+r, 2wo-1+s) w(r,s).  Hence an even input row 2i receives
+// only tap row 1 of dz row i; an odd input row 2i+1 receives tap row 2 of dz row i and tap row 0
+// of dz row i+1; columns likewise.  A thread owns V channels and TWZ columns of dz (plus one
+// halo column), walks down the dz rows keeping rows i and i+1, and writes the two input rows
+// 2i, 2i+1 (2*TWZ columns each).  Every dz element is loaded and transformed once per thread.
+template <typename T, int V, int TWZ>
+__global__ void __launch_bounds__(128) dw_bwd_data_s2_kernel(ConvGeom g, GradSrc dzs, const float* __restrict__ w9c, int th, const T* addend, T* dx) {
+    extern __shared__ float wsm[];            // [9][c]
+    const int c = g.ci, H = g.hi, W = g.wi, Ho = g.ho, Wo = g.wo;
+    for (int i = threadIdx.x; i < 9 * c; i += blockDim.x) wsm[i] = __ldg(w9c + i);
+    __syncthreads();
+    const int cv = c / V;
+    const int nrowz = (H + 1) / 2, ncolz = (W + 1) / 2;              // dz rows / columns that own input rows / columns
+    const int swz = (ncolz + TWZ - 1) / TWZ, nrc = (nrowz + th - 1) / th;
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)g.n * nrc * swz * cv) return;
+    const int j = (int)(idx % cv);
+    size_t sidx = idx / cv;
+    const int jz0 = (int)(sidx % swz) * TWZ;
+    size_t t2 = sidx / swz;
+    const int i0 = (int)(t2 % nrc) * th, n = (int)(t2 / nrc);
+    const int i1 = min(nrowz, i0 + th);
+    const int c0 = j * V;
+    GradRoll<T, V> ld(dzs, c0);
+    typedef typename GradRoll<T, V>::Raw1 Raw1;
+    float wt[9][V];
+#pragma unroll
+    for (int t = 0; t < 9; ++t) *reinterpret_cast<float4*>(wt[t]) = *reinterpret_cast<const float4*>(wsm + t * c + c0);
+    int zcol[TWZ + 1];
+    bool zok[TWZ + 1];
+#pragma unroll
+    for (int q2 = 0; q2 <= TWZ; ++q2) {
+        zok[q2] = jz0 + q2 < Wo;
+        zcol[q2] = min(jz0 + q2, Wo - 1) * c + c0;
+    }
+    float cur[TWZ + 1][V], nxt[TWZ + 1][V];
+    Raw1 raw[TWZ + 1];
+    {   // dz row i0 decoded into cur; raw of row i0+1 requested
+        const size_t rb = ((size_t)n * Ho + min(i0, Ho - 1)) * Wo * c;
+#pragma unroll
+        for (int q2 = 0; q2 <= TWZ; ++q2) raw[q2] = ld.fetch(rb + zcol[q2]);
+#pragma unroll
+        for (int q2 = 0; q2 <= TWZ; ++q2) ld.decode(raw[q2], zok[q2] && i0 < Ho, cur[q2]);
+        const size_t rb1 = ((size_t)n * Ho + min(i0 + 1, Ho - 1)) * Wo * c;
+#pragma unroll
+        for (int q2 = 0; q2 <= TWZ; ++q2) raw[q2] = ld.fetch(rb1 + zcol[q2]);
+    }
+    for (int i = i0; i < i1; ++i) {
+#pragma unroll
+        for (int q2 = 0; q2 <= TWZ; ++q2) ld.decode(raw[q2], zok[q2] && i + 1 < Ho, nxt[q2]);
+        if (i + 1 < i1) {
+            const size_t rb = ((size_t)n * Ho + min(i + 2, Ho - 1)) * Wo * c;
+#pragma unroll
+            for (int q2 = 0; q2 <= TWZ; ++q2) raw[q2] = ld.fetch(rb + zcol[q2]);
+        }
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+            const int hi = 2 * i + a;
+            if (hi >= H) continue;
+#pragma unroll
+            for (int t = 0; t < TWZ; ++t) {
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    const int wi = 2 * (jz0 + t) + b;
+                    if (wi >= W) continue;
+                    float o[V];
+#pragma unroll
+                    for (int q = 0; q < V; ++q) {
+                        float v;
+                        if (a == 0 && b == 0) {
+                            v = cur[t][q] * wt[4][q];
+                        } else if (a == 0) {
+                            v = fmaf(cur[t][q], wt[5][q], cur[t + 1][q] * wt[3][q]);
+                        } else if (b == 0) {
+                            v = fmaf(cur[t][q], wt[7][q], nxt[t][q] * wt[1][q]);
+                        } else {
+                            v = fmaf(cur[t][q], wt[8][q], fmaf(cur[t + 1][q], wt[6][q], fmaf(nxt[t][q], wt[2][q], nxt[t + 1][q] * wt[0][q])));
+                        }
+                        o[q] = v;
+                    }
+                    const size_t e = (((size_t)n * H + hi) * W + wi) * c + c0;
+                    if (addend) {
+                        float ad[V];
+                        Raw<T, V>::ld(addend, e, ad);
+#pragma unroll
+                        for (int q = 0; q < V; ++q) o[q] += ad[q];
+                    }
+                    Raw<T, V>::st(dx, e, o);
+                }
+            }
+        }
+#pragma unroll
+        for (int q2 = 0; q2 <= TWZ; ++q2)
+#pragma unroll
+            for (int q = 0; q < V; ++q) cur[q2][q] = nxt[q2][q];
+    }
+}
+
+// Stride-2 weight gradient: gw[c][r][s] = sum dz(ho,wo) x(2ho-1+r, 2wo-1+s).  A work item is TWZ
+// columns by `th` rows of dz; walking down the dz rows, x row 2ho+1 of one step is x row 2ho'-1 of
+// the next, so each x row is loaded and transformed once.
+template <typename T, int V, int TWZ>
+__global__ void __launch_bounds__(128) dw_wgrad_s2_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, int cw, int rows, int th, size_t items_per_block,
+                                                          float* __restrict__ partial) {
+    constexpr int NX = 2 * TWZ + 1;
+    extern __shared__ float red[];
+    const int cv = g.ci / V;
+    const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
+    const int j = blockIdx.x * cw + jl;
+    const bool active = row < rows && j < cv;
+    const int c0 = active ? j * V : 0;
+    const int H = g.hi, W = g.wi, Ho = g.ho, Wo = g.wo, c = g.ci;
+    const int swz = (Wo + TWZ - 1) / TWZ, nrc = (Ho + th - 1) / th;
+    const size_t n_items = (size_t)g.n * nrc * swz;
+    const size_t ibeg = (size_t)blockIdx.y * items_per_block, iend = min(n_items, ibeg + items_per_block);
+    float acc[9][V];
+#pragma unroll
+    for (int t = 0; t < 9; ++t)
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[t][q] = 0.f;
+    if (active) {
+        GradRoll<T, V> ldz(dzs, c0);
+        ValRoll<T, V> ldx(xs, c0);
+        typedef typename GradRoll<T, V>::Raw1 RawZ;
+        typedef typename ValRoll<T, V>::Raw1 RawX;
+        for (size_t item = ibeg + row; item < iend; item += rows) {
+            const int wo0 = (int)(item % swz) * TWZ;
+            size_t t2 = item / swz;
+            const int oh0 = (int)(t2 % nrc) * th, n = (int)(t2 / nrc);
+            const int oh1 = min(Ho, oh0 + th);
+            int xcol[NX], zcol[TWZ];
+            bool xok[NX], zok[TWZ];
+#pragma unroll
+            for (int q2 = 0; q2 < NX; ++q2) {
+                const int wi = 2 * wo0 - 1 + q2;
+                xok[q2] = wi >= 0 && wi < W;
+                xcol[q2] = min(max(wi, 0), W - 1) * c + c0;
+            }
+#pragma unroll
+            for (int t = 0; t < TWZ; ++t) {
+                zok[t] = wo0 + t < Wo;
+                zcol[t] = min(wo0 + t, Wo - 1) * c + c0;
+            }
+            float xp[NX][V];     // x row 2ho-1
+            {
+                const int ih = 2 * oh0 - 1;
+                const size_t rb = ((size_t)n * H + max(ih, 0)) * W * c;
+#pragma unroll
+                for (int q2 = 0; q2 < NX; ++q2) {
+                    RawX r = ldx.fetch(rb + xcol[q2]);
+                    ldx.decode(r, ih >= 0 && xok[q2], xp[q2]);
+                }
+            }
+            RawX nxa[NX], nxb[NX];
+            RawZ nz[TWZ];
+            {
+                const size_t ra = ((size_t)n * H + min(2 * oh0, H - 1)) * W * c, rb = ((size_t)n * H + min(2 * oh0 + 1, H - 1)) * W * c;
+                const size_t rz = ((size_t)n * Ho + oh0) * Wo * c;
+#pragma unroll
+                for (int q2 = 0; q2 < NX; ++q2) {
+                    nxa[q2] = ldx.fetch(ra + xcol[q2]);
+                    nxb[q2] = ldx.fetch(rb + xcol[q2]);
+                }
+#pragma unroll
+                for (int t = 0; t < TWZ; ++t) nz[t] = ldz.fetch(rz + zcol[t]);
+            }
+            for (int oh = oh0; oh < oh1; ++oh) {
+                float xa[NX][V], xb[NX][V], dv[TWZ][V];
+#pragma unroll
+                for (int q2 = 0; q2 < NX; ++q2) {
+                    ldx.decode(nxa[q2], 2 * oh < H && xok[q2], xa[q2]);
+                    ldx.decode(nxb[q2], 2 * oh + 1 < H && xok[q2], xb[q2]);
+                }
+#pragma unroll
+                for (int t = 0; t < TWZ; ++t) ldz.decode(nz[t], zok[t], dv[t]);
+                if (oh + 1 < oh1) {
+                    const size_t ra = ((size_t)n * H + min(2 * oh + 2, H - 1)) * W * c, rb = ((size_t)n * H + min(2 * oh + 3, H - 1)) * W * c;
+                    const size_t rz = ((size_t)n * Ho + oh + 1) * Wo * c;
+#pragma unroll
+                    for (int q2 = 0; q2 < NX; ++q2) {
+                        nxa[q2] = ldx.fetch(ra + xcol[q2]);
+                        nxb[q2] = ldx.fetch(rb + xcol[q2]);
+                    }
+#pragma unroll
+                    for (int t = 0; t < TWZ; ++t) nz[t] = ldz.fetch(rz + zcol[t]);
+                }
+#pragma unroll
+                for (int s = 0; s < 3; ++s)
+#pragma unroll
+                    for (int t = 0; t < TWZ; ++t)
+#pragma unroll
+                        for (int q = 0; q < V; ++q) {
+                            acc[0 * 3 + s][q] = fmaf(dv[t][q], xp[2 * t + s][q], acc[0 * 3 + s][q]);
+                            acc[1 * 3 + s][q] = fmaf(dv[t][q], xa[2 * t + s][q], acc[1 * 3 + s][q]);
+                            acc[2 * 3 + s][q] = fmaf(dv[t][q], xb[2 * t + s][q], acc[2 * 3 + s][q]);
+                        }
+#pragma unroll
+                for (int q2 = 0; q2 < NX; ++q2)
+#pragma unroll
+                    for (int q = 0; q < V; ++q) xp[q2][q] = xb[q2][q];
+            }
+        }
+    }
+    const int width = cw * V;
+    for (int t = 0; t < 9; ++t) {
+        if (row < rows) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) red[row * width + jl * V + q] = acc[t][q];
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < width; e += blockDim.x) {
+            int ch = blockIdx.x * width + e;
+            if (ch < g.ci) {
+                float s = 0.f;
+                for (int r2 = 0; r2 < rows; ++r2) s += red[r2 * width + e];
+                partial[((size_t)blockIdx.y * 9 + t) * g.ci + ch] = s;
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // gw[c][t] = sum_b partial[b][t][c]; one warp per (t, c): lanes stride over the blocks
 __global__ void __launch_bounds__(128) dw_bwd_weight_finish(const float* __restrict__ partial, int blocks, int c_total, float* __restrict__ gw) {
     int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -668,26 +754,28 @@ void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w
         // the adjoint of a stride-1 3x3 correlation is the correlation of dz with the flipped kernel
         if (dtype == 0) launch_roll<float, 4, 4, true, GradRoll<float, 4>, GradSrc>(g.n, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
         else launch_roll<B, 4, 2, true, GradRoll<B, 4>, GradSrc>(g.n, g.hi, g.wi, g.ci, dz, w9c, addend, dx, st);
-    } else if (dtype == 0) {
-        size_t total = (size_t)g.n * g.hi * g.wi * (g.ci / 4);
-        dw_bwd_data_kernel<float, 4><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const float*)addend, (float*)dx);
     } else {
-        size_t total = (size_t)g.n * g.hi * g.wi * (g.ci / 8);
-        dw_bwd_data_kernel<B, 8><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(g, dz, w9c, (const B*)addend, (B*)dx);
+        constexpr int TWZ = 2;
+        const int nrowz = (g.hi + 1) / 2, ncolz = (g.wi + 1) / 2;
+        const int th = nrowz >= 14 ? 7 : nrowz;
+        size_t total = (size_t)g.n * ((nrowz + th - 1) / th) * ((ncolz + TWZ - 1) / TWZ) * (g.ci / 4);
+        size_t smem = (size_t)9 * g.ci * sizeof(float);
+        if (dtype == 0) dw_bwd_data_s2_kernel<float, 4, TWZ><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(g, dz, w9c, th, (const float*)addend, (float*)dx);
+        else dw_bwd_data_s2_kernel<B, 4, TWZ><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(g, dz, w9c, th, (const B*)addend, (B*)dx);
     }
 }
 
 void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw,
                    cudaStream_t st) {
-    if (g.stride == 1) {
+    {
         constexpr int TWR = 2;
         const int V = 4;
         const int cv = g.ci / V;
         const int parts = (cv + 47) / 48;              // channel-vector columns per block: an even split, at most 48
         int cw = (cv + parts - 1) / parts;
         int rows = 128 / cw;
-        const int th = g.hi >= 28 ? 8 : (g.hi >= 14 ? 7 : g.hi);
-        const int sw = (g.wi + TWR - 1) / TWR, nrc = (g.hi + th - 1) / th;
+        const int th = g.ho >= 28 ? 8 : (g.ho >= 14 ? 7 : g.ho);      // rows of dz per work item
+        const int sw = (g.wo + TWR - 1) / TWR, nrc = (g.ho + th - 1) / th;
         size_t n_items = (size_t)g.n * nrc * sw;
         int gx = (cv + cw - 1) / cw;
         size_t by = (8 * 148 + gx - 1) / gx;
@@ -700,47 +788,20 @@ void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc
         by = (n_items + ipb - 1) / ipb;
         size_t smem = (size_t)rows * cw * V * sizeof(float);
         dim3 grid(gx, (unsigned)by);
-        double in_e = (double)g.n * g.hi * g.wi * g.ci;
+        double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
         {
-            LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, in_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * in_e, st);
-            if (dtype == 0) dw_wgrad_roll_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
-            else dw_wgrad_roll_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+            LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
+            if (g.stride == 1) {
+                if (dtype == 0) dw_wgrad_roll_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+                else dw_wgrad_roll_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+            } else {
+                if (dtype == 0) dw_wgrad_s2_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+                else dw_wgrad_s2_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+            }
         }
         LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
         dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
-        return;
     }
-    const int V = 4;
-    const int cv = g.ci / V;
-    int cw = cv < 64 ? cv : 64;
-    int rows = 256 / cw;
-    const int sw = (g.wo + TW - 1) / TW;
-    size_t n_strips = (size_t)g.n * g.ho * sw;
-    int gx = (cv + cw - 1) / cw;
-    size_t by = (4 * 148 + gx - 1) / gx;
-    size_t max_by = (n_strips + (size_t)rows * 2 - 1) / ((size_t)rows * 2);
-    if (by > max_by) by = max_by;
-    size_t cap = scratch_floats / ((size_t)9 * g.ci);
-    if (by > cap) by = cap;
-    if (by < 1) by = 1;
-    size_t spb = (n_strips + by - 1) / by;
-    by = (n_strips + spb - 1) / spb;
-    size_t smem = (size_t)rows * cw * V * sizeof(float);
-    dim3 grid(gx, (unsigned)by);
-    double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
-    using B = __nv_bfloat16;
-    {
-        LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
-        if (dtype == 0) {
-            if (g.stride == 1) dw_bwd_weight_kernel<float, 4, 1><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
-            else dw_bwd_weight_kernel<float, 4, 2><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
-        } else {
-            if (g.stride == 1) dw_bwd_weight_kernel<B, 4, 1><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
-            else dw_bwd_weight_kernel<B, 4, 2><<<grid, 256, smem, st>>>(g, dz, x, cw, rows, spb, scratch);
-        }
-    }
-    LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
-    dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
 }
 
 }  // namespace ast
