@@ -350,17 +350,18 @@ __global__ void reduce_splits_tc(const float* __restrict__ partial, int splits, 
 //               shared-memory stages; a tile of consecutive pixels is one contiguous byte range
 //   warp 1      MMA issuer: tcgen05.mma over the staged operand into one of two accumulators in
 //               tensor memory; tcgen05.commit releases the operand stage and publishes the tile
-//   warps 2-5   transformers: read a raw stage, apply BatchNorm+activation (or the
+//   warps 2-9   transformers: read a raw stage, apply BatchNorm+activation (or the
 //               BatchNorm-backward transform) with per-thread register-held coefficients,
 //               write bf16 into the swizzled K-major operand stage
-//   warps 6-9   epilogue: tcgen05.ld the finished accumulator, add bias / residual gradient,
+//   warps 10-13 epilogue: tcgen05.ld the finished accumulator, add bias / residual gradient,
 //               store bf16 to global
 //
 // Copy, transform, MMA and store of consecutive tiles overlap.  The weights stay resident in
 // shared memory.  Every wait is bounded; a wait that runs out raises a CTA-wide abort flag, every
 // role leaves its loop, outstanding bulk copies are waited for, tensor memory is freed and the
 // error word is set.
-constexpr int PIPE_THREADS = 320;
+constexpr int PIPE_THREADS = 448;     // producer, MMA issuer, 8 transform warps, 4 epilogue warps
+constexpr int PIPE_XF = 256;          // transform threads
 constexpr int MAX_RAW = 8;
 
 struct PipeArgs {
@@ -402,10 +403,10 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
     if (tid == 0) {
         for (int s = 0; s < R; ++s) {
             mbar_init(raw_full(s), 1);
-            mbar_init(raw_empty(s), 128);
+            mbar_init(raw_empty(s), PIPE_XF);
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(a_full(s), 128);
+            mbar_init(a_full(s), PIPE_XF);
             mbar_init(a_empty(s), 1);
             mbar_init(acc_full(s), 1);
             mbar_init(acc_empty(s), 128);
@@ -487,10 +488,10 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
                 umma_commit(acc_full(st));
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 10) {
         // ------------------------------------------------------------ transformers
         const int tix = tid - 64;
-        const int groups = 128 / vpr_pad;                 // row groups; thread (grp, j) owns chunk j of rows grp, grp+groups, ...
+        const int groups = PIPE_XF / vpr_pad;             // row groups; thread (grp, j) owns chunk j of rows grp, grp+groups, ...
         const int j = tix % vpr_pad, grp = tix / vpr_pad;
         const bool active = grp < groups;
         const bool data = j < vpr;                        // chunks beyond K are zero padding
@@ -535,6 +536,7 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
                 }
                 const uint8_t* raw = sR + (size_t)s * a.raw_bytes;
                 if (active) {
+#pragma unroll 4
                     for (int rl = grp; rl < RS; rl += groups) {
                         const int r = sub * RS + rl;
                         uint4 q4 = make_uint4(0, 0, 0, 0);
@@ -823,6 +825,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
             uint8_t* dst = sOp + (size_t)st * a.op_bytes + (isA ? 0u : (uint32_t)a.pa * PANEL) + (uint32_t)(jc >> 3) * PANEL;
             const int valid = min(WSTAGE, pend - (pbeg + it * WSTAGE));
             if (active) {
+#pragma unroll 4
                 for (int kr = grp; kr < WSTAGE; kr += groups) {
                     uint4 q4 = make_uint4(0, 0, 0, 0);
                     if (kr < valid) {
