@@ -360,6 +360,62 @@ __global__ void reduce_splits_tc(const float* __restrict__ partial, int splits, 
 // shared memory.  Every wait is bounded; a wait that runs out raises a CTA-wide abort flag, every
 // role leaves its loop, outstanding bulk copies are waited for, tensor memory is freed and the
 // error word is set.
+// Branch-free operand transforms with per-thread register coefficients.  Absent BatchNorm
+// terms take neutral values (scale 1, shift 0, k1 1, k2 = k3 0) and the activation becomes a pair
+// of bounds (ReLU6: 0..6, ReLU: 0..inf, none: -inf..inf), so that every lane runs the same
+// instruction stream whatever its operand.
+struct XfVal {
+    float cs[8], ch[8], lo, hi;
+    __device__ __forceinline__ void init(const ValSrc& s, int c0) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            cs[q] = s.scale ? __ldg(s.scale + c0 + q) : 1.f;
+            ch[q] = s.scale ? __ldg(s.shift + c0 + q) : 0.f;
+        }
+        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
+        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
+    }
+    __device__ __forceinline__ uint4 apply(const uint4& raw) const {
+        Vec<__nv_bfloat16> v;
+        v.raw = raw;
+        float f[8];
+        v.unpack(f);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) f[q] = fminf(fmaxf(fmaf(f[q], cs[q], ch[q]), lo), hi);
+        return pack8(f);
+    }
+};
+struct XfGrad {
+    float cs[8], ch[8], k1[8], k2[8], k3[8], lo, hi;
+    __device__ __forceinline__ void init(const GradSrc& s, int c0) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            cs[q] = s.scale ? __ldg(s.scale + c0 + q) : 1.f;
+            ch[q] = s.scale ? __ldg(s.shift + c0 + q) : 0.f;
+            k1[q] = s.k1 ? __ldg(s.k1 + c0 + q) : 1.f;
+            k2[q] = s.k1 ? __ldg(s.k2 + c0 + q) : 0.f;
+            k3[q] = s.k1 ? __ldg(s.k3 + c0 + q) : 0.f;
+        }
+        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
+        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
+    }
+    __device__ __forceinline__ uint4 apply(const uint4& rawdy, const uint4& rawz) const {
+        Vec<__nv_bfloat16> v;
+        float f[8], z[8];
+        v.raw = rawdy;
+        v.unpack(f);
+        v.raw = rawz;
+        v.unpack(z);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float pre = fmaf(z[q], cs[q], ch[q]);
+            const float d = (pre > lo && pre < hi) ? f[q] : 0.f;
+            f[q] = fmaf(k1[q], d, fmaf(k3[q], z[q], k2[q]));
+        }
+        return pack8(f);
+    }
+};
+
 constexpr int PIPE_THREADS = 448;     // producer, MMA issuer, 8 transform warps, 4 epilogue warps
 constexpr int PIPE_XF = 256;          // transform threads
 constexpr int MAX_RAW = 8;
@@ -495,32 +551,11 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
         const int j = tix % vpr_pad, grp = tix / vpr_pad;
         const bool active = grp < groups;
         const bool data = j < vpr;                        // chunks beyond K are zero padding
-        const int c0 = j << 3;
-        float cs[8], ch[8], k1[8], k2[8], k3[8];
-        bool affine = false, bn = false;
-        int act = ACT_NONE;
-        if (active && data) {
-            const float* scale = BWD ? a.dz.scale : a.x.scale;
-            const float* shift = BWD ? a.dz.shift : a.x.shift;
-            act = BWD ? a.dz.act : a.x.act;
-            affine = scale != nullptr;
-            if (affine) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    cs[q] = __ldg(scale + c0 + q);
-                    ch[q] = __ldg(shift + c0 + q);
-                }
-            }
-            if (BWD && a.dz.k1) {
-                bn = true;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    k1[q] = __ldg(a.dz.k1 + c0 + q);
-                    k2[q] = __ldg(a.dz.k2 + c0 + q);
-                    k3[q] = __ldg(a.dz.k3 + c0 + q);
-                }
-            }
-        }
+        const int c0 = data ? (j << 3) : 0;
+        XfVal xv;
+        XfGrad xg;
+        if (BWD) xg.init(a.dz, c0);
+        else xv.init(a.x, c0);
         int it = 0;
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
@@ -541,25 +576,14 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
                         const int r = sub * RS + rl;
                         uint4 q4 = make_uint4(0, 0, 0, 0);
                         if (data && tile * TM + r < a.P) {
-                            float f[8];
-                            Vec<__nv_bfloat16> v;
-                            v.raw = *reinterpret_cast<const uint4*>(raw + (size_t)rl * row_bytes + (j << 4));
-                            v.unpack(f);
+                            const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)rl * row_bytes + (j << 4));
                             if (!BWD) {
-#pragma unroll
-                                for (int q = 0; q < 8; ++q) f[q] = apply_act(affine ? fmaf(f[q], cs[q], ch[q]) : f[q], act);
+                                q4 = xv.apply(r0);
                             } else if (a.need_z) {
-                                float zz[8];
-                                v.raw = *reinterpret_cast<const uint4*>(raw + (size_t)RS * row_bytes + (size_t)rl * row_bytes + (j << 4));
-                                v.unpack(zz);
-#pragma unroll
-                                for (int q = 0; q < 8; ++q) {
-                                    float pre = affine ? fmaf(zz[q], cs[q], ch[q]) : zz[q];
-                                    float d = f[q] * act_mask(pre, act);
-                                    f[q] = bn ? fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q])) : d;
-                                }
+                                q4 = xg.apply(r0, *reinterpret_cast<const uint4*>(raw + (size_t)(RS + rl) * row_bytes + (j << 4)));
+                            } else {
+                                q4 = r0;
                             }
-                            q4 = pack8(f);
                         }
                         *reinterpret_cast<uint4*>(dstA + tile_off(r, j, TM)) = q4;
                     }
@@ -777,39 +801,17 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
         }
     } else {
         // ---------------------------------------------------------------- transformers, then epilogue
+        // Two uniform passes per stage: every thread first transforms its chunk ja of the dz rows
+        // ga, ga + groupsA, ..., then its chunk jb of the x rows gb, gb + groupsB, ...
         const int tix = tid - 64;
-        const int ca = a.CO >> 3, cb = a.CI >> 3, ct = ca + cb;
-        const int groups = 256 / ct;
-        const int j = tix % ct, grp = tix / ct;
-        const bool active = grp < groups;
-        const bool isA = j < ca;
-        const int jc = isA ? j : j - ca;
-        const int c0 = jc << 3;
-        float cs[8], ch[8], k1[8], k2[8], k3[8];
-        bool affine = false, bn = false;
-        int act = ACT_NONE;
-        if (active) {
-            const float* scale = isA ? a.dz.scale : a.x.scale;
-            const float* shift = isA ? a.dz.shift : a.x.shift;
-            act = isA ? a.dz.act : a.x.act;
-            affine = scale != nullptr;
-            if (affine) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    cs[q] = __ldg(scale + c0 + q);
-                    ch[q] = __ldg(shift + c0 + q);
-                }
-            }
-            if (isA && a.dz.k1) {
-                bn = true;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    k1[q] = __ldg(a.dz.k1 + c0 + q);
-                    k2[q] = __ldg(a.dz.k2 + c0 + q);
-                    k3[q] = __ldg(a.dz.k3 + c0 + q);
-                }
-            }
-        }
+        const int ca = a.CO >> 3, cb = a.CI >> 3;
+        const int groupsA = 256 / ca, groupsB = 256 / cb;
+        const int ja = tix % ca, ga = tix / ca, jb = tix % cb, gb = tix / cb;
+        const int rowsA = ga < groupsA ? WSTAGE : 0, rowsB = gb < groupsB ? WSTAGE : 0;
+        XfGrad xg;
+        XfVal xv;
+        xg.init(a.dz, ja << 3);
+        xv.init(a.x, jb << 3);
         bool ok = true;
         for (int it = 0; it < stages; ++it) {
             const int st = it & 1, n = it >> 1, s = it % R;
@@ -822,39 +824,22 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
                 break;
             }
             const uint8_t* raw = sR + (size_t)s * a.raw_bytes;
-            uint8_t* dst = sOp + (size_t)st * a.op_bytes + (isA ? 0u : (uint32_t)a.pa * PANEL) + (uint32_t)(jc >> 3) * PANEL;
+            uint8_t* dstA = sOp + (size_t)st * a.op_bytes + (uint32_t)(ja >> 3) * PANEL;
+            uint8_t* dstB = sOp + (size_t)st * a.op_bytes + (uint32_t)(a.pa + (jb >> 3)) * PANEL;
             const int valid = min(WSTAGE, pend - (pbeg + it * WSTAGE));
-            if (active) {
-#pragma unroll 4
-                for (int kr = grp; kr < WSTAGE; kr += groups) {
-                    uint4 q4 = make_uint4(0, 0, 0, 0);
-                    if (kr < valid) {
-                        float f[8];
-                        Vec<__nv_bfloat16> v;
-                        if (isA) {
-                            v.raw = *reinterpret_cast<const uint4*>(raw + (size_t)kr * rowA + (jc << 4));
-                            v.unpack(f);
-                            if (a.need_z) {
-                                float zz[8];
-                                v.raw = *reinterpret_cast<const uint4*>(raw + offZ + (size_t)kr * rowA + (jc << 4));
-                                v.unpack(zz);
-#pragma unroll
-                                for (int q = 0; q < 8; ++q) {
-                                    float pre = affine ? fmaf(zz[q], cs[q], ch[q]) : zz[q];
-                                    float d = f[q] * act_mask(pre, act);
-                                    f[q] = bn ? fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q])) : d;
-                                }
-                            }
-                        } else {
-                            v.raw = *reinterpret_cast<const uint4*>(raw + offX + (size_t)kr * rowB + (jc << 4));
-                            v.unpack(f);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) f[q] = apply_act(affine ? fmaf(f[q], cs[q], ch[q]) : f[q], act);
-                        }
-                        q4 = pack8(f);
-                    }
-                    *reinterpret_cast<uint4*>(dst + kr * 128 + (((jc & 7) ^ (kr & 7)) << 4)) = q4;
+#pragma unroll 2
+            for (int kr = ga; kr < rowsA; kr += groupsA) {
+                uint4 q4 = make_uint4(0, 0, 0, 0);
+                if (kr < valid) {
+                    const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)kr * rowA + (ja << 4));
+                    q4 = a.need_z ? xg.apply(r0, *reinterpret_cast<const uint4*>(raw + offZ + (size_t)kr * rowA + (ja << 4))) : r0;
                 }
+                *reinterpret_cast<uint4*>(dstA + kr * 128 + (((ja & 7) ^ (kr & 7)) << 4)) = q4;
+            }
+            for (int kr = gb; kr < rowsB; kr += groupsB) {
+                uint4 q4 = make_uint4(0, 0, 0, 0);
+                if (kr < valid) q4 = xv.apply(*reinterpret_cast<const uint4*>(raw + offX + (size_t)kr * rowB + (jb << 4)));
+                *reinterpret_cast<uint4*>(dstB + kr * 128 + (((jb & 7) ^ (kr & 7)) << 4)) = q4;
             }
             mbar_arrive(raw_empty(s));
             fence_async_smem();
