@@ -45,66 +45,35 @@ template <int V> __device__ __forceinline__ void ld_coef(const float* p, int c0,
     }
 }
 
-// Reads a forward value: act(raw*scale + shift) with the coefficients held in registers.
+// Reads a forward value: act(raw*scale + shift) with the coefficients held in registers; the
+// activation is a pair of bounds and a missing BatchNorm the identity map, so the transform is
+// the same instruction stream for every layer configuration.
 template <typename T, int V> struct ValLoader {
     const void* p;
-    float scale[V], shift[V];
-    bool affine;
-    int act;
-    __device__ __forceinline__ ValLoader(const ValSrc& s, int c0) : p(s.p), affine(s.scale != nullptr), act(s.act) {
-        if (affine) {
+    float scale[V], shift[V], lo, hi;
+    __device__ __forceinline__ ValLoader(const ValSrc& s, int c0) : p(s.p) {
+        if (s.scale) {
             ld_coef<V>(s.scale, c0, scale);
             ld_coef<V>(s.shift, c0, shift);
+        } else {
+#pragma unroll
+            for (int q = 0; q < V; ++q) {
+                scale[q] = 1.f;
+                shift[q] = 0.f;
+            }
         }
+        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
+        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
     }
     __device__ __forceinline__ void load(size_t e, float* f) const {
         Raw<T, V>::ld(p, e, f);
-        if (affine) {
 #pragma unroll
-            for (int q = 0; q < V; ++q) f[q] = fmaf(f[q], scale[q], shift[q]);
-        }
-        if (act != ACT_NONE) {
-#pragma unroll
-            for (int q = 0; q < V; ++q) f[q] = apply_act(f[q], act);
-        }
-    }
-};
-
-// Reads dz = k1*(dy*mask(pre)) + k2 + k3*z with the coefficients held in registers.
-template <typename T, int V> struct GradLoader {
-    const void* dy;
-    const void* z;
-    float scale[V], shift[V], k1[V], k2[V], k3[V];
-    bool affine, bn, need_z;
-    int act;
-    __device__ __forceinline__ GradLoader(const GradSrc& s, int c0)
-        : dy(s.dy), z(s.z), affine(s.scale != nullptr), bn(s.k1 != nullptr), need_z(s.act != ACT_NONE || s.k1 != nullptr), act(s.act) {
-        if (affine) {
-            ld_coef<V>(s.scale, c0, scale);
-            ld_coef<V>(s.shift, c0, shift);
-        }
-        if (bn) {
-            ld_coef<V>(s.k1, c0, k1);
-            ld_coef<V>(s.k2, c0, k2);
-            ld_coef<V>(s.k3, c0, k3);
-        }
-    }
-    __device__ __forceinline__ void load(size_t e, float* f) const {
-        Raw<T, V>::ld(dy, e, f);
-        if (!need_z) return;
-        float zz[V];
-        Raw<T, V>::ld(z, e, zz);
-#pragma unroll
-        for (int q = 0; q < V; ++q) {
-            float pre = affine ? fmaf(zz[q], scale[q], shift[q]) : zz[q];
-            float d = f[q] * act_mask(pre, act);
-            f[q] = bn ? fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q])) : d;
-        }
+        for (int q = 0; q < V; ++q) f[q] = fminf(fmaxf(fmaf(f[q], scale[q], shift[q]), lo), hi);
     }
 };
 
 // out[n,ho,wo,c] = sum_{r,s} in[n, ho*S-1+r, wo*S-1+s, c] * w[(FLIP ? 8-(3r+s) : 3r+s)][c]  (+ addend)
-// Forward: in = x (ValLoader), S = stride.  Backward-data at stride 1: in = dz (GradLoader), FLIP.
+// Forward: in = x (ValLoader), S = stride.  
 template <typename T, int V, int S, bool FLIP, typename LOADER, typename SRC>
 __global__ void __launch_bounds__(128) dw_strip_kernel(int n_img, int hi, int wi, int ho, int wo, int c, SRC src, const float* __restrict__ w9c,
                                                        const T* addend, T* out) {
@@ -190,26 +159,34 @@ __device__ __forceinline__ void raw_decode(const uint2& v, float* f) {
 }
 
 // Split-phase loaders: fetch() only issues the global loads, decode() applies the transform.
+// The transforms are branch-free: absent BatchNorm terms take neutral coefficients (scale 1,
+// shift 0, k1 1, k2 = k3 0) and the activation is a pair of bounds (ReLU6 0..6, ReLU 0..inf,
+// none -inf..inf), so no per-element decision depends on the layer's configuration.
 template <typename T, int V> struct ValRoll {
     typedef typename RawT<T, V>::type raw_t;
     struct Raw1 { raw_t a; };
     const void* p;
-    float scale[V], shift[V];
-    bool affine;
-    int act;
-    __device__ __forceinline__ ValRoll(const ValSrc& s, int c0) : p(s.p), affine(s.scale != nullptr), act(s.act) {
-        if (affine) {
+    float scale[V], shift[V], lo, hi;
+    __device__ __forceinline__ ValRoll(const ValSrc& s, int c0) : p(s.p) {
+        if (s.scale) {
             ld_coef<V>(s.scale, c0, scale);
             ld_coef<V>(s.shift, c0, shift);
+        } else {
+#pragma unroll
+            for (int q = 0; q < V; ++q) {
+                scale[q] = 1.f;
+                shift[q] = 0.f;
+            }
         }
+        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
+        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
     }
     __device__ __forceinline__ Raw1 fetch(size_t e) const { return Raw1{raw_fetch<T, V>(p, e)}; }
     __device__ __forceinline__ void decode(const Raw1& r, bool ok, float* f) const {
         raw_decode(r.a, f);
 #pragma unroll
         for (int q = 0; q < V; ++q) {
-            float v = affine ? fmaf(f[q], scale[q], shift[q]) : f[q];
-            v = apply_act(v, act);
+            const float v = fminf(fmaxf(fmaf(f[q], scale[q], shift[q]), lo), hi);
             f[q] = ok ? v : 0.f;
         }
     }
@@ -219,20 +196,28 @@ template <typename T, int V> struct GradRoll {
     struct Raw1 { raw_t a, b; };
     const void* dy;
     const void* z;
-    float scale[V], shift[V], k1[V], k2[V], k3[V];
-    bool affine, bn, need_z;
-    int act;
-    __device__ __forceinline__ GradRoll(const GradSrc& s, int c0)
-        : dy(s.dy), z(s.z), affine(s.scale != nullptr), bn(s.k1 != nullptr), need_z(s.act != ACT_NONE || s.k1 != nullptr), act(s.act) {
-        if (affine) {
+    float scale[V], shift[V], k1[V], k2[V], k3[V], lo, hi;
+    bool need_z;
+    __device__ __forceinline__ GradRoll(const GradSrc& s, int c0) : dy(s.dy), z(s.z), need_z(s.act != ACT_NONE || s.k1 != nullptr) {
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            scale[q] = 1.f;
+            shift[q] = 0.f;
+            k1[q] = 1.f;
+            k2[q] = 0.f;
+            k3[q] = 0.f;
+        }
+        if (s.scale) {
             ld_coef<V>(s.scale, c0, scale);
             ld_coef<V>(s.shift, c0, shift);
         }
-        if (bn) {
+        if (s.k1) {
             ld_coef<V>(s.k1, c0, k1);
             ld_coef<V>(s.k2, c0, k2);
             ld_coef<V>(s.k3, c0, k3);
         }
+        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
+        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
     }
     __device__ __forceinline__ Raw1 fetch(size_t e) const {
         Raw1 r;
@@ -240,18 +225,16 @@ template <typename T, int V> struct GradRoll {
         r.b = need_z ? raw_fetch<T, V>(z, e) : r.a;
         return r;
     }
+    // without z (no activation, no BatchNorm) b == a: pre = dy lies inside (-inf, inf) and the result is dy
     __device__ __forceinline__ void decode(const Raw1& r, bool ok, float* f) const {
         float zz[V];
         raw_decode(r.a, f);
         raw_decode(r.b, zz);
 #pragma unroll
         for (int q = 0; q < V; ++q) {
-            float d = f[q];
-            if (need_z) {
-                float pre = affine ? fmaf(zz[q], scale[q], shift[q]) : zz[q];
-                d *= act_mask(pre, act);
-                if (bn) d = fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q]));
-            }
+            const float pre = fmaf(zz[q], scale[q], shift[q]);
+            float d = (pre > lo && pre < hi) ? f[q] : 0.f;
+            d = fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q]));
             f[q] = ok ? d : 0.f;
         }
     }
@@ -364,16 +347,31 @@ void launch_roll(int n, int h, int w, int c, const SRC& src, const float* w9c, c
 }
 
 
+// Per-thread asynchronous prefetch ring.  A thread copies its own future vectors global -> shared
+// with cp.async (one commit group per step) and later reads back only what it copied itself, so
+// no barrier is involved: the bytes in flight no longer cost registers and a thread can run
+// several rows ahead of its arithmetic.  Slot (stage, load l) of thread t sits at
+// ((stage * NL + l) * 128 + t) vectors: consecutive threads are consecutive in shared memory.
+template <typename RAW> __device__ __forceinline__ void cp_async_vec(RAW* dst_smem, const void* src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst_smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2;" ::"r"(d), "l"(src), "n"((int)sizeof(RAW)) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // Rolling weight gradient for stride 1: gw[c][r][s] = sum dz[oh][wo] * x[oh-1+r][wo-1+s].
 // A thread owns V channels; a work item is a strip TWR wide and `th` rows high.  Walking down the
 // input rows ih, it holds dz rows ih-1, ih, ih+1 (zero outside the item's rows) and the x row ih:
 // tap row r pairs x row ih with dz row ih+1-r.  Each row of either tensor is loaded and decoded
-// once per item; the next rows' loads are issued before the current row's arithmetic.
-template <typename T, int V, int TWR>
+// once per item; the loads of the next D rows are in flight in the thread's prefetch ring.
+template <typename T, int V, int TWR, int D>
 __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, int cw, int rows, int th, size_t items_per_block,
                                                             float* __restrict__ partial) {
-    constexpr int NIN = TWR + 2;
-    extern __shared__ float red[];
+    constexpr int NIN = TWR + 2, NL = NIN + 2 * TWR;
+    typedef typename RawT<T, V>::type raw_t;
+    extern __shared__ __align__(16) uint8_t dsm[];
+    raw_t* ring = reinterpret_cast<raw_t*>(dsm) + threadIdx.x;       // + (stage * NL + l) * 128
+    float* red = reinterpret_cast<float*>(dsm);                      // reused after the main loop
     const int cv = g.ci / V;
     const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
     const int j = blockIdx.x * cw + jl;
@@ -393,6 +391,9 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
         ValRoll<T, V> ldx(xs, c0);
         typedef typename GradRoll<T, V>::Raw1 RawZ;
         typedef typename ValRoll<T, V>::Raw1 RawX;
+        const T* px = reinterpret_cast<const T*>(xs.p);
+        const T* pdy = reinterpret_cast<const T*>(dzs.dy);
+        const T* pz = reinterpret_cast<const T*>(dzs.z);
         for (size_t item = ibeg + row; item < iend; item += rows) {
             const int wo0 = (int)(item % sw) * TWR;
             size_t t2 = item / sw;
@@ -411,35 +412,51 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
                 zok[t] = wo0 + t < w;
                 zcol[t] = min(wo0 + t, w - 1) * c + c0;
             }
+            // step `ih` consumes x row ih and dz row ih+1 (row addresses clamped into the image)
+            auto issue = [&](int ih, int stage) {
+                if (ih <= oh1) {
+                    const size_t rbx = ((size_t)n * h + min(max(ih, 0), h - 1)) * w * c, rbz = ((size_t)n * h + min(max(ih + 1, 0), h - 1)) * w * c;
+                    raw_t* slot = ring + (size_t)stage * NL * 128;
+#pragma unroll
+                    for (int q2 = 0; q2 < NIN; ++q2) cp_async_vec(slot + q2 * 128, px + rbx + xcol[q2]);
+#pragma unroll
+                    for (int t = 0; t < TWR; ++t) cp_async_vec(slot + (NIN + t) * 128, pdy + rbz + zcol[t]);
+                    if (ldz.need_z) {
+#pragma unroll
+                        for (int t = 0; t < TWR; ++t) cp_async_vec(slot + (NIN + TWR + t) * 128, pz + rbz + zcol[t]);
+                    }
+                }
+                cp_async_commit();
+            };
             float dzm[TWR][V], dz0[TWR][V], dzp[TWR][V];
 #pragma unroll
             for (int t = 0; t < TWR; ++t)
 #pragma unroll
                 for (int q = 0; q < V; ++q) dzm[t][q] = dz0[t][q] = 0.f;
-            RawX nx[NIN];
-            RawZ nz[TWR];
-            {   // first x row (oh0-1, clamped) and first dz row (oh0)
-                const size_t rbx = ((size_t)n * h + max(oh0 - 1, 0)) * w * c, rbz = ((size_t)n * h + oh0) * w * c;
 #pragma unroll
-                for (int q2 = 0; q2 < NIN; ++q2) nx[q2] = ldx.fetch(rbx + xcol[q2]);
-#pragma unroll
-                for (int t = 0; t < TWR; ++t) nz[t] = ldz.fetch(rbz + zcol[t]);
-            }
+            for (int d = 0; d < D; ++d) issue(oh0 - 1 + d, d);
+            int stage = 0;
             for (int ih = oh0 - 1; ih <= oh1; ++ih) {
+                cp_async_wait<D - 1>();
+                const raw_t* slot = ring + (size_t)stage * NL * 128;
                 const bool xrow_ok = ih >= 0 && ih < h;
                 const bool zrow_ok = ih + 1 >= oh0 && ih + 1 < oh1;
                 float xin[NIN][V];
 #pragma unroll
-                for (int q2 = 0; q2 < NIN; ++q2) ldx.decode(nx[q2], xrow_ok && xok[q2], xin[q2]);
-#pragma unroll
-                for (int t = 0; t < TWR; ++t) ldz.decode(nz[t], zrow_ok && zok[t], dzp[t]);
-                if (ih < oh1) {     // next rows: x row ih+1, dz row ih+2 (addresses clamped into the image)
-                    const size_t rbx = ((size_t)n * h + min(ih + 1, h - 1)) * w * c, rbz = ((size_t)n * h + min(ih + 2, h - 1)) * w * c;
-#pragma unroll
-                    for (int q2 = 0; q2 < NIN; ++q2) nx[q2] = ldx.fetch(rbx + xcol[q2]);
-#pragma unroll
-                    for (int t = 0; t < TWR; ++t) nz[t] = ldz.fetch(rbz + zcol[t]);
+                for (int q2 = 0; q2 < NIN; ++q2) {
+                    RawX r;
+                    r.a = slot[q2 * 128];
+                    ldx.decode(r, xrow_ok && xok[q2], xin[q2]);
                 }
+#pragma unroll
+                for (int t = 0; t < TWR; ++t) {
+                    RawZ r;
+                    r.a = slot[(NIN + t) * 128];
+                    r.b = ldz.need_z ? slot[(NIN + TWR + t) * 128] : r.a;
+                    ldz.decode(r, zrow_ok && zok[t], dzp[t]);
+                }
+                issue(ih + D, stage);              // refill the stage just read
+                stage = stage + 1 == D ? 0 : stage + 1;
 #pragma unroll
                 for (int s = 0; s < 3; ++s)
 #pragma unroll
@@ -461,7 +478,183 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
             }
         }
     }
+    cp_async_wait<0>();
+    __syncthreads();                               // the ring is now free: reuse it for the block sum
     const int width = cw * V;
+    for (int t = 0; t < 9; ++t) {
+        if (row < rows) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) red[row * width + jl * V + q] = acc[t][q];
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < width; e += blockDim.x) {
+            int ch = blockIdx.x * width + e;
+            if (ch < g.ci) {
+                float s = 0.f;
+                for (int r2 = 0; r2 < rows; ++r2) s += red[r2 * width + e];
+                partial[((size_t)blockIdx.y * 9 + t) * g.ci + ch] = s;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+
+// Fused backward of a stride-1 depthwise layer: one pass over dy, z and x produces both the input
+// gradient and the weight-gradient partials, so the BatchNorm-backward transform of dz is
+// evaluated once instead of once per kernel.  A work item is a strip TWR wide over a whole image
+// column; a thread owns V channels of it and walks down the rows ih holding dz rows ih-1, ih, ih+1
+// (TWR + 2 columns: the strip and one halo column each side) and x row ih:
+//   dx[ih][wo0+t]  = sum_{r,s} dz[ih+1-r][wo0+t+1-s] * w[r][s]
+//   gw[r][s]      += sum_t dz[ih+1-r][wo0+t] * x[ih][wo0+t-1+s]
+// The halo columns of dz feed dx only; their weight-gradient terms belong to the neighbouring strip.
+template <typename T, int V, int TWR, int D>
+__global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, const float* __restrict__ w9c, const T* addend,
+                                                           T* dx, int cw, int rows, size_t items_per_block, float* __restrict__ partial) {
+    constexpr int NIN = TWR + 2, NL = 3 * NIN;
+    typedef typename RawT<T, V>::type raw_t;
+    extern __shared__ __align__(16) uint8_t dsm[];
+    const int width = cw * V;
+    float* wsm = reinterpret_cast<float*>(dsm);                                       // [9][width]
+    raw_t* ring = reinterpret_cast<raw_t*>(dsm + (((size_t)9 * width * 4 + 15) & ~(size_t)15)) + threadIdx.x;
+    float* red = reinterpret_cast<float*>(ring - threadIdx.x);                        // reused after the main loop
+    const int cv = g.ci / V;
+    const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
+    const int j = blockIdx.x * cw + jl;
+    const bool active = row < rows && j < cv;
+    const int c0 = active ? j * V : 0;
+    const int h = g.hi, w = g.wi, c = g.ci;
+    for (int i = threadIdx.x; i < 9 * width; i += blockDim.x) {
+        const int t = i / width, ch = blockIdx.x * width + (i - t * width);
+        wsm[i] = ch < c ? __ldg(w9c + t * c + ch) : 0.f;
+    }
+    __syncthreads();
+    const int sw = (w + TWR - 1) / TWR;
+    const size_t n_items = (size_t)g.n * sw;
+    const size_t ibeg = (size_t)blockIdx.y * items_per_block, iend = min(n_items, ibeg + items_per_block);
+    float acc[9][V];
+#pragma unroll
+    for (int t = 0; t < 9; ++t)
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[t][q] = 0.f;
+    if (active) {
+        GradRoll<T, V> ldz(dzs, c0);
+        ValRoll<T, V> ldx(xs, c0);
+        typedef typename GradRoll<T, V>::Raw1 RawZ;
+        typedef typename ValRoll<T, V>::Raw1 RawX;
+        const T* px = reinterpret_cast<const T*>(xs.p);
+        const T* pdy = reinterpret_cast<const T*>(dzs.dy);
+        const T* pz = reinterpret_cast<const T*>(dzs.z);
+        const float* wl = wsm + jl * V;
+        for (size_t item = ibeg + row; item < iend; item += rows) {
+            const int wo0 = (int)(item % sw) * TWR, n = (int)(item / sw);
+            int col[NIN];
+            bool cok[NIN];
+#pragma unroll
+            for (int q2 = 0; q2 < NIN; ++q2) {
+                const int wi = wo0 - 1 + q2;
+                cok[q2] = wi >= 0 && wi < w;
+                col[q2] = min(max(wi, 0), w - 1) * c + c0;
+            }
+            // step ih consumes x row ih and dz row ih+1 (row addresses clamped into the image)
+            auto issue = [&](int ih, int stage) {
+                if (ih < h) {
+                    const size_t rbx = ((size_t)n * h + max(ih, 0)) * w * c, rbz = ((size_t)n * h + min(ih + 1, h - 1)) * w * c;
+                    raw_t* slot = ring + (size_t)stage * NL * 128;
+#pragma unroll
+                    for (int q2 = 0; q2 < NIN; ++q2) cp_async_vec(slot + q2 * 128, px + rbx + col[q2]);
+#pragma unroll
+                    for (int q2 = 0; q2 < NIN; ++q2) cp_async_vec(slot + (NIN + q2) * 128, pdy + rbz + col[q2]);
+                    if (ldz.need_z) {
+#pragma unroll
+                        for (int q2 = 0; q2 < NIN; ++q2) cp_async_vec(slot + (2 * NIN + q2) * 128, pz + rbz + col[q2]);
+                    }
+                }
+                cp_async_commit();
+            };
+            float dzm[NIN][V], dz0[NIN][V], dzp[NIN][V];
+#pragma unroll
+            for (int q2 = 0; q2 < NIN; ++q2)
+#pragma unroll
+                for (int q = 0; q < V; ++q) dzm[q2][q] = dz0[q2][q] = 0.f;
+#pragma unroll
+            for (int d = 0; d < D; ++d) issue(-1 + d, d);
+            int stage = 0;
+            for (int ih = -1; ih < h; ++ih) {
+                cp_async_wait<D - 1>();
+                const raw_t* slot = ring + (size_t)stage * NL * 128;
+                const bool xrow_ok = ih >= 0, zrow_ok = ih + 1 < h;
+                float xin[NIN][V];
+#pragma unroll
+                for (int q2 = 0; q2 < NIN; ++q2) {
+                    RawX r;
+                    r.a = slot[q2 * 128];
+                    ldx.decode(r, xrow_ok && cok[q2], xin[q2]);
+                }
+#pragma unroll
+                for (int q2 = 0; q2 < NIN; ++q2) {
+                    RawZ r;
+                    r.a = slot[(NIN + q2) * 128];
+                    r.b = ldz.need_z ? slot[(2 * NIN + q2) * 128] : r.a;
+                    ldz.decode(r, zrow_ok && cok[q2], dzp[q2]);
+                }
+                issue(ih + D, stage);              // refill the stage just read
+                stage = stage + 1 == D ? 0 : stage + 1;
+                float ad[TWR][V];
+                const size_t orow = (((size_t)n * h + max(ih, 0)) * w + wo0) * c + c0;
+                if (addend && ih >= 0) {
+#pragma unroll
+                    for (int t = 0; t < TWR; ++t)
+                        if (wo0 + t < w) Raw<T, V>::ld(addend, orow + (size_t)t * c, ad[t]);
+                }
+                float o[TWR][V];
+#pragma unroll
+                for (int t = 0; t < TWR; ++t)
+#pragma unroll
+                    for (int q = 0; q < V; ++q) o[t][q] = 0.f;
+#pragma unroll
+                for (int s = 0; s < 3; ++s) {
+                    float w0[V], w1[V], w2[V];
+                    *reinterpret_cast<float4*>(w0) = *reinterpret_cast<const float4*>(wl + (0 * 3 + s) * width);
+                    *reinterpret_cast<float4*>(w1) = *reinterpret_cast<const float4*>(wl + (1 * 3 + s) * width);
+                    *reinterpret_cast<float4*>(w2) = *reinterpret_cast<const float4*>(wl + (2 * 3 + s) * width);
+#pragma unroll
+                    for (int t = 0; t < TWR; ++t)
+#pragma unroll
+                        for (int q = 0; q < V; ++q) {
+                            o[t][q] = fmaf(dzp[t + 2 - s][q], w0[q], o[t][q]);
+                            o[t][q] = fmaf(dz0[t + 2 - s][q], w1[q], o[t][q]);
+                            o[t][q] = fmaf(dzm[t + 2 - s][q], w2[q], o[t][q]);
+                            const float xv = xin[t + s][q];
+                            acc[0 * 3 + s][q] = fmaf(dzp[t + 1][q], xv, acc[0 * 3 + s][q]);
+                            acc[1 * 3 + s][q] = fmaf(dz0[t + 1][q], xv, acc[1 * 3 + s][q]);
+                            acc[2 * 3 + s][q] = fmaf(dzm[t + 1][q], xv, acc[2 * 3 + s][q]);
+                        }
+                }
+                if (ih >= 0) {
+#pragma unroll
+                    for (int t = 0; t < TWR; ++t) {
+                        if (wo0 + t < w) {
+                            if (addend) {
+#pragma unroll
+                                for (int q = 0; q < V; ++q) o[t][q] += ad[t][q];
+                            }
+                            Raw<T, V>::st(dx, orow + (size_t)t * c, o[t]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int q2 = 0; q2 < NIN; ++q2)
+#pragma unroll
+                    for (int q = 0; q < V; ++q) {
+                        dzm[q2][q] = dz0[q2][q];
+                        dz0[q2][q] = dzp[q2][q];
+                    }
+            }
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();                               // the ring is now free: reuse it for the block sum
     for (int t = 0; t < 9; ++t) {
         if (row < rows) {
 #pragma unroll
@@ -767,41 +960,98 @@ void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w
 
 void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw,
                    cudaStream_t st) {
-    {
-        constexpr int TWR = 2;
-        const int V = 4;
-        const int cv = g.ci / V;
-        const int parts = (cv + 47) / 48;              // channel-vector columns per block: an even split, at most 48
-        int cw = (cv + parts - 1) / parts;
-        int rows = 128 / cw;
-        const int th = g.ho >= 28 ? 8 : (g.ho >= 14 ? 7 : g.ho);      // rows of dz per work item
-        const int sw = (g.wo + TWR - 1) / TWR, nrc = (g.ho + th - 1) / th;
-        size_t n_items = (size_t)g.n * nrc * sw;
-        int gx = (cv + cw - 1) / cw;
-        size_t by = (8 * 148 + gx - 1) / gx;
-        size_t max_by = (n_items + (size_t)rows - 1) / (size_t)rows;
-        if (by > max_by) by = max_by;
-        size_t cap = scratch_floats / ((size_t)9 * g.ci);
+    constexpr int TWR = 2;
+    const int V = 4;
+    const int cv = g.ci / V;
+    const int parts = (cv + 47) / 48;              // channel-vector columns per block: an even split, at most 48
+    const int cw = (cv + parts - 1) / parts;
+    const int rows = 128 / cw;
+    const int gx = (cv + cw - 1) / cw;
+    const int sw = (g.wo + TWR - 1) / TWR;
+    const size_t cap = scratch_floats / ((size_t)9 * g.ci);
+    double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
+    size_t by;
+    if (g.stride == 1) {
+        // Long items (whole image columns when the batch gives enough of them) keep the prefetch
+        // ring full; all blocks are resident at once, so there is no partial last wave.
+        const size_t resident = 3 * 148;
+        int th = g.ho;
+        while (th > 7 && (size_t)g.n * ((g.ho + th - 1) / th) * sw * gx < (size_t)rows * 2 * 148) th = (th + 1) / 2;
+        const size_t n_items = (size_t)g.n * ((g.ho + th - 1) / th) * sw;
+        by = (n_items + rows - 1) / rows;
+        if (by * gx > resident) by = resident / gx;
         if (by > cap) by = cap;
         if (by < 1) by = 1;
-        size_t ipb = (n_items + by - 1) / by;
+        const size_t ipb = (n_items + by - 1) / by;
         by = (n_items + ipb - 1) / ipb;
-        size_t smem = (size_t)rows * cw * V * sizeof(float);
         dim3 grid(gx, (unsigned)by);
-        double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
-        {
-            LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
-            if (g.stride == 1) {
-                if (dtype == 0) dw_wgrad_roll_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
-                else dw_wgrad_roll_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
-            } else {
-                if (dtype == 0) dw_wgrad_s2_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
-                else dw_wgrad_s2_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
-            }
+        LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
+        constexpr int NL = TWR + 2 + 2 * TWR;
+        if (dtype == 0) {
+            constexpr int D = 2;
+            dw_wgrad_roll_kernel<float, 4, TWR, D><<<grid, 128, (size_t)D * NL * 128 * 16, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+        } else {
+            constexpr int D = 4;
+            dw_wgrad_roll_kernel<__nv_bfloat16, 4, TWR, D><<<grid, 128, (size_t)D * NL * 128 * 8, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
         }
-        LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
-        dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
+    } else {
+        const int th = g.ho >= 28 ? 8 : (g.ho >= 14 ? 7 : g.ho);      // rows of dz per work item
+        const int nrc = (g.ho + th - 1) / th;
+        const size_t n_items = (size_t)g.n * nrc * sw;
+        by = (8 * 148 + gx - 1) / gx;
+        const size_t max_by = (n_items + (size_t)rows - 1) / (size_t)rows;
+        if (by > max_by) by = max_by;
+        if (by > cap) by = cap;
+        if (by < 1) by = 1;
+        const size_t ipb = (n_items + by - 1) / by;
+        by = (n_items + ipb - 1) / ipb;
+        const size_t smem = (size_t)rows * cw * V * sizeof(float);
+        dim3 grid(gx, (unsigned)by);
+        LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
+        if (dtype == 0) dw_wgrad_s2_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+        else dw_wgrad_s2_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
     }
+    LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
+    dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
+}
+
+bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, const float* w9c, const void* addend, void* dx,
+                  float* scratch, size_t scratch_floats, float* gw, cudaStream_t st) {
+    constexpr int TWR = 2, V = 4, D = 4, NL = 3 * (TWR + 2);
+    if (dtype != 1 || g.stride != 1 || g.ci % V) return false;
+    const int cv = g.ci / V;
+    const int parts = (cv + 47) / 48;
+    const int cw = (cv + parts - 1) / parts;
+    const int rows = 128 / cw;
+    const int gx = (cv + cw - 1) / cw;
+    const int sw = (g.wo + TWR - 1) / TWR;
+    const size_t n_items = (size_t)g.n * sw;
+    // whole image columns per thread: worth it only when that still gives every SM a few warps
+    if (n_items * gx < (size_t)rows * 2 * 148) return false;
+    const size_t cap = scratch_floats / ((size_t)9 * g.ci);
+    const size_t resident = 3 * 148;              // three blocks per SM: all blocks run at once, no partial last wave
+    size_t by = (n_items + rows - 1) / rows;
+    if (by * gx > resident) by = resident / gx;
+    if (by > cap) by = cap;
+    if (by < 1) return false;
+    const size_t ipb = (n_items + by - 1) / by;
+    by = (n_items + ipb - 1) / ipb;
+    const size_t smem = (((size_t)9 * cw * V * 4 + 15) & ~(size_t)15) + (size_t)D * NL * 128 * 8;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        attr_set = true;
+    }
+    double e = (double)g.n * g.hi * g.wi * g.ci;
+    {
+        LaunchScope ls(K_DW_BWD_FUSED, grad_src_bytes(dz, e, dtype) + e * 2.0 * (addend ? 3.0 : 2.0) + 36.0 * g.ci * (by + 1), 36.0 * e, st);
+        dim3 grid(gx, (unsigned)by);
+        dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D><<<grid, 128, smem, st>>>(g, dz, x, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx, cw,
+                                                                            rows, ipb, scratch);
+    }
+    LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
+    dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
+    return true;
 }
 
 }  // namespace ast

@@ -16,7 +16,7 @@ struct ConvGeom {
 enum KernelKind {
     K_CONV_FWD = 0, K_CONV_BWD_DATA, K_CONV_BWD_WEIGHT, K_REDUCE_SPLITS, K_DW_FWD, K_DW_BWD_DATA, K_DW_BWD_WEIGHT,
     K_DW_BWD_WEIGHT_FINISH, K_BN_STATS, K_BN_STATS_FINISH, K_BN_BWD_REDUCE, K_BN_BWD_FINISH, K_EW_ADD, K_EW_MASK, K_EW_SUM,
-    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_CONV3_BWD_WEIGHT_TC, K_KINDS
+    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_CONV3_BWD_WEIGHT_TC, K_DW_BWD_FUSED, K_KINDS
 };
 const char* kernel_name(int kind);
 
@@ -63,6 +63,9 @@ void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, 
 // ---- depthwise 3x3 (weights tap-major: w9c[r*3+s][c]) ----
 void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, cudaStream_t st);
 void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w9c, const void* addend, void* dx, cudaStream_t st);
+// stride-1 bf16 layers with enough image columns: input gradient and weight gradient in one pass; false = not applicable
+bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, const float* w9c, const void* addend, void* dx,
+                  float* scratch, size_t scratch_floats, float* gw, cudaStream_t st);
 // gw[c][r][s]
 void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats,
                    float* gw, cudaStream_t st);

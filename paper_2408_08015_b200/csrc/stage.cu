@@ -440,6 +440,16 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             }
             tick(s, ui, 4, st);
             ValSrc xin = val_src(s, sv, u.in);
+            if (u.kind == U_DW && want_in) {
+                GradState& gi = gs[u.in];
+                const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
+                if (dw_bwd_fused(dt, u.g, d, xin, s->derived + u.w_off, addend, own(u.in), s->scratch, s->scratch_floats, s->g + u.w_off, st)) {
+                    gi.state = G_OWNED;
+                    gi.ptr = own(u.in);
+                    tick(s, ui, 5, st);
+                    continue;
+                }
+            }
             if (u.kind == U_CONV && pw_tc_supported(dt, u.g, false))
                 pw_bwd_weight_tc(u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, s->err, st);
             else if (u.kind == U_CONV && conv3_wgrad_tc_supported(dt, u.g))
