@@ -65,6 +65,8 @@ struct BwdOp {
 template <typename T, int V, typename OP>
 __global__ void __launch_bounds__(256) chan_reduce_kernel(OP op, size_t pixels, int c, int cw, int rows, size_t pix_per_block,
                                                           float* __restrict__ partial) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ float red[];
     const int cg = c / V;
     const int jl = threadIdx.x % cw, row = threadIdx.x / cw;
@@ -134,11 +136,11 @@ void launch_reduce(int dtype, const ReducePlan& p, const OP& op, size_t pixels, 
     LaunchScope ls(kind, bytes + 8.0 * c * p.by, 4.0 * pixels * c, st);
     dim3 grid(p.gx, (unsigned)p.by);
     if (dtype == 0) {
-        if (p.V == 1) chan_reduce_kernel<float, 1, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
-        else chan_reduce_kernel<float, 4, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        if (p.V == 1) launch_pdl(chan_reduce_kernel<float, 1, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        else launch_pdl(chan_reduce_kernel<float, 4, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
     } else {
-        if (p.V == 1) chan_reduce_kernel<__nv_bfloat16, 1, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
-        else chan_reduce_kernel<__nv_bfloat16, 8, OP><<<grid, 256, p.smem, st>>>(op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        if (p.V == 1) launch_pdl(chan_reduce_kernel<__nv_bfloat16, 1, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        else launch_pdl(chan_reduce_kernel<__nv_bfloat16, 8, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
     }
 }
 
@@ -187,6 +189,8 @@ template <typename T>
 __global__ void __launch_bounds__(1024) bn_stats_finish(const float* __restrict__ partial, int blocks, int c, const T* __restrict__ z, double count,
                                                        const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float momentum,
                                                        BnFwdOut o) {
+    pdl_wait();
+    pdl_launch();
     // the owner thread's per-channel inputs are requested before the partials so that all of the
     // kernel's global loads overlap
     const int chp = blockIdx.x * 32 + (threadIdx.x & 31);
@@ -215,6 +219,8 @@ __global__ void __launch_bounds__(1024) bn_stats_finish(const float* __restrict_
 __global__ void __launch_bounds__(1024) bn_bwd_finish(const float* __restrict__ partial, int blocks, int c, double count,
                                                      const float* __restrict__ mean, const float* __restrict__ rstd,
                                                      const float* __restrict__ gamma, BnBwdOut o) {
+    pdl_wait();
+    pdl_launch();
     const int chp = blockIdx.x * 32 + (threadIdx.x & 31);
     const bool owner = (threadIdx.x >> 5) == 0 && chp < c && o.dgamma != nullptr;
     const float pr = owner ? rstd[chp] : 0.f, pm = owner ? mean[chp] : 0.f, pg = owner ? gamma[chp] : 0.f;
@@ -235,6 +241,8 @@ __global__ void __launch_bounds__(1024) bn_bwd_finish(const float* __restrict__ 
 // ------------------------------------------------------------------ elementwise
 template <typename T, int V>
 __global__ void __launch_bounds__(256) ew_add_kernel(ValSrc a, ValSrc b, int act, size_t groups, int c, T* __restrict__ out, T* __restrict__ out2) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= groups) return;
     size_t e = i * V;
@@ -255,6 +263,8 @@ __global__ void __launch_bounds__(256) ew_add_kernel(ValSrc a, ValSrc b, int act
 // mode 0: dst = d * [out_val > 0];  mode 1: dst = a + b
 template <typename T, int V>
 __global__ void __launch_bounds__(256) ew_flat_kernel(int mode, const T* __restrict__ a, const T* __restrict__ b, size_t groups, T* __restrict__ dst) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= groups) return;
     float x[V], y[V];
@@ -266,6 +276,8 @@ __global__ void __launch_bounds__(256) ew_flat_kernel(int mode, const T* __restr
 }
 
 template <typename T> __global__ void gap_fwd_kernel(ValSrc x, int n, int hw, int c, T* __restrict__ out) {
+    pdl_wait();
+    pdl_launch();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n * c) return;
     int ch = i % c, s = i / c;
@@ -275,6 +287,8 @@ template <typename T> __global__ void gap_fwd_kernel(ValSrc x, int n, int hw, in
 }
 
 template <typename T> __global__ void gap_bwd_kernel(const T* __restrict__ da, int n, int hw, int c, const T* addend, T* dx) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (size_t)n * hw * c) return;
     int ch = (int)(i % c);
@@ -286,6 +300,8 @@ template <typename T> __global__ void gap_bwd_kernel(const T* __restrict__ da, i
 
 // ------------------------------------------------------------------ parameters
 __global__ void accumulate_kernel(float* __restrict__ G, const float* __restrict__ g, size_t n4, size_t n) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n4) {
         float4 a = reinterpret_cast<float4*>(G)[i];
@@ -307,6 +323,8 @@ __device__ __forceinline__ void sgd1(float& w, float& v, float& G, float inv_m, 
 
 __global__ void sgd_step_kernel(float* __restrict__ w, float* __restrict__ v, float* __restrict__ G, size_t n4, size_t n, float inv_m, float lr,
                                 float mu) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n4) {
         float4 a = reinterpret_cast<float4*>(w)[i], b = reinterpret_cast<float4*>(v)[i], c = reinterpret_cast<float4*>(G)[i];
@@ -325,6 +343,8 @@ __global__ void sgd_step_kernel(float* __restrict__ w, float* __restrict__ v, fl
 
 __global__ void refresh_kernel(const float* __restrict__ w, const int32_t* __restrict__ perm, float* __restrict__ d,
                                __nv_bfloat16* __restrict__ wb, __nv_bfloat16* __restrict__ wtb, size_t n) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float t = w[perm[i]];
@@ -389,6 +409,8 @@ __device__ void finish_loss(float part, float* scratch, unsigned* ticket, int np
 template <typename T>
 __global__ void __launch_bounds__(256) mse_kernel(const T* __restrict__ y, const T* __restrict__ t, size_t n, T* __restrict__ dy, float* loss,
                                                   float* scratch, unsigned* ticket) {
+    pdl_wait();
+    pdl_launch();
     __shared__ float sh[32];
     float acc = 0.f;
     const float k = 2.f / (float)n;
@@ -404,6 +426,8 @@ __global__ void __launch_bounds__(256) mse_kernel(const T* __restrict__ y, const
 template <typename T>
 __global__ void __launch_bounds__(256) xent_kernel(const T* __restrict__ logits, const int32_t* __restrict__ labels, int rows, int classes,
                                                    T* __restrict__ dl, float* loss, float* scratch, unsigned* ticket) {
+    pdl_wait();
+    pdl_launch();
     __shared__ float sh[32];
     const int r = blockIdx.x;
     const T* lg = logits + (size_t)r * classes;
@@ -437,9 +461,9 @@ void bn_stats(int dtype, const void* z, size_t pixels, int c, const float* gamma
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_STATS, (double)pixels * c * esz(dtype), st);
     LaunchScope ls(K_BN_STATS_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
     if (dtype == 0)
-        bn_stats_finish<float><<<(c + 31) / 32, 1024, 0, st>>>(scratch, (int)p.by, c, (const float*)z, (double)pixels, gamma, beta, eps, momentum, o);
+        launch_pdl(bn_stats_finish<float>, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (const float*)z, (double)pixels, gamma, beta, eps, momentum, o);
     else
-        bn_stats_finish<__nv_bfloat16><<<(c + 31) / 32, 1024, 0, st>>>(scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
+        launch_pdl(bn_stats_finish<__nv_bfloat16>, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
                                                                        momentum, o);
 }
 
@@ -450,13 +474,13 @@ void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int 
     BwdOp op{GradSrc{dy, z, scale, shift, nullptr, nullptr, nullptr, act}, mean, rstd};
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_BWD_REDUCE, (double)pixels * c * esz(dtype) * ((act != ACT_NONE || mean) ? 2.0 : 1.0), st);
     LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
-    bn_bwd_finish<<<(c + 31) / 32, 1024, 0, st>>>(scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
+    launch_pdl(bn_bwd_finish, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
 }
 
 template <typename T, int V> static void ew_add_launch(const ValSrc& a, const ValSrc& b, int act, size_t n, int c, void* out, void* out2, cudaStream_t st) {
     size_t groups = n / V;
     LaunchScope ls(K_EW_ADD, (double)n * sizeof(T) * (1 + (b.p ? 1 : 0) + 1 + (out2 ? 1 : 0)), (double)n, st);
-    ew_add_kernel<T, V><<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(a, b, act, groups, c, (T*)out, (T*)out2);
+    launch_pdl(ew_add_kernel<T, V>, (unsigned)((groups + 255) / 256), 256, 0, st, a, b, act, groups, c, (T*)out, (T*)out2);
 }
 
 void ew_add(int dtype, const ValSrc& a, const ValSrc& b, int act, size_t pixels, int c, void* out, void* out2, cudaStream_t st) {
@@ -478,7 +502,7 @@ void ew_apply(int dtype, const ValSrc& a, size_t pixels, int c, void* out, cudaS
 template <typename T, int V> static void ew_flat_launch(int mode, const void* a, const void* b, size_t n, void* dst, cudaStream_t st) {
     size_t groups = n / V;
     LaunchScope ls(mode == 0 ? K_EW_MASK : K_EW_SUM, 3.0 * n * sizeof(T), (double)n, st);
-    ew_flat_kernel<T, V><<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(mode, (const T*)a, (const T*)b, groups, (T*)dst);
+    launch_pdl(ew_flat_kernel<T, V>, (unsigned)((groups + 255) / 256), 256, 0, st, mode, (const T*)a, (const T*)b, groups, (T*)dst);
 }
 
 static void ew_flat(int dtype, int mode, const void* a, const void* b, size_t n, void* dst, cudaStream_t st) {
@@ -497,36 +521,36 @@ void ew_sum(int dtype, const void* a, const void* b, size_t n, void* dst, cudaSt
 void gap_fwd(int dtype, const ValSrc& x, int n, int hw, int c, void* out, cudaStream_t st) {
     int total = n * c;
     LaunchScope ls(K_GAP_FWD, ((double)total * hw + total) * esz(dtype), (double)total * hw, st);
-    if (dtype == 0) gap_fwd_kernel<float><<<(total + 127) / 128, 128, 0, st>>>(x, n, hw, c, (float*)out);
-    else gap_fwd_kernel<__nv_bfloat16><<<(total + 127) / 128, 128, 0, st>>>(x, n, hw, c, (__nv_bfloat16*)out);
+    if (dtype == 0) launch_pdl(gap_fwd_kernel<float>, (total + 127) / 128, 128, 0, st, x, n, hw, c, (float*)out);
+    else launch_pdl(gap_fwd_kernel<__nv_bfloat16>, (total + 127) / 128, 128, 0, st, x, n, hw, c, (__nv_bfloat16*)out);
 }
 
 void gap_bwd(int dtype, const void* da, int n, int hw, int c, const void* addend, void* dx, cudaStream_t st) {
     size_t total = (size_t)n * hw * c;
     unsigned blocks = (unsigned)((total + 255) / 256);
     LaunchScope ls(K_GAP_BWD, (double)total * esz(dtype) * (addend ? 2.0 : 1.0), (double)total, st);
-    if (dtype == 0) gap_bwd_kernel<float><<<blocks, 256, 0, st>>>((const float*)da, n, hw, c, (const float*)addend, (float*)dx);
-    else gap_bwd_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)da, n, hw, c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx);
+    if (dtype == 0) launch_pdl(gap_bwd_kernel<float>, blocks, 256, 0, st, (const float*)da, n, hw, c, (const float*)addend, (float*)dx);
+    else launch_pdl(gap_bwd_kernel<__nv_bfloat16>, blocks, 256, 0, st, (const __nv_bfloat16*)da, n, hw, c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx);
 }
 
 void accumulate(float* G, const float* g, size_t n, cudaStream_t st) {
     if (!n) return;
     size_t n4 = n / 4, threads = n4 + (n - n4 * 4);
     LaunchScope ls(K_ACCUMULATE, 12.0 * n, (double)n, st);
-    accumulate_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(G, g, n4, n);
+    launch_pdl(accumulate_kernel, (unsigned)((threads + 255) / 256), 256, 0, st, G, g, n4, n);
 }
 
 void sgd_step(float* w, float* v, float* G, size_t n, float inv_m, float lr, float mu, cudaStream_t st) {
     if (!n) return;
     size_t n4 = n / 4, threads = n4 + (n - n4 * 4);
     LaunchScope ls(K_SGD_STEP, 24.0 * n, 5.0 * n, st);
-    sgd_step_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(w, v, G, n4, n, inv_m, lr, mu);
+    launch_pdl(sgd_step_kernel, (unsigned)((threads + 255) / 256), 256, 0, st, w, v, G, n4, n, inv_m, lr, mu);
 }
 
 void refresh_derived(const float* w, const int32_t* perm, float* derived, __nv_bfloat16* wb, __nv_bfloat16* wtb, size_t n, cudaStream_t st) {
     if (!n) return;
     LaunchScope ls(K_REFRESH, (wb ? 20.0 : 12.0) * n, 0.0, st);
-    refresh_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w, perm, derived, wb, wtb, n);
+    launch_pdl(refresh_kernel, (unsigned)((n + 255) / 256), 256, 0, st, w, perm, derived, wb, wtb, n);
 }
 
 void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, cudaStream_t st) {
@@ -534,16 +558,16 @@ void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float
     int blocks = (int)(want < 1 ? 1 : (want > LOSS_MAX_BLOCKS ? LOSS_MAX_BLOCKS : want));
     unsigned* ticket = reinterpret_cast<unsigned*>(scratch + 65536);
     LaunchScope ls(K_LOSS_MSE, 3.0 * n * esz(dtype), 4.0 * n, st);
-    if (dtype == 0) mse_kernel<float><<<blocks, 256, 0, st>>>((const float*)y, (const float*)t, n, (float*)dy, loss, scratch, ticket);
-    else mse_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)y, (const __nv_bfloat16*)t, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
+    if (dtype == 0) launch_pdl(mse_kernel<float>, blocks, 256, 0, st, (const float*)y, (const float*)t, n, (float*)dy, loss, scratch, ticket);
+    else launch_pdl(mse_kernel<__nv_bfloat16>, blocks, 256, 0, st, (const __nv_bfloat16*)y, (const __nv_bfloat16*)t, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
 }
 
 void loss_xent(int dtype, const void* logits, const int32_t* labels, int rows, int classes, void* dlogits, float* loss, float* scratch,
                cudaStream_t st) {
     unsigned* ticket = reinterpret_cast<unsigned*>(scratch + 65536);
     LaunchScope ls(K_LOSS_XENT, 2.0 * rows * classes * esz(dtype), 6.0 * rows * classes, st);
-    if (dtype == 0) xent_kernel<float><<<rows, 256, 0, st>>>((const float*)logits, labels, rows, classes, (float*)dlogits, loss, scratch, ticket);
-    else xent_kernel<__nv_bfloat16><<<rows, 256, 0, st>>>((const __nv_bfloat16*)logits, labels, rows, classes, (__nv_bfloat16*)dlogits, loss, scratch, ticket);
+    if (dtype == 0) launch_pdl(xent_kernel<float>, rows, 256, 0, st, (const float*)logits, labels, rows, classes, (float*)dlogits, loss, scratch, ticket);
+    else launch_pdl(xent_kernel<__nv_bfloat16>, rows, 256, 0, st, (const __nv_bfloat16*)logits, labels, rows, classes, (__nv_bfloat16*)dlogits, loss, scratch, ticket);
 }
 
 }  // namespace ast
@@ -584,8 +608,8 @@ extern "C" int asteroid_loss_mse_noalloc(const void* y, const void* target, size
     int blocks = (int)(want < 1 ? 1 : (want > LOSS_MAX_BLOCKS ? LOSS_MAX_BLOCKS : want));
     {
         LaunchScope ls(K_LOSS_MSE, 3.0 * n * (dtype == 0 ? 4.0 : 2.0), 4.0 * n, st);
-        if (dtype == 0) mse_kernel<float><<<blocks, 256, 0, st>>>((const float*)y, (const float*)target, n, (float*)dy, loss, scratch, ticket);
-        else mse_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)y, (const __nv_bfloat16*)target, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
+        if (dtype == 0) launch_pdl(mse_kernel<float>, blocks, 256, 0, st, (const float*)y, (const float*)target, n, (float*)dy, loss, scratch, ticket);
+        else launch_pdl(mse_kernel<__nv_bfloat16>, blocks, 256, 0, st, (const __nv_bfloat16*)y, (const __nv_bfloat16*)target, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
     }
     if (cudaGetLastError() != cudaSuccess) return report_error(-5, "asteroid_loss_mse_noalloc: kernel launch failed");
     return 0;

@@ -41,6 +41,14 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// Programmatic dependent launch.  Every kernel of the library is launched with programmatic
+// stream serialization allowed and opens with pdl_wait(): nothing of the previous kernel in the
+// stream is read or overwritten before that kernel has completed and its writes are visible.
+// pdl_launch() then lets the next kernel's blocks be scheduled as soon as SM resources free up,
+// so its launch latency overlaps this kernel's execution.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float apply_act(float v, int act) {
     if (act == ACT_RELU6) return fminf(fmaxf(v, 0.f), 6.f);
     if (act == ACT_RELU) return fmaxf(v, 0.f);

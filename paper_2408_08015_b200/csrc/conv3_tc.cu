@@ -40,6 +40,8 @@ struct C3Args {
 __device__ __forceinline__ uint64_t make_desc_row(uint32_t smem_addr) { return make_desc(smem_addr); }
 
 template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kernel(const C3Args a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2];
     __shared__ uint32_t tmem_slot;
@@ -182,7 +184,7 @@ template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, cudaStream
         attr_set = true;
     }
     LaunchScope ls(kind, bytes, 2.0 * 9.0 * a.n_img * a.H * a.W * (double)a.C * a.N, st);
-    conv3_tc_kernel<BWD><<<a.n_img * a.tiles_per_img, C3_THREADS, smem, st>>>(a);
+    launch_pdl(conv3_tc_kernel<BWD>, a.n_img * a.tiles_per_img, C3_THREADS, smem, st, a);
 }
 
 
@@ -215,6 +217,8 @@ __device__ __forceinline__ uint64_t make_desc_mn_lbo(uint32_t smem_addr, uint32_
 }
 
 __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_store;
     __shared__ uint32_t tmem_slot;
@@ -332,6 +336,8 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
 }
 
 __global__ void __launch_bounds__(1024) reduce_splits_c3(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
+    pdl_wait();
+    pdl_launch();
     __shared__ float sh[32][33];
     const int il = threadIdx.x & 31, kg = threadIdx.x >> 5;
     const size_t i = (size_t)blockIdx.x * 32 + il;
@@ -423,10 +429,10 @@ void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, 
     {
         LaunchScope ls(K_CONV3_BWD_WEIGHT_TC, 2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci + 4.0 * out_elems * ctas,
                        2.0 * 9.0 * px * g.ci * g.co, st);
-        conv3_wgrad_tc_kernel<<<dim3(ctas, groups), C3_THREADS, smem, st>>>(a);
+        launch_pdl(conv3_wgrad_tc_kernel, dim3(ctas, groups), C3_THREADS, smem, st, a);
     }
     LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);
-    reduce_splits_c3<<<(unsigned)((out_elems + 31) / 32), 1024, 0, st>>>(scratch, ctas, out_elems, gw);
+    launch_pdl(reduce_splits_c3, (unsigned)((out_elems + 31) / 32), 1024, 0, st, scratch, ctas, out_elems, gw);
 }
 
 }  // namespace ast

@@ -49,6 +49,8 @@ template <typename T> __device__ __forceinline__ float operand(float v) { return
 template <> __device__ __forceinline__ float operand<__nv_bfloat16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
 template <typename T, int MODE> __global__ void __launch_bounds__(NT) igemm_kernel(const IgemmArgs a) {
+    pdl_wait();
+    pdl_launch();
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const ConvGeom& g = a.g;
@@ -178,6 +180,8 @@ template <typename T, int MODE> __global__ void __launch_bounds__(NT) igemm_kern
 }
 
 __global__ void reduce_splits_kernel(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float s = 0.f;
@@ -194,9 +198,9 @@ __global__ void reduce_splits_kernel(const float* __restrict__ partial, int spli
 template <int MODE> void launch(int dtype, const IgemmArgs& a, dim3 grid, int kind, double bytes, cudaStream_t st) {
     LaunchScope ls(kind, bytes, 2.0 * a.M * a.N * a.K, st);
     if (dtype == 0)
-        igemm_kernel<float, MODE><<<grid, NT, 0, st>>>(a);
+        launch_pdl(igemm_kernel<float, MODE>, grid, NT, 0, st, a);
     else
-        igemm_kernel<__nv_bfloat16, MODE><<<grid, NT, 0, st>>>(a);
+        launch_pdl(igemm_kernel<__nv_bfloat16, MODE>, grid, NT, 0, st, a);
 }
 
 double esz(int dtype) { return dtype == 0 ? 4.0 : 2.0; }
@@ -242,7 +246,7 @@ void conv_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValS
     double bytes = grad_src_bytes(dz, (double)a.K * g.co, dtype) + (double)g.n * g.hi * g.wi * g.ci * esz(dtype) + 4.0 * out_elems * splits;
     launch<MODE_BWD_WEIGHT>(dtype, a, dim3((a.M + BM - 1) / BM, (a.N + BN - 1) / BN, splits), K_CONV_BWD_WEIGHT, bytes, st);
     LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (splits + 1), (double)out_elems * splits, st);
-    reduce_splits_kernel<<<(unsigned)((out_elems + 255) / 256), 256, 0, st>>>(scratch, splits, out_elems, gw);
+    launch_pdl(reduce_splits_kernel, (unsigned)((out_elems + 255) / 256), 256, 0, st, scratch, splits, out_elems, gw);
 }
 
 }  // namespace ast

@@ -77,6 +77,8 @@ template <typename T, int V> struct ValLoader {
 template <typename T, int V, int S, bool FLIP, typename LOADER, typename SRC>
 __global__ void __launch_bounds__(128) dw_strip_kernel(int n_img, int hi, int wi, int ho, int wo, int c, SRC src, const float* __restrict__ w9c,
                                                        const T* addend, T* out) {
+    pdl_wait();
+    pdl_launch();
     constexpr int NIN = (TW - 1) * S + 3;
     const int cv = c / V, sw = (wo + TW - 1) / TW;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -243,6 +245,8 @@ template <typename T, int V> struct GradRoll {
 template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC>
 __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, int c, int th, SRC src, const float* __restrict__ w9c,
                                                       const T* addend, T* out) {
+    pdl_wait();
+    pdl_launch();
     constexpr int NIN = TWR + 2;
     extern __shared__ float wsm[];            // [9][c], tap order already flipped for the adjoint
     for (int i = threadIdx.x; i < 9 * c; i += blockDim.x) {
@@ -343,7 +347,7 @@ void launch_roll(int n, int h, int w, int c, const SRC& src, const float* w9c, c
     int th = h >= 28 ? 8 : (h >= 14 ? 7 : h);
     size_t total = (size_t)n * ((h + th - 1) / th) * ((w + TWR - 1) / TWR) * (c / V);
     size_t smem = (size_t)9 * c * sizeof(float);
-    dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
+    launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC>, (unsigned)((total + 127) / 128), 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
 }
 
 
@@ -367,6 +371,8 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 template <typename T, int V, int TWR, int D>
 __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, int cw, int rows, int th, size_t items_per_block,
                                                             float* __restrict__ partial) {
+    pdl_wait();
+    pdl_launch();
     constexpr int NIN = TWR + 2, NL = NIN + 2 * TWR;
     typedef typename RawT<T, V>::type raw_t;
     extern __shared__ __align__(16) uint8_t dsm[];
@@ -511,6 +517,8 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
 template <typename T, int V, int TWR, int D>
 __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, const float* __restrict__ w9c, const T* addend,
                                                            T* dx, int cw, int rows, size_t items_per_block, float* __restrict__ partial) {
+    pdl_wait();
+    pdl_launch();
     constexpr int NIN = TWR + 2, NL = 3 * NIN;
     typedef typename RawT<T, V>::type raw_t;
     extern __shared__ __align__(16) uint8_t dsm[];
@@ -683,6 +691,8 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
 // 2i, 2i+1 (2*TWZ columns each).  Every dz element is loaded and transformed once per thread.
 template <typename T, int V, int TWZ>
 __global__ void __launch_bounds__(128) dw_bwd_data_s2_kernel(ConvGeom g, GradSrc dzs, const float* __restrict__ w9c, int th, const T* addend, T* dx) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ float wsm[];            // [9][c]
     const int c = g.ci, H = g.hi, W = g.wi, Ho = g.ho, Wo = g.wo;
     for (int i = threadIdx.x; i < 9 * c; i += blockDim.x) wsm[i] = __ldg(w9c + i);
@@ -780,6 +790,8 @@ __global__ void __launch_bounds__(128) dw_bwd_data_s2_kernel(ConvGeom g, GradSrc
 template <typename T, int V, int TWZ>
 __global__ void __launch_bounds__(128) dw_wgrad_s2_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, int cw, int rows, int th, size_t items_per_block,
                                                           float* __restrict__ partial) {
+    pdl_wait();
+    pdl_launch();
     constexpr int NX = 2 * TWZ + 1;
     extern __shared__ float red[];
     const int cv = g.ci / V;
@@ -900,6 +912,8 @@ __global__ void __launch_bounds__(128) dw_wgrad_s2_kernel(ConvGeom g, GradSrc dz
 
 // gw[c][t] = sum_b partial[b][t][c]; one warp per (t, c): lanes stride over the blocks
 __global__ void __launch_bounds__(128) dw_bwd_weight_finish(const float* __restrict__ partial, int blocks, int c_total, float* __restrict__ gw) {
+    pdl_wait();
+    pdl_launch();
     int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (i >= 9 * c_total) return;
     int t = i / c_total, c = i % c_total;
@@ -921,7 +935,7 @@ double grad_src_bytes(const GradSrc& d, double elems, int dtype) { return elems 
 template <typename T, int V, int S, bool FLIP, typename LOADER, typename SRC>
 void launch_strip(int n, int hi, int wi, int ho, int wo, int c, const SRC& src, const float* w9c, const void* addend, void* out, cudaStream_t st) {
     size_t total = (size_t)n * ho * ((wo + TW - 1) / TW) * (c / V);
-    dw_strip_kernel<T, V, S, FLIP, LOADER, SRC><<<(unsigned)((total + 127) / 128), 128, 0, st>>>(n, hi, wi, ho, wo, c, src, w9c, (const T*)addend, (T*)out);
+    launch_pdl(dw_strip_kernel<T, V, S, FLIP, LOADER, SRC>, (unsigned)((total + 127) / 128), 128, 0, st, n, hi, wi, ho, wo, c, src, w9c, (const T*)addend, (T*)out);
 }
 
 }  // namespace
@@ -953,8 +967,8 @@ void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w
         const int th = nrowz >= 14 ? 7 : nrowz;
         size_t total = (size_t)g.n * ((nrowz + th - 1) / th) * ((ncolz + TWZ - 1) / TWZ) * (g.ci / 4);
         size_t smem = (size_t)9 * g.ci * sizeof(float);
-        if (dtype == 0) dw_bwd_data_s2_kernel<float, 4, TWZ><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(g, dz, w9c, th, (const float*)addend, (float*)dx);
-        else dw_bwd_data_s2_kernel<B, 4, TWZ><<<(unsigned)((total + 127) / 128), 128, smem, st>>>(g, dz, w9c, th, (const B*)addend, (B*)dx);
+        if (dtype == 0) launch_pdl(dw_bwd_data_s2_kernel<float, 4, TWZ>, (unsigned)((total + 127) / 128), 128, smem, st, g, dz, w9c, th, (const float*)addend, (float*)dx);
+        else launch_pdl(dw_bwd_data_s2_kernel<B, 4, TWZ>, (unsigned)((total + 127) / 128), 128, smem, st, g, dz, w9c, th, (const B*)addend, (B*)dx);
     }
 }
 
@@ -989,10 +1003,10 @@ void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc
         constexpr int NL = TWR + 2 + 2 * TWR;
         if (dtype == 0) {
             constexpr int D = 2;
-            dw_wgrad_roll_kernel<float, 4, TWR, D><<<grid, 128, (size_t)D * NL * 128 * 16, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+            launch_pdl(dw_wgrad_roll_kernel<float, 4, TWR, D>, grid, 128, (size_t)D * NL * 128 * 16, st, g, dz, x, cw, rows, th, ipb, scratch);
         } else {
             constexpr int D = 4;
-            dw_wgrad_roll_kernel<__nv_bfloat16, 4, TWR, D><<<grid, 128, (size_t)D * NL * 128 * 8, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+            launch_pdl(dw_wgrad_roll_kernel<__nv_bfloat16, 4, TWR, D>, grid, 128, (size_t)D * NL * 128 * 8, st, g, dz, x, cw, rows, th, ipb, scratch);
         }
     } else {
         const int th = g.ho >= 28 ? 8 : (g.ho >= 14 ? 7 : g.ho);      // rows of dz per work item
@@ -1008,11 +1022,11 @@ void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc
         const size_t smem = (size_t)rows * cw * V * sizeof(float);
         dim3 grid(gx, (unsigned)by);
         LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
-        if (dtype == 0) dw_wgrad_s2_kernel<float, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
-        else dw_wgrad_s2_kernel<__nv_bfloat16, 4, TWR><<<grid, 128, smem, st>>>(g, dz, x, cw, rows, th, ipb, scratch);
+        if (dtype == 0) launch_pdl(dw_wgrad_s2_kernel<float, 4, TWR>, grid, 128, smem, st, g, dz, x, cw, rows, th, ipb, scratch);
+        else launch_pdl(dw_wgrad_s2_kernel<__nv_bfloat16, 4, TWR>, grid, 128, smem, st, g, dz, x, cw, rows, th, ipb, scratch);
     }
     LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
-    dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
+    launch_pdl(dw_bwd_weight_finish, (9 * g.ci + 3) / 4, 128, 0, st, scratch, (int)by, g.ci, gw);
 }
 
 bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, const float* w9c, const void* addend, void* dx,
@@ -1046,11 +1060,11 @@ bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc&
     {
         LaunchScope ls(K_DW_BWD_FUSED, grad_src_bytes(dz, e, dtype) + e * 2.0 * (addend ? 3.0 : 2.0) + 36.0 * g.ci * (by + 1), 36.0 * e, st);
         dim3 grid(gx, (unsigned)by);
-        dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D><<<grid, 128, smem, st>>>(g, dz, x, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx, cw,
+        launch_pdl(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D>, grid, 128, smem, st, g, dz, x, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx, cw,
                                                                             rows, ipb, scratch);
     }
     LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
-    dw_bwd_weight_finish<<<(9 * g.ci + 3) / 4, 128, 0, st>>>(scratch, (int)by, g.ci, gw);
+    launch_pdl(dw_bwd_weight_finish, (9 * g.ci + 3) / 4, 128, 0, st, scratch, (int)by, g.ci, gw);
     return true;
 }
 

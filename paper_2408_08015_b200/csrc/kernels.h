@@ -20,6 +20,23 @@ enum KernelKind {
 };
 const char* kernel_name(int kind);
 
+// Launches `kernel` on `st` with programmatic stream serialization allowed (the kernel must open
+// with pdl_wait()).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Brackets one kernel launch: counts it and, while a trace is active, records a CUDA event on
 // `st` before and after it together with the bytes the kernel must move (each tensor once)
 // and its floating-point operations.

@@ -39,6 +39,8 @@ struct PwArgs {
 };
 
 template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(const PwArgs a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t mbar_store;
     __shared__ uint32_t tmem_slot;
@@ -204,6 +206,8 @@ __device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr) {
 }
 
 __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArgs a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t mbar_store[2];
     __shared__ uint32_t tmem_slot;
@@ -328,6 +332,8 @@ __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArg
 }
 
 __global__ void reduce_splits_tc(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
+    pdl_wait();
+    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float s = 0.f;
@@ -437,6 +443,8 @@ struct PipeArgs {
 };
 
 template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const PipeArgs a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * MAX_RAW + 8];   // raw_full[R], raw_empty[R], a_full[2], a_empty[2], acc_full[2], acc_empty[2]
     __shared__ uint32_t tmem_slot;
@@ -684,7 +692,7 @@ template <bool BWD> void launch_pipe(const PipeArgs& a, size_t smem, int kind, d
     }
     LaunchScope ls(kind, bytes, 2.0 * a.P * a.N * a.K, st);
     int grid = a.tiles < n_sm ? a.tiles : n_sm;
-    pw_pipe_kernel<BWD><<<grid, PIPE_THREADS, smem, st>>>(a);
+    launch_pdl(pw_pipe_kernel<BWD>, grid, PIPE_THREADS, smem, st, a);
 }
 
 
@@ -715,6 +723,8 @@ struct WgArgs {
 };
 
 __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgArgs a) {
+    pdl_wait();
+    pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * MAX_RAW + 5];    // raw_full[R], raw_empty[R], op_full[2], op_empty[2], done
     __shared__ uint32_t tmem_slot;
@@ -883,6 +893,8 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
 // load: coalesced; all of a thread's loads are issued before the additions), the 32 sub-sums
 // are combined in fixed order through shared memory.
 __global__ void __launch_bounds__(1024) reduce_splits_2d(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
+    pdl_wait();
+    pdl_launch();
     __shared__ float sh[32][33];
     const int il = threadIdx.x & 31, kg = threadIdx.x >> 5;
     const size_t i = (size_t)blockIdx.x * 32 + il;
@@ -970,7 +982,7 @@ template <bool BWD> void launch(const PwArgs& a0, const Tiling& t, int kind, dou
     }
     LaunchScope ls(kind, bytes, 2.0 * a.P * a.N * a.K, st);
     dim3 grid((a.P + TM - 1) / TM, t.ntiles);
-    pw_tc_kernel<BWD><<<grid, NTHREADS, t.smem, st>>>(a);
+    launch_pdl(pw_tc_kernel<BWD>, grid, NTHREADS, t.smem, st, a);
 }
 
 }  // namespace
@@ -1054,11 +1066,11 @@ void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, flo
             double bytes = 2.0 * (double)wa.P * wa.CO * (wa.need_z ? 2.0 : 1.0) + 2.0 * (double)wa.P * wa.CI + 4.0 * wa.CO * wa.CI * (2.0 * ctas + 1);
             {
                 LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * wa.P * wa.CO * wa.CI, st);
-                pw_wgrad_pipe_kernel<<<ctas, WG_THREADS, smem, st>>>(wa);
+                launch_pdl(pw_wgrad_pipe_kernel, ctas, WG_THREADS, smem, st, wa);
             }
             size_t out_elems = (size_t)wa.CO * wa.CI;
             LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);
-            reduce_splits_2d<<<(unsigned)((out_elems + 31) / 32), 1024, 0, st>>>(scratch, ctas, out_elems, gw);
+            launch_pdl(reduce_splits_2d, (unsigned)((out_elems + 31) / 32), 1024, 0, st, scratch, ctas, out_elems, gw);
             return;
         }
     }
@@ -1093,10 +1105,10 @@ void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, flo
                    4.0 * out_elems * splits;
     {
         LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * a.P * a.CO * a.CI, st);
-        pw_bwd_weight_tc_kernel<<<dim3(mtiles, splits, ntiles), NTHREADS, smem, st>>>(a);
+        launch_pdl(pw_bwd_weight_tc_kernel, dim3(mtiles, splits, ntiles), NTHREADS, smem, st, a);
     }
     LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (splits + 1), (double)out_elems * splits, st);
-    reduce_splits_tc<<<(unsigned)((out_elems + 255) / 256), 256, 0, st>>>(scratch, splits, out_elems, gw);
+    launch_pdl(reduce_splits_tc, (unsigned)((out_elems + 255) / 256), 256, 0, st, scratch, splits, out_elems, gw);
 }
 
 }  // namespace ast
