@@ -234,9 +234,11 @@ template <typename T, int V> struct GradRoll {
         raw_decode(r.b, zz);
 #pragma unroll
         for (int q = 0; q < V; ++q) {
+            // lo < pre < hi  <=>  (pre - lo) * (hi - pre) > 0 (exact signs; infinite bounds give +inf,
+            // 0 * inf = NaN compares false): the test runs on the FMA pipe and guards one fused multiply-add
             const float pre = fmaf(zz[q], scale[q], shift[q]);
-            float d = (pre > lo && pre < hi) ? f[q] : 0.f;
-            d = fmaf(k1[q], d, fmaf(k3[q], zz[q], k2[q]));
+            float d = fmaf(k3[q], zz[q], k2[q]);
+            if ((pre - lo) * (hi - pre) > 0.f) d = fmaf(k1[q], f[q], d);
             f[q] = ok ? d : 0.f;
         }
     }

@@ -414,9 +414,13 @@ struct XfGrad {
         v.unpack(z);
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
+            // lo < pre < hi  <=>  (pre - lo) * (hi - pre) > 0: differences of floats keep their sign
+            // exactly, infinite bounds give +inf, and 0 * inf = NaN compares false (pre == 0 under ReLU);
+            // the test runs on the FMA pipe and guards one predicated fused multiply-add
             const float pre = fmaf(z[q], cs[q], ch[q]);
-            const float d = (pre > lo && pre < hi) ? f[q] : 0.f;
-            f[q] = fmaf(k1[q], d, fmaf(k3[q], z[q], k2[q]));
+            float o = fmaf(k3[q], z[q], k2[q]);
+            if ((pre - lo) * (hi - pre) > 0.f) o = fmaf(k1[q], f[q], o);
+            f[q] = o;
         }
         return pack8(f);
     }
@@ -579,21 +583,24 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
                 }
                 const uint8_t* raw = sR + (size_t)s * a.raw_bytes;
                 if (active) {
+                    // straight-line body (rows past the end of the tensor and the K padding are
+                    // read like any other and zeroed afterwards) so that the unrolled iterations'
+                    // loads and arithmetic interleave
+                    const int jl = data ? j : 0;
+                    const int rows_left = a.P - tile * TM - sub * RS;
 #pragma unroll 4
                     for (int rl = grp; rl < RS; rl += groups) {
-                        const int r = sub * RS + rl;
-                        uint4 q4 = make_uint4(0, 0, 0, 0);
-                        if (data && tile * TM + r < a.P) {
-                            const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)rl * row_bytes + (j << 4));
-                            if (!BWD) {
-                                q4 = xv.apply(r0);
-                            } else if (a.need_z) {
-                                q4 = xg.apply(r0, *reinterpret_cast<const uint4*>(raw + (size_t)(RS + rl) * row_bytes + (j << 4)));
-                            } else {
-                                q4 = r0;
-                            }
+                        const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)rl * row_bytes + (jl << 4));
+                        uint4 q4;
+                        if (!BWD) {
+                            q4 = xv.apply(r0);
+                        } else if (a.need_z) {
+                            q4 = xg.apply(r0, *reinterpret_cast<const uint4*>(raw + (size_t)(RS + rl) * row_bytes + (jl << 4)));
+                        } else {
+                            q4 = r0;
                         }
-                        *reinterpret_cast<uint4*>(dstA + tile_off(r, j, TM)) = q4;
+                        if (!data || rl >= rows_left) q4 = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4*>(dstA + tile_off(sub * RS + rl, j, TM)) = q4;
                     }
                 }
                 mbar_arrive(raw_empty(s));
@@ -837,18 +844,19 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
             uint8_t* dstA = sOp + (size_t)st * a.op_bytes + (uint32_t)(ja >> 3) * PANEL;
             uint8_t* dstB = sOp + (size_t)st * a.op_bytes + (uint32_t)(a.pa + (jb >> 3)) * PANEL;
             const int valid = min(WSTAGE, pend - (pbeg + it * WSTAGE));
-#pragma unroll 2
+            // straight-line bodies: rows past the end of the CTA's range are transformed like any
+            // other (stale but in-bounds shared memory) and zeroed afterwards
+#pragma unroll 4
             for (int kr = ga; kr < rowsA; kr += groupsA) {
-                uint4 q4 = make_uint4(0, 0, 0, 0);
-                if (kr < valid) {
-                    const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)kr * rowA + (ja << 4));
-                    q4 = a.need_z ? xg.apply(r0, *reinterpret_cast<const uint4*>(raw + offZ + (size_t)kr * rowA + (ja << 4))) : r0;
-                }
+                const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)kr * rowA + (ja << 4));
+                uint4 q4 = a.need_z ? xg.apply(r0, *reinterpret_cast<const uint4*>(raw + offZ + (size_t)kr * rowA + (ja << 4))) : r0;
+                if (kr >= valid) q4 = make_uint4(0, 0, 0, 0);
                 *reinterpret_cast<uint4*>(dstA + kr * 128 + (((ja & 7) ^ (kr & 7)) << 4)) = q4;
             }
+#pragma unroll 2
             for (int kr = gb; kr < rowsB; kr += groupsB) {
-                uint4 q4 = make_uint4(0, 0, 0, 0);
-                if (kr < valid) q4 = xv.apply(*reinterpret_cast<const uint4*>(raw + offX + (size_t)kr * rowB + (jb << 4)));
+                uint4 q4 = xv.apply(*reinterpret_cast<const uint4*>(raw + offX + (size_t)kr * rowB + (jb << 4)));
+                if (kr >= valid) q4 = make_uint4(0, 0, 0, 0);
                 *reinterpret_cast<uint4*>(dstB + kr * 128 + (((jb & 7) ^ (kr & 7)) << 4)) = q4;
             }
             mbar_arrive(raw_empty(s));
