@@ -195,8 +195,10 @@ __global__ void __launch_bounds__(1024) bn_stats_finish(const float* __restrict_
     // kernel's global loads overlap
     const int chp = blockIdx.x * 32 + (threadIdx.x & 31);
     const bool owner = (threadIdx.x >> 5) == 0 && chp < c;
-    const float pv = owner ? to_f<T>(z[chp]) : 0.f, gm = owner ? gamma[chp] : 0.f, bt = owner ? beta[chp] : 0.f;
+    // pivot: the first pixel's value, or (z == nullptr: partials written by the producing kernel) the running mean
+    // as it stands before this update
     const float rm = owner ? o.run_mean[chp] : 0.f, rv = owner ? o.run_var[chp] : 0.f;
+    const float pv = owner ? (z ? to_f<T>(z[chp]) : rm) : 0.f, gm = owner ? gamma[chp] : 0.f, bt = owner ? beta[chp] : 0.f;
     int ch;
     double s1, s2;
     if (!sum_partials(partial, blocks, c, ch, s1, s2)) return;
@@ -465,6 +467,13 @@ void bn_stats(int dtype, const void* z, size_t pixels, int c, const float* gamma
     else
         launch_pdl(bn_stats_finish<__nv_bfloat16>, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (const __nv_bfloat16*)z, (double)pixels, gamma, beta, eps,
                                                                        momentum, o);
+}
+
+void bn_stats_finish_partials(const float* partial, int blocks, size_t pixels, int c, const float* gamma, const float* beta, float eps,
+                              float momentum, const BnFwdOut& o, cudaStream_t st) {
+    LaunchScope ls(K_BN_STATS_FINISH, 8.0 * c * (blocks + 4), 10.0 * c, st);
+    launch_pdl(bn_stats_finish<float>, (c + 31) / 32, 1024, 0, st, partial, blocks, c, (const float*)nullptr, (double)pixels, gamma, beta, eps, momentum,
+               o);
 }
 
 void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int c, const float* scale, const float* shift, int act,

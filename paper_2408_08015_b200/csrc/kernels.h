@@ -62,7 +62,11 @@ void conv_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValS
 // ---- pointwise conv on tcgen05 tensor cores (bf16 storage, channel counts multiples of 8) ----
 bool pw_tc_supported(int dtype, const ConvGeom& g, bool bwd_data);
 // wb: bf16 weights [co][ci]; wtb: bf16 transposed weights [ci][co]; err: device error word
-void pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const float* bias, void* z, int* err, cudaStream_t st);
+// With `pivot` and `partial` given, the pipelined kernel also writes the BatchNorm statistics partials of its output,
+// partial[cta][2][co] = sums of (z - pivot[c]) and (z - pivot[c])^2 over the CTA's pixels (z as stored, after rounding),
+// and returns the number of CTAs (for bn_stats_finish_partials); 0 = no partials written, statistics need their own pass.
+int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const float* bias, void* z, const float* pivot, float* partial,
+              size_t partial_floats, int* err, cudaStream_t st);
 void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st);
 // gw[co][ci]; per-CTA partial sums in scratch, summed in fixed order by a second kernel
 void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
@@ -93,6 +97,10 @@ struct BnFwdOut {
 };
 void bn_stats(int dtype, const void* z, size_t pixels, int c, const float* gamma, const float* beta, float eps, float momentum,
               float* scratch, size_t scratch_floats, const BnFwdOut& o, cudaStream_t st);
+// finishing step alone, for statistics partials written by the producing kernel; the pivot is the running mean
+// as it stood before this call (the value the producer read)
+void bn_stats_finish_partials(const float* partial, int blocks, size_t pixels, int c, const float* gamma, const float* beta, float eps,
+                              float momentum, const BnFwdOut& o, cudaStream_t st);
 struct BnBwdOut {
     float *dgamma, *dbeta, *k1, *k2, *k3;   // dgamma/k* null: only dbeta = sum of dpre (bias gradient)
 };

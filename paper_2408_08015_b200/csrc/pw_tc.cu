@@ -444,9 +444,15 @@ struct PipeArgs {
     int need_z;                 // backward: the transform also reads z
     uint32_t raw_bytes;         // bytes of one raw stage (both tensors), multiple of 128
     uint32_t a_bytes, b_bytes;  // one operand stage / the resident weights
+    uint32_t o_bytes;           // one output staging tile [128][N] bf16 (multiple of 128)
+    int OS;                     // output staging tiles: 1 or 2
+    const float* pivot;         // forward, optional: per-channel pivot of the fused BatchNorm statistics
+    float* stat_partial;        // [CTAs][2][N]: sums of (z - pivot) and (z - pivot)^2 over the CTA's pixels
 };
 
-template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const PipeArgs a) {
+// EXTRA: the epilogue adds the bias (forward) or the residual gradient (backward); a template
+// parameter because even a never-taken branch around those loads slows the epilogue's inner loop.
+template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const PipeArgs a) {
     pdl_wait();
     pdl_launch();
     extern __shared__ uint8_t smem_raw[];
@@ -458,6 +464,7 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
     uint8_t* sA = base;                               // two operand stages
     uint8_t* sB = base + 2 * (size_t)a.a_bytes;       // resident weights
     uint8_t* sR = sB + a.b_bytes;                     // raw ring
+    uint8_t* sO = sR + (size_t)a.R * a.raw_bytes;     // output staging tiles
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = a.R, RS = a.RS, subs = TM / RS;
     const uint32_t bar0 = smem_u32(&bars[0]);
@@ -611,41 +618,122 @@ template <bool BWD> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_k
         }
     } else {
         // ------------------------------------------------------------ epilogue
+        // The 128 epilogue threads (one accumulator row each) round the tile to bf16 into a
+        // shared-memory staging tile laid out exactly like the output rows in global memory, which
+        // are one contiguous byte range; one thread then stores the tile with a single bulk copy.
+        // Forward with statistics: the same threads then sum (z - pivot) and (z - pivot)^2 down the
+        // columns of the staged (rounded) tile, eight channels per thread, accumulating over the
+        // CTA's tiles in registers.
         const int q = warp & 3;                            // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
+        const int et = tid - (PIPE_THREADS - 128);
+        const uint32_t row_out = (uint32_t)a.N * 2u;
+        const bool stats = !BWD && a.stat_partial != nullptr;
+        const int units = a.N >> 3;                        // 8-channel column groups
+        const int rsplit = 128 / units;                    // threads per column group (N <= 256: at least 4)
+        const int cu = et % units, rh = et / units;
+        const bool sactive = stats && rh < rsplit;
+        float s1[8], s2[8], piv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            s1[i] = s2[i] = 0.f;
+            piv[i] = sactive ? __ldg(a.pivot + (cu << 3) + i) : 0.f;
+        }
+        int issued = 0;
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
             const int st = t & 1, n = t >> 1;
-            if (!mbar_wait_abortable(acc_full(st), (uint32_t)(n & 1), abort_flag)) break;
+            const int ob = a.OS == 2 ? (t & 1) : 0;
+            uint8_t* so = sO + (size_t)ob * a.o_bytes;
+            bool ok = mbar_wait_abortable(acc_full(st), (uint32_t)(n & 1), abort_flag);
+            // the bulk store that last read this staging tile must have finished reading it
+            if (et == 0) {
+                if (a.OS == 2) bulk_wait_read<1>();
+                else bulk_wait_read<0>();
+            }
+            ok = named_bar_and(1, 128, ok);
+            if (!ok) break;
             fence_after_sync();
             const int p = tile * TM + row;
-            for (int g = 0; g < (NT >> 4); ++g) {
-                float v[16];
-                tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(st * NT + (g << 4)), v);
+            // accumulator columns in batches of up to 64: the batch's tcgen05.ld are all issued
+            // before the one wait, so their latencies overlap
+            for (int g0 = 0; g0 < (NT >> 4); g0 += 4) {
+                uint32_t rr[4][16];
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int nn = (g << 4) + (hh << 3);
-                    if (p < a.P && nn < a.N) {
-                        float* vv = v + (hh << 3);
-                        const size_t e = (size_t)p * a.N + nn;
-                        if (!BWD && a.bias) {
+                for (int u = 0; u < 4; ++u)
+                    if (g0 + u < (NT >> 4)) tmem_ld16_issue(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(st * NT + ((g0 + u) << 4)), rr[u]);
+                tmem_ld_wait();
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) vv[i] += __ldg(a.bias + nn + i);
+                for (int u = 0; u < 4; ++u) {
+                    if (g0 + u < (NT >> 4)) tmem_ld_pin16(rr[u]);
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int nn = ((g0 + u) << 4) + (hh << 3);
+                        if (nn < a.N) {
+                            float vv[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) vv[i] = __uint_as_float(rr[u][(hh << 3) + i]);
+                            if (!BWD && EXTRA) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) vv[i] += __ldg(a.bias + nn + i);
+                            }
+                            if (BWD && EXTRA && p < a.P) {
+                                float ad[8];
+                                Vec<__nv_bfloat16> av;
+                                av.load(a.addend, ((size_t)p * a.N + nn) >> 3);
+                                av.unpack(ad);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) vv[i] += ad[i];
+                            }
+                            *reinterpret_cast<uint4*>(so + (size_t)row * row_out + (nn << 1)) = pack8(vv);
                         }
-                        if (BWD && a.addend) {
-                            float ad[8];
-                            Vec<__nv_bfloat16> av;
-                            av.load(a.addend, e >> 3);
-                            av.unpack(ad);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) vv[i] += ad[i];
-                        }
-                        *reinterpret_cast<uint4*>(a.out + e) = pack8(vv);
                     }
                 }
             }
             fence_before_sync();
             mbar_arrive(acc_empty(st));
+            fence_async_smem();
+            named_bar_sync(1, 128);
+            const int valid = min(TM, a.P - tile * TM);
+            if (et == 0) {
+                bulk_s2g(a.out + (size_t)tile * TM * a.N, smem_u32(so), (uint32_t)valid * row_out);
+                bulk_commit();
+                ++issued;
+            }
+            if (sactive) {
+#pragma unroll 4
+                for (int r = rh; r < valid; r += rsplit) {
+                    Vec<__nv_bfloat16> zv;
+                    zv.raw = *reinterpret_cast<const uint4*>(so + (size_t)r * row_out + (cu << 4));
+                    float f[8];
+                    zv.unpack(f);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float d = f[i] - piv[i];
+                        s1[i] += d;
+                        s2[i] = fmaf(d, d, s2[i]);
+                    }
+                }
+            }
+        }
+        if (et == 0 && issued > 0) bulk_wait<0>();
+        if (stats) {
+            // combine the rsplit row classes of every column group in fixed order
+            named_bar_sync(1, 128);
+            float* red = reinterpret_cast<float*>(sO);        // [rsplit][2][N]; the staging tiles are free now
+            if (sactive) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    red[(rh * 2 + 0) * a.N + (cu << 3) + i] = s1[i];
+                    red[(rh * 2 + 1) * a.N + (cu << 3) + i] = s2[i];
+                }
+            }
+            named_bar_sync(1, 128);
+            for (int e = et; e < 2 * a.N; e += 128) {
+                float acc = 0.f;
+                for (int k = 0; k < rsplit; ++k) acc += red[k * 2 * a.N + e];
+                a.stat_partial[(size_t)blockIdx.x * 2 * a.N + e] = acc;
+            }
         }
     }
     fence_before_sync();
@@ -665,10 +753,14 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
     const int nkb = (a.K + KB - 1) / KB;
     a.a_bytes = (uint32_t)nkb * TM * 128u;
     a.b_bytes = (uint32_t)nkb * (uint32_t)a.NT * 128u;
+    a.o_bytes = ((uint32_t)TM * (uint32_t)a.N * 2u + 127u) / 128u * 128u;
+    if (a.o_bytes < 8192u) a.o_bytes = 8192u;      // also holds the [128 / (N/8)][2][N] floats of the statistics' block sum
     const size_t budget = 220 * 1024 - 1024;
-    const size_t fixed = 2 * (size_t)a.a_bytes + a.b_bytes;
-    if (fixed >= budget) return false;
     const int tensors = a.need_z ? 2 : 1;
+    // two output staging tiles if that still leaves room for two 64-pixel raw stages
+    a.OS = 2 * (size_t)a.a_bytes + a.b_bytes + 2 * (size_t)a.o_bytes + 2 * (((size_t)64 * a.K * 2 * tensors + 127) / 128 * 128) <= budget ? 2 : 1;
+    const size_t fixed = 2 * (size_t)a.a_bytes + a.b_bytes + (size_t)a.OS * a.o_bytes;
+    if (fixed >= budget) return false;
     for (int rs = 128; rs >= 32; rs >>= 1) {
         size_t rb = ((size_t)rs * a.K * 2 * tensors + 127) / 128 * 128;
         size_t r = (budget - fixed) / rb;
@@ -687,19 +779,24 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
     return false;
 }
 
-template <bool BWD> void launch_pipe(const PipeArgs& a, size_t smem, int kind, double bytes, cudaStream_t st) {
+template <bool BWD> int launch_pipe(PipeArgs& a, size_t smem, int kind, double bytes, size_t partial_floats, cudaStream_t st) {
     static bool attr_set = false;
     static int n_sm = 0;
     if (!attr_set) {
-        cudaFuncSetAttribute(pw_pipe_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+        cudaFuncSetAttribute(pw_pipe_kernel<BWD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
+        cudaFuncSetAttribute(pw_pipe_kernel<BWD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
         attr_set = true;
     }
-    LaunchScope ls(kind, bytes, 2.0 * a.P * a.N * a.K, st);
     int grid = a.tiles < n_sm ? a.tiles : n_sm;
-    launch_pdl(pw_pipe_kernel<BWD>, grid, PIPE_THREADS, smem, st, a);
+    if (a.stat_partial && (size_t)grid * 2 * a.N > partial_floats) a.stat_partial = nullptr;
+    LaunchScope ls(kind, bytes + (a.stat_partial ? 8.0 * a.N * grid : 0.0), 2.0 * a.P * a.N * a.K, st);
+    const bool extra = BWD ? a.addend != nullptr : a.bias != nullptr;
+    if (extra) launch_pdl(pw_pipe_kernel<BWD, true>, grid, PIPE_THREADS, smem, st, a);
+    else launch_pdl(pw_pipe_kernel<BWD, false>, grid, PIPE_THREADS, smem, st, a);
+    return a.stat_partial ? grid : 0;
 }
 
 
@@ -1000,7 +1097,8 @@ bool pw_tc_supported(int dtype, const ConvGeom& g, bool bwd_data) {
     return dtype == 1 && g.k == 1 && g.pad == 0 && g.ci % 8 == 0 && g.co % 8 == 0 && g.ci >= 8 && g.co >= 8;
 }
 
-void pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const float* bias, void* z, int* err, cudaStream_t st) {
+int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const float* bias, void* z, const float* pivot, float* partial,
+              size_t partial_floats, int* err, cudaStream_t st) {
     PwArgs a{};
     a.x = x; a.w = wb; a.bias = bias; a.out = (__nv_bfloat16*)z; a.err = err;
     a.P = g.n * g.ho * g.wo; a.K = g.ci; a.N = g.co;
@@ -1010,14 +1108,16 @@ void pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, cons
         PipeArgs pa{};
         pa.x = x; pa.w = wb; pa.bias = bias; pa.out = (__nv_bfloat16*)z; pa.err = err;
         pa.P = a.P; pa.K = a.K; pa.N = a.N; pa.tiles = (a.P + TM - 1) / TM; pa.need_z = 0;
-        size_t smem = 0;
-        if (plan_pipe(pa, &smem)) {
-            launch_pipe<false>(pa, smem, K_PW_FWD_TC, bytes, st);
-            return;
+        if (pivot && partial) {
+            pa.pivot = pivot;
+            pa.stat_partial = partial;
         }
+        size_t smem = 0;
+        if (plan_pipe(pa, &smem)) return launch_pipe<false>(pa, smem, K_PW_FWD_TC, bytes, partial_floats, st);
     }
     Tiling t = pick_tiling(a.K, a.N);
     launch<false>(a, t, K_PW_FWD_TC, bytes, st);
+    return 0;
 }
 
 void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st) {
@@ -1044,7 +1144,7 @@ void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* w
         pa.P = a.P; pa.K = a.K; pa.N = a.N; pa.tiles = (a.P + TM - 1) / TM; pa.need_z = (dz.act != ACT_NONE || dz.k1) ? 1 : 0;
         size_t smem = 0;
         if (plan_pipe(pa, &smem)) {
-            launch_pipe<true>(pa, smem, K_PW_BWD_DATA_TC, bytes, st);
+            launch_pipe<true>(pa, smem, K_PW_BWD_DATA_TC, bytes, 0, st);
             return;
         }
     }

@@ -359,9 +359,13 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
         const bool is_last = ui + 1 == s->units.size();
         void* obuf = sv.base + o.buf_off;
         tick(s, ui, 0, st);
+        int fused_stats = 0;       // > 0: the producing kernel wrote that many statistics partials into the scratch arena
         if (u.kind == U_CONV) {
             const float* bias = u.b_off >= 0 ? s->w + u.b_off : nullptr;
-            if (pw_tc_supported(dt, u.g, false)) pw_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, bias, obuf, s->err, st);
+            const bool bn = u.l_bn >= 0;
+            if (pw_tc_supported(dt, u.g, false))
+                fused_stats = pw_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, bias, obuf, bn ? s->run + u.run_off : nullptr,
+                                        bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
             else if (conv3_tc_supported(dt, u.g)) conv3_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, obuf, s->err, st);
             else conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, bias, obuf, st);
         } else if (u.kind == U_DW) {
@@ -376,7 +380,10 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
         if (u.l_bn >= 0) {
             float* stt = sv.stats + o.stat_off;
             BnFwdOut bo{stt, stt + o.c, stt + 2 * (size_t)o.c, stt + 3 * (size_t)o.c, s->run + u.run_off, s->run + u.run_off + o.c};
-            bn_stats(dt, obuf, o.elems / o.c, o.c, s->w + u.gamma_off, s->w + u.beta_off, s->eps, s->bn_mom, s->scratch, s->scratch_floats, bo, st);
+            if (fused_stats > 0)
+                bn_stats_finish_partials(s->scratch, fused_stats, o.elems / o.c, o.c, s->w + u.gamma_off, s->w + u.beta_off, s->eps, s->bn_mom, bo, st);
+            else
+                bn_stats(dt, obuf, o.elems / o.c, o.c, s->w + u.gamma_off, s->w + u.beta_off, s->eps, s->bn_mom, s->scratch, s->scratch_floats, bo, st);
         }
         tick(s, ui, 2, st);
         if (is_last) {
