@@ -244,7 +244,7 @@ template <typename T, int V> struct GradRoll {
     }
 };
 
-template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC>
+template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC, bool ADD>
 __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, int c, int th, SRC src, const float* __restrict__ w9c,
                                                       const T* addend, T* out) {
     pdl_wait();
@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
             for (int t = 0; t < TWR; ++t) {
                 if (wo0 + t < w) {
                     size_t e = (((size_t)n * h + orow) * w + wo0 + t) * c + c0;
-                    if (addend) {
+                    if (ADD) {
                         float ad[V];
                         Raw<T, V>::ld(addend, e, ad);
 #pragma unroll
@@ -349,7 +349,8 @@ void launch_roll(int n, int h, int w, int c, const SRC& src, const float* w9c, c
     int th = h >= 28 ? 8 : (h >= 14 ? 7 : h);
     size_t total = (size_t)n * ((h + th - 1) / th) * ((w + TWR - 1) / TWR) * (c / V);
     size_t smem = (size_t)9 * c * sizeof(float);
-    launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC>, (unsigned)((total + 127) / 128), 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
+    if (addend) launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC, true>, (unsigned)((total + 127) / 128), 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
+    else launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC, false>, (unsigned)((total + 127) / 128), 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
 }
 
 
@@ -516,7 +517,9 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
 //   dx[ih][wo0+t]  = sum_{r,s} dz[ih+1-r][wo0+t+1-s] * w[r][s]
 //   gw[r][s]      += sum_t dz[ih+1-r][wo0+t] * x[ih][wo0+t-1+s]
 // The halo columns of dz feed dx only; their weight-gradient terms belong to the neighbouring strip.
-template <typename T, int V, int TWR, int D>
+// ADD: the residual gradient `addend` is added to dx (a template parameter: even never-executed
+// loads in the inner loop cost issue slots).
+template <typename T, int V, int TWR, int D, bool ADD>
 __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, const float* __restrict__ w9c, const T* addend,
                                                            T* dx, int cw, int rows, size_t items_per_block, float* __restrict__ partial) {
     pdl_wait();
@@ -612,7 +615,7 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
                 stage = stage + 1 == D ? 0 : stage + 1;
                 float ad[TWR][V];
                 const size_t orow = (((size_t)n * h + max(ih, 0)) * w + wo0) * c + c0;
-                if (addend && ih >= 0) {
+                if (ADD && ih >= 0) {
 #pragma unroll
                     for (int t = 0; t < TWR; ++t)
                         if (wo0 + t < w) Raw<T, V>::ld(addend, orow + (size_t)t * c, ad[t]);
@@ -645,7 +648,7 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
 #pragma unroll
                     for (int t = 0; t < TWR; ++t) {
                         if (wo0 + t < w) {
-                            if (addend) {
+                            if (ADD) {
 #pragma unroll
                                 for (int q = 0; q < V; ++q) o[t][q] += ad[t][q];
                             }
@@ -691,7 +694,7 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
 // of dz row i+1; columns likewise.  A thread owns V channels and TWZ columns of dz (plus one
 // halo column), walks down the dz rows keeping rows i and i+1, and writes the two input rows
 // 2i, 2i+1 (2*TWZ columns each).  Every dz element is loaded and transformed once per thread.
-template <typename T, int V, int TWZ>
+template <typename T, int V, int TWZ, bool ADD>
 __global__ void __launch_bounds__(128) dw_bwd_data_s2_kernel(ConvGeom g, GradSrc dzs, const float* __restrict__ w9c, int th, const T* addend, T* dx) {
     pdl_wait();
     pdl_launch();
@@ -769,7 +772,7 @@ __global__ void __launch_bounds__(128) dw_bwd_data_s2_kernel(ConvGeom g, GradSrc
                         o[q] = v;
                     }
                     const size_t e = (((size_t)n * H + hi) * W + wi) * c + c0;
-                    if (addend) {
+                    if (ADD) {
                         float ad[V];
                         Raw<T, V>::ld(addend, e, ad);
 #pragma unroll
@@ -969,8 +972,14 @@ void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w
         const int th = nrowz >= 14 ? 7 : nrowz;
         size_t total = (size_t)g.n * ((nrowz + th - 1) / th) * ((ncolz + TWZ - 1) / TWZ) * (g.ci / 4);
         size_t smem = (size_t)9 * g.ci * sizeof(float);
-        if (dtype == 0) launch_pdl(dw_bwd_data_s2_kernel<float, 4, TWZ>, (unsigned)((total + 127) / 128), 128, smem, st, g, dz, w9c, th, (const float*)addend, (float*)dx);
-        else launch_pdl(dw_bwd_data_s2_kernel<B, 4, TWZ>, (unsigned)((total + 127) / 128), 128, smem, st, g, dz, w9c, th, (const B*)addend, (B*)dx);
+        const unsigned blocks = (unsigned)((total + 127) / 128);
+        if (dtype == 0) {
+            if (addend) launch_pdl(dw_bwd_data_s2_kernel<float, 4, TWZ, true>, blocks, 128, smem, st, g, dz, w9c, th, (const float*)addend, (float*)dx);
+            else launch_pdl(dw_bwd_data_s2_kernel<float, 4, TWZ, false>, blocks, 128, smem, st, g, dz, w9c, th, (const float*)addend, (float*)dx);
+        } else {
+            if (addend) launch_pdl(dw_bwd_data_s2_kernel<B, 4, TWZ, true>, blocks, 128, smem, st, g, dz, w9c, th, (const B*)addend, (B*)dx);
+            else launch_pdl(dw_bwd_data_s2_kernel<B, 4, TWZ, false>, blocks, 128, smem, st, g, dz, w9c, th, (const B*)addend, (B*)dx);
+        }
     }
 }
 
@@ -1055,14 +1064,17 @@ bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc&
     const size_t smem = (((size_t)9 * cw * V * 4 + 15) & ~(size_t)15) + (size_t)D * NL * 128 * 8;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaFuncSetAttribute(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        cudaFuncSetAttribute(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        cudaFuncSetAttribute(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
         attr_set = true;
     }
     double e = (double)g.n * g.hi * g.wi * g.ci;
     {
         LaunchScope ls(K_DW_BWD_FUSED, grad_src_bytes(dz, e, dtype) + e * 2.0 * (addend ? 3.0 : 2.0) + 36.0 * g.ci * (by + 1), 36.0 * e, st);
         dim3 grid(gx, (unsigned)by);
-        launch_pdl(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D>, grid, 128, smem, st, g, dz, x, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx, cw,
+        if (addend) launch_pdl(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, true>, grid, 128, smem, st, g, dz, x, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx, cw,
+                                                                            rows, ipb, scratch);
+        else launch_pdl(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, false>, grid, 128, smem, st, g, dz, x, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx, cw,
                                                                             rows, ipb, scratch);
     }
     LaunchScope ls(K_DW_BWD_WEIGHT_FINISH, 36.0 * g.ci * (by + 1), 9.0 * g.ci * by, st);
