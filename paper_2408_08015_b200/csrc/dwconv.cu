@@ -363,6 +363,10 @@ template <typename RAW> __device__ __forceinline__ void cp_async_vec(RAW* dst_sm
     const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst_smem);
     asm volatile("cp.async.ca.shared.global [%0], [%1], %2;" ::"r"(d), "l"(src), "n"((int)sizeof(RAW)) : "memory");
 }
+// same with a 32-bit shared address and a compile-time byte offset (folded into the instruction)
+template <int BYTES, int OFF> __device__ __forceinline__ void cp_async_off(uint32_t dst_smem, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0+%2], [%1], %3;" ::"r"(dst_smem), "l"(src), "n"(OFF), "n"(BYTES) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -542,6 +546,10 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
         wsm[i] = ch < c ? __ldg(w9c + t * c + ch) : 0.f;
     }
     __syncthreads();
+    static_assert(TWR == 2, "the prefetch issue below is written out for four columns");
+    constexpr int RB = (int)sizeof(raw_t), SLOT = 128 * RB;          // bytes of one vector / of one load's slots
+    const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
+    const int wc = w * c;
     const int sw = (w + TWR - 1) / TWR;
     const size_t n_items = (size_t)g.n * sw;
     const size_t ibeg = (size_t)blockIdx.y * items_per_block, iend = min(n_items, ibeg + items_per_block);
@@ -570,17 +578,29 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
                 col[q2] = min(max(wi, 0), w - 1) * c + c0;
             }
             // step ih consumes x row ih and dz row ih+1 (row addresses clamped into the image)
+            const T* px_n = px + (size_t)n * h * wc;
+            const T* pdy_n = pdy + (size_t)n * h * wc;
+            const T* pz_n = pz + (size_t)n * h * wc;
             auto issue = [&](int ih, int stage) {
                 if (ih < h) {
-                    const size_t rbx = ((size_t)n * h + max(ih, 0)) * w * c, rbz = ((size_t)n * h + min(ih + 1, h - 1)) * w * c;
-                    raw_t* slot = ring + (size_t)stage * NL * 128;
-#pragma unroll
-                    for (int q2 = 0; q2 < NIN; ++q2) cp_async_vec(slot + q2 * 128, px + rbx + col[q2]);
-#pragma unroll
-                    for (int q2 = 0; q2 < NIN; ++q2) cp_async_vec(slot + (NIN + q2) * 128, pdy + rbz + col[q2]);
+                    const T* rx = px_n + max(ih, 0) * wc;
+                    const int zoff = min(ih + 1, h - 1) * wc;
+                    const T* rdy = pdy_n + zoff;
+                    const T* rz = pz_n + zoff;
+                    const uint32_t s0 = ring_s + (uint32_t)stage * (uint32_t)(NL * SLOT);
+                    cp_async_off<RB, 0 * SLOT>(s0, rx + col[0]);
+                    cp_async_off<RB, 1 * SLOT>(s0, rx + col[1]);
+                    cp_async_off<RB, 2 * SLOT>(s0, rx + col[2]);
+                    cp_async_off<RB, 3 * SLOT>(s0, rx + col[3]);
+                    cp_async_off<RB, 4 * SLOT>(s0, rdy + col[0]);
+                    cp_async_off<RB, 5 * SLOT>(s0, rdy + col[1]);
+                    cp_async_off<RB, 6 * SLOT>(s0, rdy + col[2]);
+                    cp_async_off<RB, 7 * SLOT>(s0, rdy + col[3]);
                     if (ldz.need_z) {
-#pragma unroll
-                        for (int q2 = 0; q2 < NIN; ++q2) cp_async_vec(slot + (2 * NIN + q2) * 128, pz + rbz + col[q2]);
+                        cp_async_off<RB, 8 * SLOT>(s0, rz + col[0]);
+                        cp_async_off<RB, 9 * SLOT>(s0, rz + col[1]);
+                        cp_async_off<RB, 10 * SLOT>(s0, rz + col[2]);
+                        cp_async_off<RB, 11 * SLOT>(s0, rz + col[3]);
                     }
                 }
                 cp_async_commit();
