@@ -311,11 +311,15 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
 #pragma unroll
             for (int t = 0; t < TWR; ++t)
 #pragma unroll
-                for (int q = 0; q < V; ++q) {
-                    const float xv = xin[t + s][q];
-                    a0[t][q] = fmaf(xv, w2[q], a0[t][q]);      // input row ih is tap row 2 of output row ih-1
-                    a1[t][q] = fmaf(xv, w1[q], a1[t][q]);      // tap row 1 of output row ih
-                    a2[t][q] = fmaf(xv, w0[q], a2[t][q]);      // tap row 0 of output row ih+1
+                for (int q = 0; q < V; q += 2) {               // two channels per packed fp32 fused multiply-add
+                    const float2 xv = make_float2(xin[t + s][q], xin[t + s][q + 1]);
+                    // input row ih is tap row 2 of output row ih-1, tap row 1 of row ih, tap row 0 of row ih+1
+                    const float2 r0 = __ffma2_rn(xv, make_float2(w2[q], w2[q + 1]), make_float2(a0[t][q], a0[t][q + 1]));
+                    const float2 r1 = __ffma2_rn(xv, make_float2(w1[q], w1[q + 1]), make_float2(a1[t][q], a1[t][q + 1]));
+                    const float2 r2 = __ffma2_rn(xv, make_float2(w0[q], w0[q + 1]), make_float2(a2[t][q], a2[t][q + 1]));
+                    a0[t][q] = r0.x; a0[t][q + 1] = r0.y;
+                    a1[t][q] = r1.x; a1[t][q + 1] = r1.y;
+                    a2[t][q] = r2.x; a2[t][q + 1] = r2.y;
                 }
         }
         const int orow = ih - 1;
@@ -475,11 +479,14 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
 #pragma unroll
                     for (int t = 0; t < TWR; ++t)
 #pragma unroll
-                        for (int q = 0; q < V; ++q) {
-                            const float xv = xin[t + s][q];
-                            acc[0 * 3 + s][q] = fmaf(dzp[t][q], xv, acc[0 * 3 + s][q]);
-                            acc[1 * 3 + s][q] = fmaf(dz0[t][q], xv, acc[1 * 3 + s][q]);
-                            acc[2 * 3 + s][q] = fmaf(dzm[t][q], xv, acc[2 * 3 + s][q]);
+                        for (int q = 0; q < V; q += 2) {       // two channels per packed fp32 fused multiply-add
+                            const float2 xv = make_float2(xin[t + s][q], xin[t + s][q + 1]);
+                            const float2 r0 = __ffma2_rn(make_float2(dzp[t][q], dzp[t][q + 1]), xv, make_float2(acc[0 * 3 + s][q], acc[0 * 3 + s][q + 1]));
+                            const float2 r1 = __ffma2_rn(make_float2(dz0[t][q], dz0[t][q + 1]), xv, make_float2(acc[1 * 3 + s][q], acc[1 * 3 + s][q + 1]));
+                            const float2 r2 = __ffma2_rn(make_float2(dzm[t][q], dzm[t][q + 1]), xv, make_float2(acc[2 * 3 + s][q], acc[2 * 3 + s][q + 1]));
+                            acc[0 * 3 + s][q] = r0.x; acc[0 * 3 + s][q + 1] = r0.y;
+                            acc[1 * 3 + s][q] = r1.x; acc[1 * 3 + s][q + 1] = r1.y;
+                            acc[2 * 3 + s][q] = r2.x; acc[2 * 3 + s][q + 1] = r2.y;
                         }
 #pragma unroll
                 for (int t = 0; t < TWR; ++t)
@@ -651,17 +658,27 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
                     *reinterpret_cast<float4*>(w0) = *reinterpret_cast<const float4*>(wl + (0 * 3 + s) * width);
                     *reinterpret_cast<float4*>(w1) = *reinterpret_cast<const float4*>(wl + (1 * 3 + s) * width);
                     *reinterpret_cast<float4*>(w2) = *reinterpret_cast<const float4*>(wl + (2 * 3 + s) * width);
+                    // two channels per instruction (packed fp32 fused multiply-add)
 #pragma unroll
                     for (int t = 0; t < TWR; ++t)
 #pragma unroll
-                        for (int q = 0; q < V; ++q) {
-                            o[t][q] = fmaf(dzp[t + 2 - s][q], w0[q], o[t][q]);
-                            o[t][q] = fmaf(dz0[t + 2 - s][q], w1[q], o[t][q]);
-                            o[t][q] = fmaf(dzm[t + 2 - s][q], w2[q], o[t][q]);
-                            const float xv = xin[t + s][q];
-                            acc[0 * 3 + s][q] = fmaf(dzp[t + 1][q], xv, acc[0 * 3 + s][q]);
-                            acc[1 * 3 + s][q] = fmaf(dz0[t + 1][q], xv, acc[1 * 3 + s][q]);
-                            acc[2 * 3 + s][q] = fmaf(dzm[t + 1][q], xv, acc[2 * 3 + s][q]);
+                        for (int q = 0; q < V; q += 2) {
+                            float2 oo = make_float2(o[t][q], o[t][q + 1]);
+                            oo = __ffma2_rn(make_float2(dzp[t + 2 - s][q], dzp[t + 2 - s][q + 1]), make_float2(w0[q], w0[q + 1]), oo);
+                            oo = __ffma2_rn(make_float2(dz0[t + 2 - s][q], dz0[t + 2 - s][q + 1]), make_float2(w1[q], w1[q + 1]), oo);
+                            oo = __ffma2_rn(make_float2(dzm[t + 2 - s][q], dzm[t + 2 - s][q + 1]), make_float2(w2[q], w2[q + 1]), oo);
+                            o[t][q] = oo.x;
+                            o[t][q + 1] = oo.y;
+                            const float2 xv = make_float2(xin[t + s][q], xin[t + s][q + 1]);
+                            float2 a0 = make_float2(acc[0 * 3 + s][q], acc[0 * 3 + s][q + 1]);
+                            float2 a1 = make_float2(acc[1 * 3 + s][q], acc[1 * 3 + s][q + 1]);
+                            float2 a2 = make_float2(acc[2 * 3 + s][q], acc[2 * 3 + s][q + 1]);
+                            a0 = __ffma2_rn(make_float2(dzp[t + 1][q], dzp[t + 1][q + 1]), xv, a0);
+                            a1 = __ffma2_rn(make_float2(dz0[t + 1][q], dz0[t + 1][q + 1]), xv, a1);
+                            a2 = __ffma2_rn(make_float2(dzm[t + 1][q], dzm[t + 1][q + 1]), xv, a2);
+                            acc[0 * 3 + s][q] = a0.x; acc[0 * 3 + s][q + 1] = a0.y;
+                            acc[1 * 3 + s][q] = a1.x; acc[1 * 3 + s][q + 1] = a1.y;
+                            acc[2 * 3 + s][q] = a2.x; acc[2 * 3 + s][q + 1] = a2.y;
                         }
                 }
                 if (ih >= 0) {
