@@ -63,7 +63,7 @@ struct BwdOp {
 };
 
 template <typename T, int V, typename OP>
-__global__ void __launch_bounds__(256) chan_reduce_kernel(OP op, size_t pixels, int c, int cw, int rows, size_t pix_per_block,
+__global__ void __launch_bounds__(512) chan_reduce_kernel(OP op, size_t pixels, int c, int cw, int rows, size_t pix_per_block,
                                                           float* __restrict__ partial) {
     pdl_wait();
     pdl_launch();
@@ -115,9 +115,9 @@ ReducePlan plan_reduce(int dtype, size_t pixels, int c, int nacc, size_t scratch
     p.V = (c % vmax == 0) ? vmax : 1;
     int cg = c / p.V;
     p.cw = cg < 32 ? cg : 32;
-    p.rows = 256 / p.cw;
+    p.rows = 512 / p.cw;
     p.gx = (cg + p.cw - 1) / p.cw;
-    size_t by = (2 * 148 + p.gx - 1) / p.gx;
+    size_t by = (148 + p.gx - 1) / p.gx;            // one 512-thread block per SM: half the partials of two 256-thread blocks
     size_t max_by = (pixels + (size_t)p.rows * 4 - 1) / ((size_t)p.rows * 4);
     if (by > max_by) by = max_by;
     size_t cap = scratch_floats / ((size_t)nacc * c);
@@ -136,11 +136,11 @@ void launch_reduce(int dtype, const ReducePlan& p, const OP& op, size_t pixels, 
     LaunchScope ls(kind, bytes + 8.0 * c * p.by, 4.0 * pixels * c, st);
     dim3 grid(p.gx, (unsigned)p.by);
     if (dtype == 0) {
-        if (p.V == 1) launch_pdl(chan_reduce_kernel<float, 1, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
-        else launch_pdl(chan_reduce_kernel<float, 4, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        if (p.V == 1) launch_pdl(chan_reduce_kernel<float, 1, OP>, grid, 512, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        else launch_pdl(chan_reduce_kernel<float, 4, OP>, grid, 512, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
     } else {
-        if (p.V == 1) launch_pdl(chan_reduce_kernel<__nv_bfloat16, 1, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
-        else launch_pdl(chan_reduce_kernel<__nv_bfloat16, 8, OP>, grid, 256, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        if (p.V == 1) launch_pdl(chan_reduce_kernel<__nv_bfloat16, 1, OP>, grid, 512, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
+        else launch_pdl(chan_reduce_kernel<__nv_bfloat16, 8, OP>, grid, 512, p.smem, st, op, pixels, c, p.cw, p.rows, p.ppb, partial);
     }
 }
 
