@@ -486,6 +486,12 @@ void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int 
     launch_pdl(bn_bwd_finish, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
 }
 
+void bn_bwd_finish_partials(const float* partial, int blocks, size_t pixels, int c, const float* mean, const float* rstd, const float* gamma,
+                            const BnBwdOut& o, cudaStream_t st) {
+    LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (blocks + 4), 10.0 * c, st);
+    launch_pdl(bn_bwd_finish, (c + 31) / 32, 1024, 0, st, partial, blocks, c, (double)pixels, mean, rstd, gamma, o);
+}
+
 template <typename T, int V> static void ew_add_launch(const ValSrc& a, const ValSrc& b, int act, size_t n, int c, void* out, void* out2, cudaStream_t st) {
     size_t groups = n / V;
     LaunchScope ls(K_EW_ADD, (double)n * sizeof(T) * (1 + (b.p ? 1 : 0) + 1 + (out2 ? 1 : 0)), (double)n, st);

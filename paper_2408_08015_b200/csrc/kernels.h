@@ -50,6 +50,16 @@ uint64_t launches();
 // records `msg` as the calling thread's last error and returns `code`
 int report_error(int code, const char* msg);
 
+// BatchNorm-backward reduction fused into the kernel that writes the gradient dy of a conv->BN->activation unit's
+// output: z is that unit's raw conv output, scale/shift/mean/rstd its forward statistics, act its activation.
+struct BnRed {
+    const void* z;
+    const float *scale, *shift, *mean, *rstd;
+    int act;
+    float* partial;          // [blocks][2][c]
+    size_t partial_floats;
+};
+
 // ---- dense convolution as implicit GEMM (plain FFMA tiles; float and bfloat16 storage) ----
 // z[n,ho,wo,ko] = sum_{r,s,c} x[n,ho*st-pad+r,wo*st-pad+s,c] * w[ko][r][s][c]  (+ bias[ko])
 void conv_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w, const float* bias, void* z, cudaStream_t st);
@@ -67,7 +77,12 @@ bool pw_tc_supported(int dtype, const ConvGeom& g, bool bwd_data);
 // and returns the number of CTAs (for bn_stats_finish_partials); 0 = no partials written, statistics need their own pass.
 int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const float* bias, void* z, const float* pivot, float* partial,
               size_t partial_floats, int* err, cudaStream_t st);
-void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st);
+// With `red` given, the pipelined kernel also writes the BatchNorm-backward partial sums of the gradient it produces,
+// partial[cta][2][ci] = sums over the CTA's pixels of dpre = dx * [pre inside the activation's linear region] and of
+// dpre * xhat (dx as stored, after rounding and after the addend), where pre / xhat come from red->z, the raw output
+// of the unit that produced this conv's input.  Returns the number of CTAs (for bn_bwd_finish_partials); 0 = none written.
+int pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, const BnRed* red, int* err,
+                   cudaStream_t st);
 // gw[co][ci]; per-CTA partial sums in scratch, summed in fixed order by a second kernel
 void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                       cudaStream_t st);
@@ -107,6 +122,10 @@ struct BnBwdOut {
 void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int c, const float* scale, const float* shift, int act,
                    const float* mean, const float* rstd, const float* gamma, float* scratch, size_t scratch_floats,
                    const BnBwdOut& o, cudaStream_t st);
+
+// finishing step alone, for partial sums written by the kernel that produced dy
+void bn_bwd_finish_partials(const float* partial, int blocks, size_t pixels, int c, const float* mean, const float* rstd, const float* gamma,
+                            const BnBwdOut& o, cudaStream_t st);
 
 // ---- elementwise over [pixels][c] ----
 void ew_add(int dtype, const ValSrc& a, const ValSrc& b, int act, size_t pixels, int c, void* out, void* out2, cudaStream_t st);

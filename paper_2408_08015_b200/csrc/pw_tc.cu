@@ -448,6 +448,11 @@ struct PipeArgs {
     int OS;                     // output staging tiles: 1 or 2
     const float* pivot;         // forward, optional: per-channel pivot of the fused BatchNorm statistics
     float* stat_partial;        // [CTAs][2][N]: sums of (z - pivot) and (z - pivot)^2 over the CTA's pixels
+    // backward, optional: BatchNorm-backward sums of the produced gradient (the unit that made this conv's input)
+    const __nv_bfloat16* rz;    // that unit's raw output [P][N]
+    const float *r_scale, *r_shift, *r_mean, *r_rstd;
+    int r_act;
+    float* r_partial;           // [CTAs][2][N]: sums of dpre and dpre * xhat over the CTA's pixels
 };
 
 // EXTRA: the epilogue adds the bias (forward) or the residual gradient (backward); a template
@@ -456,7 +461,8 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     pdl_wait();
     pdl_launch();
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * MAX_RAW + 8];   // raw_full[R], raw_empty[R], a_full[2], a_empty[2], acc_full[2], acc_empty[2]
+    // raw_full[R], raw_empty[R], a_full[2], a_empty[2], acc_full[2], acc_empty[2], zp_full[2], zp_empty[2], so_full[2], so_free[2]
+    __shared__ uint64_t bars[2 * MAX_RAW + 16];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_store;
     volatile int* abort_flag = &abort_store;
@@ -465,6 +471,8 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     uint8_t* sB = base + 2 * (size_t)a.a_bytes;       // resident weights
     uint8_t* sR = sB + a.b_bytes;                     // raw ring
     uint8_t* sO = sR + (size_t)a.R * a.raw_bytes;     // output staging tiles
+    uint8_t* sZ = sO + (size_t)a.OS * a.o_bytes;      // backward sums: two tiles of the producing unit's raw output
+    const bool bred = BWD && a.r_partial != nullptr;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = a.R, RS = a.RS, subs = TM / RS;
     const uint32_t bar0 = smem_u32(&bars[0]);
@@ -474,6 +482,10 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     auto a_empty = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 2 + s); };
     auto acc_full = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 4 + s); };
     auto acc_empty = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 6 + s); };
+    auto zp_full = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 8 + s); };
+    auto zp_empty = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 10 + s); };
+    auto so_full = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 12 + s); };
+    auto so_free = [&](int s) { return bar0 + 8u * (2 * MAX_RAW + 14 + s); };
 
     if (tid == 0) {
         for (int s = 0; s < R; ++s) {
@@ -485,6 +497,10 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             mbar_init(a_empty(s), 1);
             mbar_init(acc_full(s), 1);
             mbar_init(acc_empty(s), 128);
+            mbar_init(zp_full(s), 1);
+            mbar_init(zp_empty(s), PIPE_XF);
+            mbar_init(so_full(s), 1);
+            mbar_init(so_free(s), PIPE_XF);
         }
         abort_store = 0;
     }
@@ -541,6 +557,20 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             // never leave while a bulk copy into this CTA's shared memory may still be in flight
             const int issued = it;
             for (int k = (issued > R ? issued - R : 0); k < issued; ++k) mbar_wait(raw_full(k % R), (uint32_t)((k / R) & 1));
+        } else if (lane == 1 && bred) {
+            // second copy stream (its own thread, so that waiting for a free tile buffer never holds back the raw
+            // ring's prefetch): for every output tile, the matching tile of the producing unit's raw output
+            int zissued = 0;
+            for (int t = 0; t < my_tiles; ++t, ++zissued) {
+                const int tile = blockIdx.x + t * gridDim.x;
+                const int zb = t & 1, zn = t >> 1;
+                if (zn > 0 && !mbar_wait_abortable(zp_empty(zb), (uint32_t)((zn - 1) & 1), abort_flag)) break;
+                const int valid = min(TM, a.P - tile * TM);
+                const uint32_t bytes = (uint32_t)valid * (uint32_t)a.N * 2u;
+                mbar_expect_tx(zp_full(zb), bytes);
+                bulk_g2s(smem_u32(sZ + (size_t)zb * a.o_bytes), a.rz + (size_t)tile * TM * a.N, bytes, zp_full(zb));
+            }
+            for (int k = (zissued > 2 ? zissued - 2 : 0); k < zissued; ++k) mbar_wait(zp_full(k & 1), (uint32_t)((k >> 1) & 1));
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
@@ -575,7 +605,56 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
         XfGrad xg;
         if (BWD) xg.init(a.dz, c0);
         else xv.init(a.x, c0);
-        int it = 0;
+        // Backward sums (optional): the transform warps also take, for every finished output tile, the column sums of
+        // dpre = dx * [pre inside the activation's linear region] and dpre * xhat over the staged (rounded) gradient
+        // tile and the matching tile of the producing unit's raw output; thread (cu, rh) owns four channels and the
+        // rows rh, rh + rsplit, ...  (pre = z*rcs + rch, xhat = z*rrs + rms)
+        const int r_units = a.N >> 2, r_split = PIPE_XF / r_units;
+        const int cu = tix % r_units, rh = tix / r_units;
+        const bool ractive = bred && rh < r_split;
+        float s1[4], s2[4], rcs[4], rch[4], rrs[4], rms[4];
+        const float rlo = a.r_act == ACT_NONE ? -INFINITY : 0.f, rhi = a.r_act == ACT_RELU6 ? 6.f : INFINITY;
+        if (BWD) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                s1[i] = s2[i] = 0.f;
+                rcs[i] = ractive ? __ldg(a.r_scale + cu * 4 + i) : 1.f;
+                rch[i] = ractive ? __ldg(a.r_shift + cu * 4 + i) : 0.f;
+                rrs[i] = ractive ? __ldg(a.r_rstd + cu * 4 + i) : 0.f;
+                rms[i] = ractive ? -__ldg(a.r_mean + cu * 4 + i) * rrs[i] : 0.f;
+            }
+        }
+        auto reduce_tile = [&](int r) -> bool {
+            const int ob = a.OS == 2 ? (r & 1) : 0, zb = r & 1;
+            const bool got = mbar_wait_abortable(so_full(ob), (uint32_t)((r / a.OS) & 1), abort_flag) &&
+                             mbar_wait_abortable(zp_full(zb), (uint32_t)((r >> 1) & 1), abort_flag);
+            if (got && ractive) {
+                const uint32_t row_out = (uint32_t)a.N * 2u;
+                const uint8_t* so = sO + (size_t)ob * a.o_bytes;
+                const uint8_t* sz = sZ + (size_t)zb * a.o_bytes;
+                const int valid = min(TM, a.P - ((int)blockIdx.x + r * (int)gridDim.x) * TM);
+#pragma unroll 4
+                for (int rr = rh; rr < valid; rr += r_split) {
+                    const uint2 dr = *reinterpret_cast<const uint2*>(so + (size_t)rr * row_out + (cu << 3));
+                    const uint2 zr = *reinterpret_cast<const uint2*>(sz + (size_t)rr * row_out + (cu << 3));
+                    const float d[4] = {__uint_as_float(dr.x << 16), __uint_as_float(dr.x & 0xffff0000u), __uint_as_float(dr.y << 16),
+                                        __uint_as_float(dr.y & 0xffff0000u)};
+                    const float z[4] = {__uint_as_float(zr.x << 16), __uint_as_float(zr.x & 0xffff0000u), __uint_as_float(zr.y << 16),
+                                        __uint_as_float(zr.y & 0xffff0000u)};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float pre = fmaf(z[i], rcs[i], rch[i]);
+                        const float dm = (pre > rlo && pre < rhi) ? d[i] : 0.f;
+                        s1[i] += dm;
+                        s2[i] = fmaf(dm, fmaf(z[i], rrs[i], rms[i]), s2[i]);
+                    }
+                }
+            }
+            mbar_arrive(so_free(ob));
+            mbar_arrive(zp_empty(zb));
+            return got;
+        };
+        int it = 0, reduced_tiles = 0;
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
@@ -615,6 +694,31 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             if (!ok) break;
             fence_async_smem();
             mbar_arrive(a_full(st));
+            // one tile behind: the epilogue of tile t-1 ran while this tile was being transformed
+            if (BWD && bred && t > 0) {
+                ok = reduce_tile(t - 1);
+                ++reduced_tiles;
+            }
+        }
+        if (BWD && bred) {
+            if (ok && reduced_tiles < my_tiles) reduce_tile(my_tiles - 1);
+            // combine the r_split row classes of every column group in fixed order (every transform thread gets here,
+            // also after an abort: all waits are bounded); the raw-output tiles are free now
+            named_bar_sync(2, PIPE_XF);
+            float* red = reinterpret_cast<float*>(sZ);        // [r_split][2][N]
+            if (ractive) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    red[(rh * 2 + 0) * a.N + cu * 4 + i] = s1[i];
+                    red[(rh * 2 + 1) * a.N + cu * 4 + i] = s2[i];
+                }
+            }
+            named_bar_sync(2, PIPE_XF);
+            for (int e = tix; e < 2 * a.N; e += PIPE_XF) {
+                float acc = 0.f;
+                for (int k = 0; k < r_split; ++k) acc += red[k * 2 * a.N + e];
+                a.r_partial[(size_t)blockIdx.x * 2 * a.N + e] = acc;
+            }
         }
     } else {
         // ------------------------------------------------------------ epilogue
@@ -646,6 +750,8 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             const int ob = a.OS == 2 ? (t & 1) : 0;
             uint8_t* so = sO + (size_t)ob * a.o_bytes;
             bool ok = mbar_wait_abortable(acc_full(st), (uint32_t)(n & 1), abort_flag);
+            // the transform warps must have finished the backward sums over this staging tile's previous contents
+            if (bred && t >= a.OS) ok = mbar_wait_abortable(so_free(ob), (uint32_t)((t / a.OS - 1) & 1), abort_flag) && ok;
             // the bulk store that last read this staging tile must have finished reading it
             if (et == 0) {
                 if (a.OS == 2) bulk_wait_read<1>();
@@ -699,6 +805,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
                 bulk_s2g(a.out + (size_t)tile * TM * a.N, smem_u32(so), (uint32_t)valid * row_out);
                 bulk_commit();
                 ++issued;
+                if (bred) mbar_arrive(so_full(ob));      // the staged tile is complete (ordered by the named barrier above)
             }
             if (sactive) {
 #pragma unroll 4
@@ -757,9 +864,10 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
     if (a.o_bytes < 8192u) a.o_bytes = 8192u;      // also holds the [128 / (N/8)][2][N] floats of the statistics' block sum
     const size_t budget = 220 * 1024 - 1024;
     const int tensors = a.need_z ? 2 : 1;
+    const size_t zp = a.r_partial ? 2 * (size_t)a.o_bytes : 0;      // two tiles of the raw output the backward sums read
     // two output staging tiles if that still leaves room for two 64-pixel raw stages
-    a.OS = 2 * (size_t)a.a_bytes + a.b_bytes + 2 * (size_t)a.o_bytes + 2 * (((size_t)64 * a.K * 2 * tensors + 127) / 128 * 128) <= budget ? 2 : 1;
-    const size_t fixed = 2 * (size_t)a.a_bytes + a.b_bytes + (size_t)a.OS * a.o_bytes;
+    a.OS = 2 * (size_t)a.a_bytes + a.b_bytes + 2 * (size_t)a.o_bytes + zp + 2 * (((size_t)64 * a.K * 2 * tensors + 127) / 128 * 128) <= budget ? 2 : 1;
+    const size_t fixed = 2 * (size_t)a.a_bytes + a.b_bytes + (size_t)a.OS * a.o_bytes + zp;
     if (fixed >= budget) return false;
     for (int rs = 128; rs >= 32; rs >>= 1) {
         size_t rb = ((size_t)rs * a.K * 2 * tensors + 127) / 128 * 128;
@@ -792,11 +900,13 @@ template <bool BWD> int launch_pipe(PipeArgs& a, size_t smem, int kind, double b
     }
     int grid = a.tiles < n_sm ? a.tiles : n_sm;
     if (a.stat_partial && (size_t)grid * 2 * a.N > partial_floats) a.stat_partial = nullptr;
-    LaunchScope ls(kind, bytes + (a.stat_partial ? 8.0 * a.N * grid : 0.0), 2.0 * a.P * a.N * a.K, st);
+    if (a.r_partial && (size_t)grid * 2 * a.N > partial_floats) a.r_partial = nullptr;
+    const bool fused = BWD ? a.r_partial != nullptr : a.stat_partial != nullptr;
+    LaunchScope ls(kind, bytes + (fused ? 8.0 * a.N * grid : 0.0) + (BWD && fused ? 2.0 * a.P * a.N : 0.0), 2.0 * a.P * a.N * a.K, st);
     const bool extra = BWD ? a.addend != nullptr : a.bias != nullptr;
     if (extra) launch_pdl(pw_pipe_kernel<BWD, true>, grid, PIPE_THREADS, smem, st, a);
     else launch_pdl(pw_pipe_kernel<BWD, false>, grid, PIPE_THREADS, smem, st, a);
-    return a.stat_partial ? grid : 0;
+    return fused ? grid : 0;
 }
 
 
@@ -1120,7 +1230,8 @@ int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const
     return 0;
 }
 
-void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st) {
+int pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, const BnRed* red, int* err,
+                   cudaStream_t st) {
     PwArgs a{};
     a.dz = dz; a.w = wtb; a.addend = addend; a.out = (__nv_bfloat16*)dx; a.err = err;
     a.P = g.n * g.ho * g.wo; a.K = g.co; a.N = g.ci;
@@ -1136,20 +1247,24 @@ void pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* w
         a.addend = dx;
         Tiling t = pick_tiling(a.K, a.N);
         launch<true>(a, t, K_PW_BWD_DATA_TC, bytes + (double)full, st);
-        return;
+        return 0;
     }
-    {
+    for (int with_red = red ? 1 : 0; with_red >= 0; --with_red) {
         PipeArgs pa{};
         pa.dz = dz; pa.w = wtb; pa.addend = addend; pa.out = (__nv_bfloat16*)dx; pa.err = err;
         pa.P = a.P; pa.K = a.K; pa.N = a.N; pa.tiles = (a.P + TM - 1) / TM; pa.need_z = (dz.act != ACT_NONE || dz.k1) ? 1 : 0;
-        size_t smem = 0;
-        if (plan_pipe(pa, &smem)) {
-            launch_pipe<true>(pa, smem, K_PW_BWD_DATA_TC, bytes, 0, st);
-            return;
+        if (with_red) {
+            pa.rz = (const __nv_bfloat16*)red->z;
+            pa.r_scale = red->scale; pa.r_shift = red->shift; pa.r_mean = red->mean; pa.r_rstd = red->rstd;
+            pa.r_act = red->act;
+            pa.r_partial = red->partial;
         }
+        size_t smem = 0;
+        if (plan_pipe(pa, &smem)) return launch_pipe<true>(pa, smem, K_PW_BWD_DATA_TC, bytes, with_red ? red->partial_floats : 0, st);
     }
     Tiling t = pick_tiling(a.K, a.N);
     launch<true>(a, t, K_PW_BWD_DATA_TC, bytes, st);
+    return 0;
 }
 
 void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,

@@ -47,6 +47,8 @@ struct Val {
     size_t stat_off = 0;    // floats into a slot's statistics area: mean, rstd, scale, shift (c each)
     size_t grad_off = 0;    // bytes into the gradient workspace
     int consumers = 0;
+    int first_cons = -1;    // lowest-index consuming unit: the last one to run in the backward pass, so the
+                            // kernel that writes its input gradient writes the value's complete gradient
 };
 
 struct Unit {
@@ -239,8 +241,12 @@ static int build_plan(asteroid_stage* s) {
         } else {
             return fail(AST_ERR_UNSUPPORTED, "layer %d: a BN or activation must directly follow the conv (or add) it belongs to", i);
         }
-        s->vals[u.in].consumers++;
-        if (u.in2 >= 0) s->vals[u.in2].consumers++;
+        for (int vin : {u.in, u.in2}) {
+            if (vin < 0) continue;
+            Val& iv = s->vals[vin];
+            iv.consumers++;
+            if (iv.first_cons < 0) iv.first_cons = (int)s->units.size();
+        }
         s->units.push_back(u);
     }
     for (size_t v = 0; v + 1 < s->vals.size(); ++v)
@@ -400,6 +406,28 @@ struct GradState {
     const void* ptr = nullptr;
 };
 
+// The conv->BN unit whose BatchNorm-backward sums can be taken by the kernel that writes the complete gradient of
+// value `v`: the unit that produced v, or, when v is a plain residual sum, the one operand branch that is used
+// nowhere else (its gradient is the sum's gradient, by alias).  -1: none, or more than one.
+static int bn_reduce_target(const asteroid_stage* s, int v) {
+    const int p = s->vals[v].unit;
+    if (p < 0) return -1;
+    const Unit& pu = s->units[p];
+    if (pu.kind == U_CONV || pu.kind == U_DW) return pu.l_bn >= 0 ? p : -1;
+    if (pu.kind != U_ADD || pu.act != ACT_NONE) return -1;
+    int target = -1, n = 0;
+    for (int o : {pu.in, pu.in2}) {
+        const Val& ov = s->vals[o];
+        if (ov.consumers != 1 || ov.unit < 0) continue;
+        const Unit& q = s->units[ov.unit];
+        if ((q.kind == U_CONV || q.kind == U_DW) && q.l_bn >= 0) {
+            target = ov.unit;
+            ++n;
+        }
+    }
+    return n == 1 ? target : -1;
+}
+
 static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, cudaStream_t st) {
     SlotView sv = slot_view(s, slot);
     const int dt = s->dtype;
@@ -418,6 +446,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
     };
     gs.back().state = G_ALIAS;
     gs.back().ptr = dy;
+    std::vector<char> reduced(s->units.size(), 0);   // BatchNorm-backward sums already taken by the kernel that wrote dy
 
     for (int ui = (int)s->units.size() - 1; ui >= 0; --ui) {
         const Unit& u = s->units[ui];
@@ -436,8 +465,9 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                 d.scale = stt + 2 * (size_t)o.c;
                 d.shift = stt + 3 * (size_t)o.c;
                 BnBwdOut bo{s->g + u.gamma_off, s->g + u.beta_off, kc, kc + o.c, kc + 2 * (size_t)o.c};
-                bn_bwd_reduce(dt, d.dy, d.z, o.elems / o.c, o.c, d.scale, d.shift, u.act, stt, stt + o.c, s->w + u.gamma_off, s->scratch,
-                              s->scratch_floats, bo, st);
+                if (!reduced[ui])
+                    bn_bwd_reduce(dt, d.dy, d.z, o.elems / o.c, o.c, d.scale, d.shift, u.act, stt, stt + o.c, s->w + u.gamma_off, s->scratch,
+                                  s->scratch_floats, bo, st);
                 d.k1 = kc; d.k2 = kc + o.c; d.k3 = kc + 2 * (size_t)o.c;
             }
             if (u.b_off >= 0) {
@@ -466,8 +496,28 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             if (want_in) {
                 GradState& gi = gs[u.in];
                 const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
-                if (u.kind == U_CONV && pw_tc_supported(dt, u.g, true)) pw_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
-                else if (u.kind == U_CONV && conv3_tc_supported(dt, u.g)) conv3_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
+                // this kernel writes the complete gradient of its input value: let it also take the BatchNorm-backward
+                // sums of the unit that gradient belongs to
+                const int tgt = (s->vals[u.in].first_cons == ui && !s->tm.on) ? bn_reduce_target(s, u.in) : -1;
+                if (u.kind == U_CONV && pw_tc_supported(dt, u.g, true)) {
+                    BnRed red{};
+                    if (tgt >= 0) {
+                        const Unit& tu = s->units[tgt];
+                        const Val& tv = s->vals[tu.out];
+                        float* ts = sv.stats + tv.stat_off;
+                        red = BnRed{sv.base + tv.buf_off, ts + 2 * (size_t)tv.c, ts + 3 * (size_t)tv.c, ts, ts + tv.c, tu.act, s->scratch, s->scratch_floats};
+                    }
+                    const int blocks = pw_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), tgt >= 0 ? &red : nullptr, s->err, st);
+                    if (blocks > 0) {
+                        const Unit& tu = s->units[tgt];
+                        const Val& tv = s->vals[tu.out];
+                        float* ts = sv.stats + tv.stat_off;
+                        float* tk = s->coef + tu.k_off;
+                        BnBwdOut tbo{s->g + tu.gamma_off, s->g + tu.beta_off, tk, tk + tv.c, tk + 2 * (size_t)tv.c};
+                        bn_bwd_finish_partials(s->scratch, blocks, tv.elems / tv.c, tv.c, ts, ts + tv.c, s->w + tu.gamma_off, tbo, st);
+                        reduced[tgt] = 1;
+                    }
+                } else if (u.kind == U_CONV && conv3_tc_supported(dt, u.g)) conv3_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
                 else if (u.kind == U_CONV) conv_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 else dw_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 gi.state = G_OWNED;
