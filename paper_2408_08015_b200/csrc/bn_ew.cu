@@ -345,16 +345,20 @@ __global__ void sgd_step_kernel(float* __restrict__ w, float* __restrict__ v, fl
 
 __global__ void refresh_kernel(const float* __restrict__ w, const int32_t* __restrict__ perm, float* __restrict__ d,
                                __nv_bfloat16* __restrict__ wb, __nv_bfloat16* __restrict__ wtb, size_t n) {
+    // This kernel writes the derived weight copies that other kernels stage before their dependency wait, so it
+    // releases its dependents only after its own stores are visible device-wide.
     pdl_wait();
-    pdl_launch();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    float t = w[perm[i]];
-    d[i] = t;
-    if (wb) {
-        wb[i] = __float2bfloat16_rn(w[i]);
-        wtb[i] = __float2bfloat16_rn(t);
+    if (i < n) {
+        float t = w[perm[i]];
+        d[i] = t;
+        if (wb) {
+            wb[i] = __float2bfloat16_rn(w[i]);
+            wtb[i] = __float2bfloat16_rn(t);
+        }
     }
+    __threadfence();
+    pdl_launch();
 }
 
 // ------------------------------------------------------------------ losses

@@ -244,21 +244,31 @@ template <typename T, int V> struct GradRoll {
     }
 };
 
-template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC, bool ADD>
+// STATS (forward): the kernel also writes the BatchNorm statistics partials of its output,
+// stat_partial[block][2][c] = sums of (z - pivot[c]) and (z - pivot[c])^2 over the block's outputs (z as stored, after
+// rounding); the threads of a block that own the same channels are combined in thread order.
+template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC, bool ADD, bool STATS>
 __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, int c, int th, SRC src, const float* __restrict__ w9c,
-                                                      const T* addend, T* out) {
-    pdl_wait();
+                                                      const T* addend, T* out, const float* __restrict__ pivot, float* __restrict__ stat_partial) {
     pdl_launch();
     constexpr int NIN = TWR + 2;
     extern __shared__ float wsm[];            // [9][c], tap order already flipped for the adjoint
+    // the weights are not written by the previous kernel in the stream (only the refresh kernel writes them, and it
+    // releases its dependents after its stores): staging them overlaps that kernel's tail
     for (int i = threadIdx.x; i < 9 * c; i += blockDim.x) {
         int t = i / c, ch = i - t * c;
         wsm[i] = __ldg(w9c + (FLIP ? 8 - t : t) * c + ch);
     }
     __syncthreads();
+    pdl_wait();
     const int cv = c / V, sw = (w + TWR - 1) / TWR, nrc = (h + th - 1) / th;
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (size_t)n_img * nrc * sw * cv) return;
+    const bool in_range = idx < (size_t)n_img * nrc * sw * cv;
+    if (!STATS && !in_range) return;
+    float st1[V], st2[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) st1[q] = st2[q] = 0.f;
+    if (in_range) {
     const int j = (int)(idx % cv);
     size_t sidx = idx / cv;
     const int wo0 = (int)(sidx % sw) * TWR;
@@ -268,6 +278,9 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
     const int c0 = j * V;
     LOADER ld(src, c0);
     typedef typename LOADER::Raw1 Raw1;
+    float piv[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) piv[q] = STATS ? __ldg(pivot + c0 + q) : 0.f;
     float a0[TWR][V], a1[TWR][V];               // partial sums of output rows ih-1 and ih
 #pragma unroll
     for (int t = 0; t < TWR; ++t)
@@ -335,6 +348,14 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
                         for (int q = 0; q < V; ++q) a0[t][q] += ad[q];
                     }
                     Raw<T, V>::st(out, e, a0[t]);
+                    if (STATS) {
+#pragma unroll
+                        for (int q = 0; q < V; ++q) {
+                            const float d = to_f<T>(from_f<T>(a0[t][q])) - piv[q];
+                            st1[q] += d;
+                            st2[q] = fmaf(d, d, st2[q]);
+                        }
+                    }
                 }
             }
         }
@@ -346,15 +367,58 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
                 a1[t][q] = a2[t][q];
             }
     }
+    }
+    if (STATS) {
+        // thread t owns channel vector (first + t) % cv: vector jv is summed over its threads in thread order
+        __syncthreads();                          // the weights in shared memory are no longer needed
+        float* red = wsm;                         // [128][2 * V] (the launcher sizes the buffer for both uses)
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            red[threadIdx.x * 2 * V + q] = st1[q];
+            red[threadIdx.x * 2 * V + V + q] = st2[q];
+        }
+        __syncthreads();
+        const int first = (int)(((size_t)blockIdx.x * blockDim.x) % cv);
+        for (int jv = threadIdx.x; jv < cv; jv += blockDim.x) {
+            float a1s[V], a2s[V];
+#pragma unroll
+            for (int q = 0; q < V; ++q) a1s[q] = a2s[q] = 0.f;
+            for (int t = (jv - first + cv) % cv; t < (int)blockDim.x; t += cv) {
+#pragma unroll
+                for (int q = 0; q < V; ++q) {
+                    a1s[q] += red[t * 2 * V + q];
+                    a2s[q] += red[t * 2 * V + V + q];
+                }
+            }
+            float* dst = stat_partial + (size_t)blockIdx.x * 2 * c + jv * V;
+#pragma unroll
+            for (int q = 0; q < V; ++q) {
+                dst[q] = a1s[q];
+                dst[c + q] = a2s[q];
+            }
+        }
+    }
 }
 
+// Returns the number of blocks that wrote statistics partials (0: none).
 template <typename T, int V, int TWR, bool FLIP, typename LOADER, typename SRC>
-void launch_roll(int n, int h, int w, int c, const SRC& src, const float* w9c, const void* addend, void* out, cudaStream_t st) {
+int launch_roll(int n, int h, int w, int c, const SRC& src, const float* w9c, const void* addend, void* out, cudaStream_t st,
+                const float* pivot = nullptr, float* stat_partial = nullptr, size_t partial_floats = 0) {
     int th = h >= 28 ? 8 : (h >= 14 ? 7 : h);
     size_t total = (size_t)n * ((h + th - 1) / th) * ((w + TWR - 1) / TWR) * (c / V);
     size_t smem = (size_t)9 * c * sizeof(float);
-    if (addend) launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC, true>, (unsigned)((total + 127) / 128), 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
-    else launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC, false>, (unsigned)((total + 127) / 128), 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out);
+    const unsigned blocks = (unsigned)((total + 127) / 128);
+    if (!FLIP && !addend && pivot && stat_partial && (size_t)blocks * 2 * c <= partial_floats) {
+        if (smem < (size_t)128 * 2 * V * sizeof(float)) smem = (size_t)128 * 2 * V * sizeof(float);
+        launch_pdl(dw_roll_kernel<T, V, TWR, false, LOADER, SRC, false, true>, blocks, 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out, pivot,
+                   stat_partial);
+        return (int)blocks;
+    }
+    if (addend) launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC, true, false>, blocks, 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out,
+                           (const float*)nullptr, (float*)nullptr);
+    else launch_pdl(dw_roll_kernel<T, V, TWR, FLIP, LOADER, SRC, false, false>, blocks, 128, smem, st, n, h, w, c, th, src, w9c, (const T*)addend, (T*)out,
+                    (const float*)nullptr, (float*)nullptr);
+    return 0;
 }
 
 
@@ -533,8 +597,7 @@ __global__ void __launch_bounds__(128) dw_wgrad_roll_kernel(ConvGeom g, GradSrc 
 template <typename T, int V, int TWR, int D, bool ADD>
 __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSrc dzs, ValSrc xs, const float* __restrict__ w9c, const T* addend,
                                                            T* dx, int cw, int rows, size_t items_per_block, float* __restrict__ partial) {
-    pdl_wait();
-    pdl_launch();
+    pdl_launch();             // the weights are staged before the dependency wait (see dw_roll_kernel)
     constexpr int NIN = TWR + 2, NL = 3 * NIN;
     typedef typename RawT<T, V>::type raw_t;
     extern __shared__ __align__(16) uint8_t dsm[];
@@ -553,6 +616,7 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
         wsm[i] = ch < c ? __ldg(w9c + t * c + ch) : 0.f;
     }
     __syncthreads();
+    pdl_wait();
     static_assert(TWR == 2, "the prefetch issue below is written out for four columns");
     constexpr int RB = (int)sizeof(raw_t), SLOT = 128 * RB;          // bytes of one vector / of one load's slots
     const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
@@ -733,12 +797,12 @@ __global__ void __launch_bounds__(128, 3) dw_bwd_fused_kernel(ConvGeom g, GradSr
 // 2i, 2i+1 (2*TWZ columns each).  Every dz element is loaded and transformed once per thread.
 template <typename T, int V, int TWZ, bool ADD>
 __global__ void __launch_bounds__(128) dw_bwd_data_s2_kernel(ConvGeom g, GradSrc dzs, const float* __restrict__ w9c, int th, const T* addend, T* dx) {
-    pdl_wait();
-    pdl_launch();
+    pdl_launch();             // the weights are staged before the dependency wait (see dw_roll_kernel)
     extern __shared__ float wsm[];            // [9][c]
     const int c = g.ci, H = g.hi, W = g.wi, Ho = g.ho, Wo = g.wo;
     for (int i = threadIdx.x; i < 9 * c; i += blockDim.x) wsm[i] = __ldg(w9c + i);
     __syncthreads();
+    pdl_wait();
     const int cv = c / V;
     const int nrowz = (H + 1) / 2, ncolz = (W + 1) / 2;              // dz rows / columns that own input rows / columns
     const int swz = (ncolz + TWZ - 1) / TWZ, nrc = (nrowz + th - 1) / th;
@@ -982,17 +1046,19 @@ void launch_strip(int n, int hi, int wi, int ho, int wo, int c, const SRC& src, 
 
 }  // namespace
 
-void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, cudaStream_t st) {
+int dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, const float* pivot, float* partial, size_t partial_floats,
+           cudaStream_t st) {
     double in_e = (double)g.n * g.hi * g.wi * g.ci, out_e = (double)g.n * g.ho * g.wo * g.ci;
     LaunchScope ls(K_DW_FWD, (in_e + out_e) * esz(dtype) + 36.0 * g.ci, 18.0 * out_e, st);
     using B = __nv_bfloat16;
     if (dtype == 0) {
-        if (g.stride == 1) launch_roll<float, 4, 4, false, ValRoll<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st);
-        else launch_strip<float, 4, 2, false, ValLoader<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
+        if (g.stride == 1) return launch_roll<float, 4, 4, false, ValRoll<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st, pivot, partial, partial_floats);
+        launch_strip<float, 4, 2, false, ValLoader<float, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     } else {
-        if (g.stride == 1) launch_roll<B, 4, 4, false, ValRoll<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st);
-        else launch_strip<B, 4, 2, false, ValLoader<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
+        if (g.stride == 1) return launch_roll<B, 4, 4, false, ValRoll<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ci, x, w9c, nullptr, z, st, pivot, partial, partial_floats);
+        launch_strip<B, 4, 2, false, ValLoader<B, 4>, ValSrc>(g.n, g.hi, g.wi, g.ho, g.wo, g.ci, x, w9c, nullptr, z, st);
     }
+    return 0;
 }
 
 void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w9c, const void* addend, void* dx, cudaStream_t st) {

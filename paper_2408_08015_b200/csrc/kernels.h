@@ -97,7 +97,10 @@ void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, 
                          cudaStream_t st);
 
 // ---- depthwise 3x3 (weights tap-major: w9c[r*3+s][c]) ----
-void dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, cudaStream_t st);
+// With `pivot` and `partial` given, the stride-1 kernel also writes the BatchNorm statistics partials of its output
+// (layout and meaning as for pw_fwd_tc) and returns the number of blocks that wrote them; 0 = none.
+int dw_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* w9c, void* z, const float* pivot, float* partial, size_t partial_floats,
+           cudaStream_t st);
 void dw_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* w9c, const void* addend, void* dx, cudaStream_t st);
 // stride-1 bf16 layers with enough image columns: input gradient and weight gradient in one pass; false = not applicable
 bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, const float* w9c, const void* addend, void* dx,

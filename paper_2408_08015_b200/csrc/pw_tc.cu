@@ -458,7 +458,9 @@ struct PipeArgs {
 // EXTRA: the epilogue adds the bias (forward) or the residual gradient (backward); a template
 // parameter because even a never-taken branch around those loads slows the epilogue's inner loop.
 template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const PipeArgs a) {
-    pdl_wait();
+    // Set-up that reads nothing the previous kernel in the stream writes (barriers, tensor memory, the resident
+    // weights: written only by the refresh kernel, which releases its dependents after its stores) runs before
+    // the dependency wait and so overlaps the previous kernel's tail.
     pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     // raw_full[R], raw_empty[R], a_full[2], a_empty[2], acc_full[2], acc_empty[2], zp_full[2], zp_empty[2], so_full[2], so_free[2]
@@ -521,6 +523,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     fence_before_sync();
     __syncthreads();
     fence_after_sync();
+    pdl_wait();
     const uint32_t tmem = tmem_slot;
     const int my_tiles = (a.tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const uint32_t row_bytes = (uint32_t)a.K * 2u;
@@ -937,8 +940,7 @@ struct WgArgs {
 };
 
 __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgArgs a) {
-    pdl_wait();
-    pdl_launch();
+    pdl_launch();             // barrier and tensor-memory set-up overlaps the previous kernel; the wait follows it
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * MAX_RAW + 5];    // raw_full[R], raw_empty[R], op_full[2], op_empty[2], done
     __shared__ uint32_t tmem_slot;
@@ -974,6 +976,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
     fence_before_sync();
     __syncthreads();
     fence_after_sync();
+    pdl_wait();
     const uint32_t tmem = tmem_slot;
     const int pbeg = blockIdx.x * a.pix_per_cta, pend = min(a.P, pbeg + a.pix_per_cta);
     const int stages = (pend - pbeg + WSTAGE - 1) / WSTAGE;

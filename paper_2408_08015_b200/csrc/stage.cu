@@ -358,7 +358,13 @@ static void tick(asteroid_stage* s, size_t unit, int which, cudaStream_t st) {
 static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cudaStream_t st) {
     SlotView sv = slot_view(s, slot);
     const int dt = s->dtype;
-    CU(cudaMemcpyAsync(sv.base + s->vals[0].buf_off, x, s->vals[0].elems * s->esz, cudaMemcpyDeviceToDevice, st));
+    {
+        // the slot's copy of x (backward reads it); a kernel rather than a memcpy node where the channel count allows
+        // vector accesses, so that the chain of programmatic dependent launches is not interrupted
+        const Val& v0 = s->vals[0];
+        if (v0.c % (dt == AST_F32 ? 4 : 8) == 0) ew_apply(dt, ValSrc{x, nullptr, nullptr, ACT_NONE}, v0.elems / v0.c, v0.c, sv.base + v0.buf_off, st);
+        else CU(cudaMemcpyAsync(sv.base + v0.buf_off, x, v0.elems * s->esz, cudaMemcpyDeviceToDevice, st));
+    }
     for (size_t ui = 0; ui < s->units.size(); ++ui) {
         const Unit& u = s->units[ui];
         const Val& o = s->vals[u.out];
@@ -375,7 +381,9 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
             else if (conv3_tc_supported(dt, u.g)) conv3_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, obuf, s->err, st);
             else conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, bias, obuf, st);
         } else if (u.kind == U_DW) {
-            dw_fwd(dt, u.g, val_src(s, sv, u.in), s->derived + u.w_off, obuf, st);
+            const bool bn = u.l_bn >= 0;
+            fused_stats = dw_fwd(dt, u.g, val_src(s, sv, u.in), s->derived + u.w_off, obuf, bn ? s->run + u.run_off : nullptr, bn ? s->scratch : nullptr,
+                                 s->scratch_floats, st);
         } else if (u.kind == U_ADD) {
             ew_add(dt, val_src(s, sv, u.in), val_src(s, sv, u.in2), u.act, o.elems / o.c, o.c, obuf, is_last ? y : nullptr, st);
         } else {
