@@ -120,8 +120,11 @@ int asteroid_stage_export_bn_running(asteroid_stage* s, float* mean, float* var,
  * micro-batches already resident). */
 int asteroid_stage_forward(asteroid_stage* s, int mb, const void* x, void* y, void* stream);
 /* BP of micro-batch `mb`: reads dy = dL/dy, writes dx = dL/dx (ignored when need_input_grad==0) and the
- * parameter gradients g_mb of this micro-batch, then releases the slot.  Errors: AST_ERR_ORDER
- * (no resident FP of mb, or the previous g not yet accumulated). */
+ * parameter gradients g_mb of this micro-batch, then releases the slot.  The weight-gradient kernels,
+ * on which nothing else in the pass depends, run on a stream the stage owns, forked from `stream`
+ * after the coefficients they need and joined back into `stream` before the call returns: in
+ * `stream` order the call is complete like any other.  Errors: AST_ERR_ORDER (no resident FP of mb,
+ * or the previous g not yet accumulated). */
 int asteroid_stage_backward(asteroid_stage* s, int mb, const void* dy, void* dx, void* stream);
 /* G += g_mb: accumulate the gradients of the micro-batch whose BP ran last (Section 3.2: each device
  * accumulates gradients for all micro-batches of the mini-batch).  AST_ERR_ORDER if mb is not that one. */
@@ -163,8 +166,9 @@ int asteroid_loss_softmax_xent(const void* logits, const int32_t* labels, int ro
  * stream; stop synchronises the device and returns, per kernel kind that ran, the number of
  * launches, the summed device time, the summed algorithmic bytes (each tensor the kernel must
  * read or write, once) and floating-point operations.  At most `capacity` records are written,
- * *n_out receives the count.  Tracing adds two event records per launch: do not time throughput
- * while it is on. */
+ * *n_out receives the count.  Tracing adds two event records per launch and keeps every kernel on the
+ * caller's stream (no overlap with the stage's second stream), so that a recorded duration is that of
+ * the kernel running alone: do not time throughput while it is on. */
 typedef struct {
     char name[48];
     uint64_t launches;

@@ -47,6 +47,8 @@ struct LaunchScope {
     cudaStream_t st;
 };
 uint64_t launches();
+// true while a per-launch event trace is being recorded
+bool tracing();
 // records `msg` as the calling thread's last error and returns `code`
 int report_error(int code, const char* msg);
 

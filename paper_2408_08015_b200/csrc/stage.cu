@@ -85,6 +85,12 @@ struct asteroid_stage {
     int32_t* perm = nullptr;
     __nv_bfloat16 *wb = nullptr, *wtb = nullptr;   // bf16 copies of the weights and of the derived (transposed) weights
     int* err = nullptr;                            // device error word (bounded waits)
+    // Weight-gradient kernels depend only on the BatchNorm-backward coefficients of their unit and nothing in the rest of
+    // the backward pass depends on them: they run on a second stream (forked from and joined back into the caller's
+    // stream inside each backward call), with their own split-sum scratch, and fill the gaps of the dependent chain.
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    float* scratch_side = nullptr;
     char *slot_mem = nullptr, *grad_mem = nullptr;
     size_t slot_bytes = 0, slot_stat_off = 0, grad_bytes = 0, scratch_floats = 0;
     size_t bytes_mod = 0, bytes_opt = 0, bytes_work = 0;
@@ -303,7 +309,10 @@ static void free_stage(asteroid_stage* s) {
     for (auto e : s->tm.ev) cudaEventDestroy(e);
     cudaFree(s->w); cudaFree(s->v); cudaFree(s->G); cudaFree(s->g); cudaFree(s->derived); cudaFree(s->run);
     cudaFree(s->coef); cudaFree(s->scratch); cudaFree(s->perm); cudaFree(s->slot_mem); cudaFree(s->grad_mem);
-    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err);
+    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err); cudaFree(s->scratch_side);
+    if (s->ev_fork) cudaEventDestroy(s->ev_fork);
+    if (s->ev_join) cudaEventDestroy(s->ev_join);
+    if (s->side) cudaStreamDestroy(s->side);
     delete s;
 }
 
@@ -455,6 +464,20 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
     gs.back().state = G_ALIAS;
     gs.back().ptr = dy;
     std::vector<char> reduced(s->units.size(), 0);   // BatchNorm-backward sums already taken by the kernel that wrote dy
+    // weight gradients go to the second stream (not while a profile run times the units one by one, nor while a
+    // per-launch trace brackets every kernel with events: a kernel's duration is then that of the kernel running alone)
+    const bool use_side = s->side != nullptr && !s->tm.on && !tracing();
+    bool side_used = false;
+    cudaStream_t wst = use_side ? s->side : st;
+    float* wscratch = use_side ? s->scratch_side : s->scratch;
+    // everything enqueued on the caller's stream so far (the coefficients of the unit at hand) precedes what follows on the second
+    auto fork = [&]() -> int {
+        if (!use_side) return AST_OK;
+        CU(cudaEventRecord(s->ev_fork, st));
+        CU(cudaStreamWaitEvent(s->side, s->ev_fork, 0));
+        side_used = true;
+        return AST_OK;
+    };
 
     for (int ui = (int)s->units.size() - 1; ui >= 0; --ui) {
         const Unit& u = s->units[ui];
@@ -495,12 +518,16 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                     continue;
                 }
             }
+            {
+                int frc = fork();
+                if (frc) return frc;
+            }
             if (u.kind == U_CONV && pw_tc_supported(dt, u.g, false))
-                pw_bwd_weight_tc(u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, s->err, st);
+                pw_bwd_weight_tc(u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst);
             else if (u.kind == U_CONV && conv3_wgrad_tc_supported(dt, u.g))
-                conv3_bwd_weight_tc(u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, s->err, st);
-            else if (u.kind == U_CONV) conv_bwd_weight(dt, u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, st);
-            else dw_bwd_weight(dt, u.g, d, xin, s->scratch, s->scratch_floats, s->g + u.w_off, st);
+                conv3_bwd_weight_tc(u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst);
+            else if (u.kind == U_CONV) conv_bwd_weight(dt, u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, wst);
+            else dw_bwd_weight(dt, u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, wst);
             if (want_in) {
                 GradState& gi = gs[u.in];
                 const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
@@ -555,6 +582,10 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
     }
     if (s->need_dx && gs[0].state == G_ALIAS)
         CU(cudaMemcpyAsync(dx, gs[0].ptr, s->vals[0].elems * s->esz, cudaMemcpyDeviceToDevice, st));
+    if (side_used) {            // join: the call's work is complete, in the caller's stream order, when the second stream's is
+        CU(cudaEventRecord(s->ev_join, s->side));
+        CU(cudaStreamWaitEvent(st, s->ev_join, 0));
+    }
     CU(cudaGetLastError());
     return AST_OK;
 }
@@ -595,6 +626,10 @@ static int create_impl(const ast_layer* net, int n_layers, int first, int last, 
     for (const auto& u : s->units)
         if (u.kind == U_CONV) s->scratch_floats = std::max(s->scratch_floats, (size_t)4 * u.g.co * u.g.k * u.g.k * u.g.ci);
     if ((rc = dev_alloc(&s->scratch, s->scratch_floats * 4, &work))) return rc;
+    if ((rc = dev_alloc(&s->scratch_side, s->scratch_floats * 4, &work))) return rc;
+    CU(cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking));
+    CU(cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming));
+    CU(cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming));
     s->bytes_mod = mod; s->bytes_opt = opt; s->bytes_work = work;
     std::vector<int32_t> perm;
     fill_perm(s, perm);

@@ -40,6 +40,7 @@ const char* const kNames[K_KINDS] = {
 
 const char* kernel_name(int kind) { return (kind >= 0 && kind < K_KINDS) ? kNames[kind] : "?"; }
 uint64_t launches() { return g_launches; }
+bool tracing() { return g_tracing; }
 
 LaunchScope::LaunchScope(int kind, double alg_bytes, double flops, cudaStream_t s) : slot(-1), st(s) {
     std::lock_guard<std::mutex> lk(g_mu);
