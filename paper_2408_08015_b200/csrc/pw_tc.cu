@@ -475,6 +475,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     uint8_t* sO = sR + (size_t)a.R * a.raw_bytes;     // output staging tiles
     uint8_t* sZ = sO + (size_t)a.OS * a.o_bytes;      // backward sums: two tiles of the producing unit's raw output
     const bool bred = BWD && a.r_partial != nullptr;
+    const bool csum = bred || (!BWD && a.stat_partial != nullptr);   // the transform warps take column sums of every output tile
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = a.R, RS = a.RS, subs = TM / RS;
     const uint32_t bar0 = smem_u32(&bars[0]);
@@ -608,29 +609,32 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
         XfGrad xg;
         if (BWD) xg.init(a.dz, c0);
         else xv.init(a.x, c0);
-        // Backward sums (optional): the transform warps also take, for every finished output tile, the column sums of
-        // dpre = dx * [pre inside the activation's linear region] and dpre * xhat over the staged (rounded) gradient
-        // tile and the matching tile of the producing unit's raw output; thread (cu, rh) owns four channels and the
-        // rows rh, rh + rsplit, ...  (pre = z*rcs + rch, xhat = z*rrs + rms)
+        // Column sums (optional): the transform warps also take, for every finished output tile, per-channel sums down the
+        // staged (rounded) tile; thread (cu, rh) owns four channels and the rows rh, rh + r_split, ...
+        //   forward:  sums of (z - pivot) and (z - pivot)^2, the BatchNorm statistics partials of the output;
+        //   backward: sums of dpre = dx * [pre inside the activation's linear region] and dpre * xhat, with pre = z*rcs + rch
+        //             and xhat = z*rrs + rms taken from the matching tile of the producing unit's raw output z.
         const int r_units = a.N >> 2, r_split = PIPE_XF / r_units;
         const int cu = tix % r_units, rh = tix / r_units;
-        const bool ractive = bred && rh < r_split;
-        float s1[4], s2[4], rcs[4], rch[4], rrs[4], rms[4];
+        const bool ractive = csum && rh < r_split;
+        float s1[4], s2[4], rcs[4], rch[4], rrs[4], rms[4];     // forward: rcs holds the pivot
         const float rlo = a.r_act == ACT_NONE ? -INFINITY : 0.f, rhi = a.r_act == ACT_RELU6 ? 6.f : INFINITY;
-        if (BWD) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                s1[i] = s2[i] = 0.f;
+        for (int i = 0; i < 4; ++i) {
+            s1[i] = s2[i] = 0.f;
+            if (BWD) {
                 rcs[i] = ractive ? __ldg(a.r_scale + cu * 4 + i) : 1.f;
                 rch[i] = ractive ? __ldg(a.r_shift + cu * 4 + i) : 0.f;
                 rrs[i] = ractive ? __ldg(a.r_rstd + cu * 4 + i) : 0.f;
                 rms[i] = ractive ? -__ldg(a.r_mean + cu * 4 + i) * rrs[i] : 0.f;
+            } else {
+                rcs[i] = ractive ? __ldg(a.pivot + cu * 4 + i) : 0.f;
             }
         }
         auto reduce_tile = [&](int r) -> bool {
             const int ob = a.OS == 2 ? (r & 1) : 0, zb = r & 1;
-            const bool got = mbar_wait_abortable(so_full(ob), (uint32_t)((r / a.OS) & 1), abort_flag) &&
-                             mbar_wait_abortable(zp_full(zb), (uint32_t)((r >> 1) & 1), abort_flag);
+            bool got = mbar_wait_abortable(so_full(ob), (uint32_t)((r / a.OS) & 1), abort_flag);
+            if (BWD) got = got && mbar_wait_abortable(zp_full(zb), (uint32_t)((r >> 1) & 1), abort_flag);
             if (got && ractive) {
                 const uint32_t row_out = (uint32_t)a.N * 2u;
                 const uint8_t* so = sO + (size_t)ob * a.o_bytes;
@@ -639,22 +643,31 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
 #pragma unroll 4
                 for (int rr = rh; rr < valid; rr += r_split) {
                     const uint2 dr = *reinterpret_cast<const uint2*>(so + (size_t)rr * row_out + (cu << 3));
-                    const uint2 zr = *reinterpret_cast<const uint2*>(sz + (size_t)rr * row_out + (cu << 3));
                     const float d[4] = {__uint_as_float(dr.x << 16), __uint_as_float(dr.x & 0xffff0000u), __uint_as_float(dr.y << 16),
                                         __uint_as_float(dr.y & 0xffff0000u)};
-                    const float z[4] = {__uint_as_float(zr.x << 16), __uint_as_float(zr.x & 0xffff0000u), __uint_as_float(zr.y << 16),
-                                        __uint_as_float(zr.y & 0xffff0000u)};
+                    if (BWD) {
+                        const uint2 zr = *reinterpret_cast<const uint2*>(sz + (size_t)rr * row_out + (cu << 3));
+                        const float z[4] = {__uint_as_float(zr.x << 16), __uint_as_float(zr.x & 0xffff0000u), __uint_as_float(zr.y << 16),
+                                            __uint_as_float(zr.y & 0xffff0000u)};
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float pre = fmaf(z[i], rcs[i], rch[i]);
-                        const float dm = (pre > rlo && pre < rhi) ? d[i] : 0.f;
-                        s1[i] += dm;
-                        s2[i] = fmaf(dm, fmaf(z[i], rrs[i], rms[i]), s2[i]);
+                        for (int i = 0; i < 4; ++i) {
+                            const float pre = fmaf(z[i], rcs[i], rch[i]);
+                            const float dm = (pre > rlo && pre < rhi) ? d[i] : 0.f;
+                            s1[i] += dm;
+                            s2[i] = fmaf(dm, fmaf(z[i], rrs[i], rms[i]), s2[i]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float dd = d[i] - rcs[i];
+                            s1[i] += dd;
+                            s2[i] = fmaf(dd, dd, s2[i]);
+                        }
                     }
                 }
             }
             mbar_arrive(so_free(ob));
-            mbar_arrive(zp_empty(zb));
+            if (BWD) mbar_arrive(zp_empty(zb));
             return got;
         };
         int it = 0, reduced_tiles = 0;
@@ -697,18 +710,23 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             if (!ok) break;
             fence_async_smem();
             mbar_arrive(a_full(st));
-            // one tile behind: the epilogue of tile t-1 ran while this tile was being transformed
-            if (BWD && bred && t > 0) {
-                ok = reduce_tile(t - 1);
+            // as many tiles behind as there are staging tiles: by then that tile's MMA and epilogue have had the time of
+            // a whole transform + sum step, and the staging tile it occupies is the next one the epilogue needs back
+            if (csum && t >= a.OS) {
+                ok = reduce_tile(reduced_tiles);
                 ++reduced_tiles;
             }
         }
-        if (BWD && bred) {
-            if (ok && reduced_tiles < my_tiles) reduce_tile(my_tiles - 1);
+        if (csum) {
+            while (ok && reduced_tiles < my_tiles) {
+                ok = reduce_tile(reduced_tiles);
+                ++reduced_tiles;
+            }
             // combine the r_split row classes of every column group in fixed order (every transform thread gets here,
-            // also after an abort: all waits are bounded); the raw-output tiles are free now
+            // also after an abort: all waits are bounded); the operand stages are free now: the last tile's sums were
+            // taken after its epilogue, hence after its MMAs
             named_bar_sync(2, PIPE_XF);
-            float* red = reinterpret_cast<float*>(sZ);        // [r_split][2][N]
+            float* red = reinterpret_cast<float*>(sA);        // [r_split][2][N]
             if (ractive) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -720,7 +738,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             for (int e = tix; e < 2 * a.N; e += PIPE_XF) {
                 float acc = 0.f;
                 for (int k = 0; k < r_split; ++k) acc += red[k * 2 * a.N + e];
-                a.r_partial[(size_t)blockIdx.x * 2 * a.N + e] = acc;
+                (BWD ? a.r_partial : a.stat_partial)[(size_t)blockIdx.x * 2 * a.N + e] = acc;
             }
         }
     } else {
@@ -728,24 +746,10 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
         // The 128 epilogue threads (one accumulator row each) round the tile to bf16 into a
         // shared-memory staging tile laid out exactly like the output rows in global memory, which
         // are one contiguous byte range; one thread then stores the tile with a single bulk copy.
-        // Forward with statistics: the same threads then sum (z - pivot) and (z - pivot)^2 down the
-        // columns of the staged (rounded) tile, eight channels per thread, accumulating over the
-        // CTA's tiles in registers.
         const int q = warp & 3;                            // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
         const int et = tid - (PIPE_THREADS - 128);
         const uint32_t row_out = (uint32_t)a.N * 2u;
-        const bool stats = !BWD && a.stat_partial != nullptr;
-        const int units = a.N >> 3;                        // 8-channel column groups
-        const int rsplit = 128 / units;                    // threads per column group (N <= 256: at least 4)
-        const int cu = et % units, rh = et / units;
-        const bool sactive = stats && rh < rsplit;
-        float s1[8], s2[8], piv[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            s1[i] = s2[i] = 0.f;
-            piv[i] = sactive ? __ldg(a.pivot + (cu << 3) + i) : 0.f;
-        }
         int issued = 0;
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
@@ -753,8 +757,8 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             const int ob = a.OS == 2 ? (t & 1) : 0;
             uint8_t* so = sO + (size_t)ob * a.o_bytes;
             bool ok = mbar_wait_abortable(acc_full(st), (uint32_t)(n & 1), abort_flag);
-            // the transform warps must have finished the backward sums over this staging tile's previous contents
-            if (bred && t >= a.OS) ok = mbar_wait_abortable(so_free(ob), (uint32_t)((t / a.OS - 1) & 1), abort_flag) && ok;
+            // the transform warps must have finished the column sums over this staging tile's previous contents
+            if (csum && t >= a.OS) ok = mbar_wait_abortable(so_free(ob), (uint32_t)((t / a.OS - 1) & 1), abort_flag) && ok;
             // the bulk store that last read this staging tile must have finished reading it
             if (et == 0) {
                 if (a.OS == 2) bulk_wait_read<1>();
@@ -808,43 +812,10 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
                 bulk_s2g(a.out + (size_t)tile * TM * a.N, smem_u32(so), (uint32_t)valid * row_out);
                 bulk_commit();
                 ++issued;
-                if (bred) mbar_arrive(so_full(ob));      // the staged tile is complete (ordered by the named barrier above)
-            }
-            if (sactive) {
-#pragma unroll 4
-                for (int r = rh; r < valid; r += rsplit) {
-                    Vec<__nv_bfloat16> zv;
-                    zv.raw = *reinterpret_cast<const uint4*>(so + (size_t)r * row_out + (cu << 4));
-                    float f[8];
-                    zv.unpack(f);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float d = f[i] - piv[i];
-                        s1[i] += d;
-                        s2[i] = fmaf(d, d, s2[i]);
-                    }
-                }
+                if (csum) mbar_arrive(so_full(ob));      // the staged tile is complete (ordered by the named barrier above)
             }
         }
         if (et == 0 && issued > 0) bulk_wait<0>();
-        if (stats) {
-            // combine the rsplit row classes of every column group in fixed order
-            named_bar_sync(1, 128);
-            float* red = reinterpret_cast<float*>(sO);        // [rsplit][2][N]; the staging tiles are free now
-            if (sactive) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    red[(rh * 2 + 0) * a.N + (cu << 3) + i] = s1[i];
-                    red[(rh * 2 + 1) * a.N + (cu << 3) + i] = s2[i];
-                }
-            }
-            named_bar_sync(1, 128);
-            for (int e = et; e < 2 * a.N; e += 128) {
-                float acc = 0.f;
-                for (int k = 0; k < rsplit; ++k) acc += red[k * 2 * a.N + e];
-                a.stat_partial[(size_t)blockIdx.x * 2 * a.N + e] = acc;
-            }
-        }
     }
     fence_before_sync();
     __syncthreads();
