@@ -153,19 +153,19 @@ __device__ __forceinline__ bool sum_partials(const float* __restrict__ partial, 
     ch = blockIdx.x * 32 + cl;
     double a1 = 0.0, a2 = 0.0;
     if (ch < c) {
-        // eight partials per round are loaded before any is added: the loads overlap, the order of
+        // sixteen partials per round are loaded before any is added: the loads overlap, the order of
         // the additions stays fixed
-        for (int b0 = bg; b0 < blocks; b0 += 32 * 8) {
-            float v1[8], v2[8];
+        for (int b0 = bg; b0 < blocks; b0 += 32 * 16) {
+            float v1[16], v2[16];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 const int b = b0 + 32 * u;
                 const bool ok = b < blocks;
                 v1[u] = ok ? partial[((size_t)b * 2 + 0) * c + ch] : 0.f;
                 v2[u] = ok ? partial[((size_t)b * 2 + 1) * c + ch] : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 a1 += v1[u];
                 a2 += v2[u];
             }
