@@ -195,6 +195,81 @@ __global__ void reduce_splits_kernel(const float* __restrict__ partial, int spli
     out[i] = s;
 }
 
+// ---- small-c_in dense convs (the 3-channel stem) as an explicit im2col + pointwise tensor-core GEMM ----
+// col[p][kk] = x value feeding output pixel p through tap kk = (r, s, c) (the weight layout's order), zero in the
+// padding and for kk >= K; rows are Kp bf16 values (Kp a multiple of 8, at most 64).  One thread writes one pixel's
+// row; the decomposition of kk (tap row, tap column, channel, offset from the pixel's first input element) comes from
+// a table in shared memory, so that the per-element work is a lookup, two bit tests and a load.
+__global__ void __launch_bounds__(256) im2col_kernel(ConvGeom g, ValSrc x, int K, int Kp, __nv_bfloat16* __restrict__ col, size_t pixels) {
+    pdl_launch();
+    __shared__ int t_off[64];
+    __shared__ unsigned char t_r[64], t_s[64], t_c[64];
+    for (int kk = threadIdx.x; kk < Kp; kk += blockDim.x) {
+        int c = 0, r = 31, s2 = 31, off = 0;         // kk >= K: a tap position no mask has
+        if (kk < K) {
+            c = kk % g.ci;
+            const int rs = kk / g.ci;
+            s2 = rs % g.k;
+            r = rs / g.k;
+            off = (r * g.wi + s2) * g.ci + c;
+        }
+        t_off[kk] = off; t_r[kk] = (unsigned char)r; t_s[kk] = (unsigned char)s2; t_c[kk] = (unsigned char)c;
+    }
+    __syncthreads();
+    pdl_wait();
+    const size_t p = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= pixels) return;
+    const int wo = (int)(p % g.wo);
+    const size_t t = p / g.wo;
+    const int ho = (int)(t % g.ho), n = (int)(t / g.ho);
+    const int h0 = ho * g.stride - g.pad, w0 = wo * g.stride - g.pad;
+    unsigned rmask = 0, smask = 0;                   // taps whose input row / column lies inside the image
+    for (int q = 0; q < g.k; ++q) {
+        rmask |= (h0 + q >= 0 && h0 + q < g.hi) ? (1u << q) : 0u;
+        smask |= (w0 + q >= 0 && w0 + q < g.wi) ? (1u << q) : 0u;
+    }
+    const long long base = ((long long)(n * g.hi + h0) * g.wi + w0) * g.ci;
+    uint4* dst = reinterpret_cast<uint4*>(col + p * (size_t)Kp);
+    for (int j = 0; j < (Kp >> 3); ++j) {
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float v2[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int kk = (j << 3) + 2 * q + e;
+                const bool ok = ((rmask >> t_r[kk]) & (smask >> t_s[kk]) & 1u) != 0;
+                v2[e] = ok ? ld_val<__nv_bfloat16>(x, (size_t)(base + t_off[kk]), t_c[kk]) : 0.f;
+            }
+            __nv_bfloat162 h = __floats2bfloat162_rn(v2[0], v2[1]);
+            w[q] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+// wpad[ko][kk] = bf16(w[ko][kk]) for kk < K, zero up to Kp
+__global__ void pad_weights_kernel(const float* __restrict__ w, int co, int K, int Kp, __nv_bfloat16* __restrict__ wpad) {
+    pdl_wait();
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < co * Kp) {
+        const int ko = i / Kp, kk = i - ko * Kp;
+        wpad[i] = __float2bfloat16_rn(kk < K ? w[(size_t)ko * K + kk] : 0.f);
+    }
+    __threadfence();          // other kernels stage these weights before their dependency wait
+    pdl_launch();
+}
+
+// gw[ko][kk] = gpad[ko][kk], kk < K
+__global__ void unpad_grad_kernel(const float* __restrict__ gpad, int co, int K, int Kp, float* __restrict__ gw) {
+    pdl_wait();
+    pdl_launch();
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= co * K) return;
+    const int ko = i / K, kk = i - ko * K;
+    gw[i] = gpad[(size_t)ko * Kp + kk];
+}
+
 template <int MODE> void launch(int dtype, const IgemmArgs& a, dim3 grid, int kind, double bytes, cudaStream_t st) {
     LaunchScope ls(kind, bytes, 2.0 * a.M * a.N * a.K, st);
     if (dtype == 0)
@@ -247,6 +322,23 @@ void conv_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValS
     launch<MODE_BWD_WEIGHT>(dtype, a, dim3((a.M + BM - 1) / BM, (a.N + BN - 1) / BN, splits), K_CONV_BWD_WEIGHT, bytes, st);
     LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (splits + 1), (double)out_elems * splits, st);
     launch_pdl(reduce_splits_kernel, (unsigned)((out_elems + 255) / 256), 256, 0, st, scratch, splits, out_elems, gw);
+}
+
+void conv_im2col(const ConvGeom& g, const ValSrc& x, int Kp, void* col, cudaStream_t st) {
+    const int K = g.k * g.k * g.ci;
+    const size_t pixels = (size_t)g.n * g.ho * g.wo;
+    LaunchScope ls(K_IM2COL, 2.0 * ((double)g.n * g.hi * g.wi * g.ci + (double)pixels * Kp), 0.0, st);
+    launch_pdl(im2col_kernel, (unsigned)((pixels + 255) / 256), 256, 0, st, g, x, K, Kp, (__nv_bfloat16*)col, pixels);
+}
+
+void conv_pad_weights(const float* w, int co, int K, int Kp, __nv_bfloat16* wpad, cudaStream_t st) {
+    LaunchScope ls(K_COL_AUX, 4.0 * co * K + 2.0 * co * Kp, 0.0, st);
+    launch_pdl(pad_weights_kernel, (co * Kp + 255) / 256, 256, 0, st, w, co, K, Kp, wpad);
+}
+
+void conv_unpad_grad(const float* gpad, int co, int K, int Kp, float* gw, cudaStream_t st) {
+    LaunchScope ls(K_COL_AUX, 8.0 * co * K, 0.0, st);
+    launch_pdl(unpad_grad_kernel, (co * K + 255) / 256, 256, 0, st, gpad, co, K, Kp, gw);
 }
 
 }  // namespace ast

@@ -16,7 +16,7 @@ struct ConvGeom {
 enum KernelKind {
     K_CONV_FWD = 0, K_CONV_BWD_DATA, K_CONV_BWD_WEIGHT, K_REDUCE_SPLITS, K_DW_FWD, K_DW_BWD_DATA, K_DW_BWD_WEIGHT,
     K_DW_BWD_WEIGHT_FINISH, K_BN_STATS, K_BN_STATS_FINISH, K_BN_BWD_REDUCE, K_BN_BWD_FINISH, K_EW_ADD, K_EW_MASK, K_EW_SUM,
-    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_CONV3_BWD_WEIGHT_TC, K_DW_BWD_FUSED, K_KINDS
+    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_CONV3_BWD_WEIGHT_TC, K_DW_BWD_FUSED, K_IM2COL, K_COL_AUX, K_KINDS
 };
 const char* kernel_name(int kind);
 
@@ -70,6 +70,12 @@ void conv_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float*
 // gw[ko][r][s][c] = sum_{n,ho,wo} dz[n,ho,wo,ko] * x[n,ho*st-pad+r,wo*st-pad+s,c]; split over pixels, partials in scratch
 void conv_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats,
                      float* gw, cudaStream_t st);
+
+// ---- dense conv with a short reduction (k*k*c_in <= 64, e.g. the 3-channel stem) in bfloat16 mode: explicit im2col,
+// then the pointwise tensor-core kernels over col[pixels][Kp] with weights padded to [co][Kp] ----
+void conv_im2col(const ConvGeom& g, const ValSrc& x, int Kp, void* col, cudaStream_t st);
+void conv_pad_weights(const float* w, int co, int K, int Kp, __nv_bfloat16* wpad, cudaStream_t st);
+void conv_unpad_grad(const float* gpad, int co, int K, int Kp, float* gw, cudaStream_t st);
 
 // ---- pointwise conv on tcgen05 tensor cores (bf16 storage, channel counts multiples of 8) ----
 bool pw_tc_supported(int dtype, const ConvGeom& g, bool bwd_data);

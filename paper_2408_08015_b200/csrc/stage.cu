@@ -60,6 +60,11 @@ struct Unit {
     long w_off = -1, b_off = -1, gamma_off = -1, beta_off = -1;   // floats into the parameter arena
     size_t k_off = 0;       // floats into the backward-coefficient arena (k1,k2,k3)
     size_t run_off = 0;     // floats into the running-statistics arena
+    // dense conv with a short reduction, bfloat16 mode: forward and weight gradient run as pointwise tensor-core GEMMs
+    // over an explicit im2col tensor kept in the slot (col_kp = padded reduction length, 0 = not such a unit)
+    int col_kp = 0;
+    size_t col_off = 0;     // bytes into a slot
+    size_t wpad_off = 0;    // elements into the padded bf16 weight arena
 };
 
 struct Timing {
@@ -84,6 +89,9 @@ struct asteroid_stage {
     float *w = nullptr, *v = nullptr, *G = nullptr, *g = nullptr, *derived = nullptr, *run = nullptr, *coef = nullptr, *scratch = nullptr;
     int32_t* perm = nullptr;
     __nv_bfloat16 *wb = nullptr, *wtb = nullptr;   // bf16 copies of the weights and of the derived (transposed) weights
+    __nv_bfloat16* wpad = nullptr;                 // [co][Kp] bf16 weights of the im2col units
+    float* gpad = nullptr;                         // [co][Kp] padded weight gradient of the im2col unit at hand
+    size_t n_wpad = 0, n_gpad = 0;
     int* err = nullptr;                            // device error word (bounded waits)
     // Weight-gradient kernels depend only on the BatchNorm-backward coefficients of their unit and nothing in the rest of
     // the backward pass depends on them: they run on a second stream (forked from and joined back into the caller's
@@ -267,6 +275,17 @@ static int build_plan(asteroid_stage* s) {
         v.grad_off = gb;
         gb += align_up(v.elems * s->esz, 256);
     }
+    for (auto& u : s->units) {
+        const int K = u.g.k * u.g.k * u.g.ci;
+        if (u.kind == U_CONV && s->dtype == AST_BF16 && u.g.k > 1 && K <= 64 && u.g.co % 8 == 0 && u.g.co <= 256 && u.b_off < 0) {
+            u.col_kp = (K + 15) / 16 * 16;
+            u.col_off = sb;
+            sb += align_up((size_t)u.g.n * u.g.ho * u.g.wo * u.col_kp * 2, 256);
+            u.wpad_off = s->n_wpad;
+            s->n_wpad += (size_t)u.g.co * u.col_kp;
+            s->n_gpad = std::max(s->n_gpad, (size_t)u.g.co * u.col_kp);
+        }
+    }
     s->slot_stat_off = sb;
     for (auto& u : s->units) {
         if (u.l_bn >= 0) {
@@ -309,7 +328,7 @@ static void free_stage(asteroid_stage* s) {
     for (auto e : s->tm.ev) cudaEventDestroy(e);
     cudaFree(s->w); cudaFree(s->v); cudaFree(s->G); cudaFree(s->g); cudaFree(s->derived); cudaFree(s->run);
     cudaFree(s->coef); cudaFree(s->scratch); cudaFree(s->perm); cudaFree(s->slot_mem); cudaFree(s->grad_mem);
-    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err); cudaFree(s->scratch_side);
+    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err); cudaFree(s->scratch_side); cudaFree(s->wpad); cudaFree(s->gpad);
     if (s->ev_fork) cudaEventDestroy(s->ev_fork);
     if (s->ev_join) cudaEventDestroy(s->ev_join);
     if (s->side) cudaStreamDestroy(s->side);
@@ -337,6 +356,20 @@ static int reset_bn_running(asteroid_stage* s) {
             for (int c = 0; c < u.g.co; ++c) h[u.run_off + u.g.co + c] = 1.f;
     CU(cudaMemcpy(s->run, h.data(), h.size() * sizeof(float), cudaMemcpyHostToDevice));
     return AST_OK;
+}
+
+// derived weight copies of every kind, after the master weights changed
+static void refresh_weights(asteroid_stage* s, cudaStream_t st) {
+    refresh_derived(s->w, s->perm, s->derived, s->wb, s->wtb, s->n_params, st);
+    for (const auto& u : s->units)
+        if (u.col_kp) conv_pad_weights(s->w + u.w_off, u.g.co, u.g.k * u.g.k * u.g.ci, u.col_kp, s->wpad + u.wpad_off, st);
+}
+
+// geometry of the pointwise GEMM that stands for an im2col unit
+static ConvGeom col_geom(const Unit& u) {
+    ConvGeom g = u.g;
+    g.hi = u.g.ho; g.wi = u.g.wo; g.ci = u.col_kp; g.k = 1; g.stride = 1; g.pad = 0;
+    return g;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -384,7 +417,12 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
         if (u.kind == U_CONV) {
             const float* bias = u.b_off >= 0 ? s->w + u.b_off : nullptr;
             const bool bn = u.l_bn >= 0;
-            if (pw_tc_supported(dt, u.g, false))
+            if (u.col_kp) {
+                void* col = sv.base + u.col_off;
+                conv_im2col(u.g, val_src(s, sv, u.in), u.col_kp, col, st);
+                fused_stats = pw_fwd_tc(col_geom(u), ValSrc{col, nullptr, nullptr, ACT_NONE}, s->wpad + u.wpad_off, nullptr, obuf,
+                                        bn ? s->run + u.run_off : nullptr, bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
+            } else if (pw_tc_supported(dt, u.g, false))
                 fused_stats = pw_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, bias, obuf, bn ? s->run + u.run_off : nullptr,
                                         bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
             else if (conv3_tc_supported(dt, u.g)) conv3_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, obuf, s->err, st);
@@ -522,7 +560,10 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                 int frc = fork();
                 if (frc) return frc;
             }
-            if (u.kind == U_CONV && pw_tc_supported(dt, u.g, false))
+            if (u.kind == U_CONV && u.col_kp) {
+                pw_bwd_weight_tc(col_geom(u), d, ValSrc{sv.base + u.col_off, nullptr, nullptr, ACT_NONE}, wscratch, s->scratch_floats, s->gpad, s->err, wst);
+                conv_unpad_grad(s->gpad, u.g.co, u.g.k * u.g.k * u.g.ci, u.col_kp, s->g + u.w_off, wst);
+            } else if (u.kind == U_CONV && pw_tc_supported(dt, u.g, false))
                 pw_bwd_weight_tc(u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst);
             else if (u.kind == U_CONV && conv3_wgrad_tc_supported(dt, u.g))
                 conv3_bwd_weight_tc(u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst);
@@ -617,6 +658,10 @@ static int create_impl(const ast_layer* net, int n_layers, int first, int last, 
         if ((rc = dev_alloc(&s->wb, np * 2, &mod))) return rc;
         if ((rc = dev_alloc(&s->wtb, np * 2, &mod))) return rc;
     }
+    if (s->n_wpad) {
+        if ((rc = dev_alloc(&s->wpad, s->n_wpad * 2, &mod))) return rc;
+        if ((rc = dev_alloc(&s->gpad, s->n_gpad * 4, &work))) return rc;
+    }
     if ((rc = dev_alloc(&s->err, 256, &work))) return rc;
     if ((rc = dev_alloc(&s->v, np * 4, &opt))) return rc;
     if ((rc = dev_alloc(&s->slot_mem, s->slot_bytes * s->slots, &act))) return rc;
@@ -692,7 +737,7 @@ int asteroid_stage_import_state(asteroid_stage* s, const float* params, const fl
         if (momentum) CU(cudaMemcpy(s->v, momentum, n * 4, cudaMemcpyHostToDevice));
         else CU(cudaMemset(s->v, 0, n * 4));
         CU(cudaMemset(s->G, 0, n * 4));
-        refresh_derived(s->w, s->perm, s->derived, s->wb, s->wtb, n, 0);
+        refresh_weights(s, 0);
     }
     int rc = reset_bn_running(s);
     if (rc) return rc;
@@ -786,7 +831,7 @@ int asteroid_stage_step(asteroid_stage* s, float lr, float momentum, void* strea
     if (s->n_acc != s->M) return fail(AST_ERR_ORDER, "step after %d of %d micro-batches accumulated", s->n_acc, s->M);
     cudaStream_t st = (cudaStream_t)stream;
     sgd_step(s->w, s->v, s->G, s->n_params, 1.f / (float)s->M, lr, momentum, st);
-    refresh_derived(s->w, s->perm, s->derived, s->wb, s->wtb, s->n_params, st);
+    refresh_weights(s, st);
     CU(cudaGetLastError());
     s->n_acc = 0;
     return AST_OK;
@@ -846,6 +891,7 @@ int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_pr
                 CU(cudaMemcpy(t->wb, s->wb, s->n_params * 2, cudaMemcpyDeviceToDevice));
                 CU(cudaMemcpy(t->wtb, s->wtb, s->n_params * 2, cudaMemcpyDeviceToDevice));
             }
+            if (s->wpad && t->wpad && s->n_wpad == t->n_wpad) CU(cudaMemcpy(t->wpad, s->wpad, s->n_wpad * 2, cudaMemcpyDeviceToDevice));
         }
         const Val &vi = t->vals[0], &vo = t->vals.back();
         char *x = nullptr, *y = nullptr, *dy = nullptr, *dx = nullptr;
