@@ -277,6 +277,46 @@ __global__ void __launch_bounds__(256) ew_flat_kernel(int mode, const T* __restr
     st_raw_w<T, V>(dst, i * V, x);
 }
 
+// Stride-2 3x3 convs on the stride-1 tensor-core kernels.
+// Backward: up[n][2*ho][2*wo][c] = dz[n][ho][wo][c] (formed on load), zero elsewhere on the hi x wi grid: the input
+// gradient of the stride-2 conv is the stride-1 input gradient of `up`.
+template <typename T, int V>
+__global__ void __launch_bounds__(256) ew_upsample2_kernel(GradSrc d, int hi, int wi, int ho, int wo, int c, size_t groups, T* __restrict__ up) {
+    pdl_wait();
+    pdl_launch();
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= groups) return;
+    const int cv = c / V;
+    const int j = (int)(i % cv);
+    size_t t = i / cv;
+    const int v = (int)(t % wi);
+    t /= wi;
+    const int u = (int)(t % hi), n = (int)(t / hi);
+    float f[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) f[q] = 0.f;
+    if (!(u & 1) && !(v & 1) && (u >> 1) < ho && (v >> 1) < wo)
+        ld_grad_w<T, V>(d, (((size_t)n * ho + (u >> 1)) * wo + (v >> 1)) * c + (size_t)j * V, j * V, f);
+    st_raw_w<T, V>(up, i * V, f);
+}
+// Forward: z[n][ho][wo][c] = full[n][2*ho][2*wo][c], `full` the stride-1 output on the hi x wi grid.
+template <typename T, int V>
+__global__ void __launch_bounds__(256) ew_subsample2_kernel(const T* __restrict__ full, int hi, int wi, int ho, int wo, int c, size_t groups, T* __restrict__ z) {
+    pdl_wait();
+    pdl_launch();
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= groups) return;
+    const int cv = c / V;
+    const int j = (int)(i % cv);
+    size_t t = i / cv;
+    const int x = (int)(t % wo);
+    t /= wo;
+    const int y = (int)(t % ho), n = (int)(t / ho);
+    float f[V];
+    ld_raw_w<T, V>(full, (((size_t)n * hi + 2 * y) * wi + 2 * x) * c + (size_t)j * V, f);
+    st_raw_w<T, V>(z, i * V, f);
+}
+
 template <typename T> __global__ void gap_fwd_kernel(ValSrc x, int n, int hw, int c, T* __restrict__ out) {
     pdl_wait();
     pdl_launch();
@@ -536,6 +576,19 @@ static void ew_flat(int dtype, int mode, const void* a, const void* b, size_t n,
 
 void ew_relu_mask(int dtype, const void* d, const void* out_val, size_t n, void* dst, cudaStream_t st) { ew_flat(dtype, 0, d, out_val, n, dst, st); }
 void ew_sum(int dtype, const void* a, const void* b, size_t n, void* dst, cudaStream_t st) { ew_flat(dtype, 1, a, b, n, dst, st); }
+
+void ew_upsample2_grad(const GradSrc& d, int n, int hi, int wi, int ho, int wo, int c, void* up, cudaStream_t st) {
+    const size_t groups = (size_t)n * hi * wi * (c / 8);
+    LaunchScope ls(K_EW_SUM, 2.0 * ((double)n * ho * wo * c * ((d.act != ACT_NONE || d.k1) ? 2.0 : 1.0) + (double)n * hi * wi * c), 0.0, st);
+    launch_pdl(ew_upsample2_kernel<__nv_bfloat16, 8>, (unsigned)((groups + 255) / 256), 256, 0, st, d, hi, wi, ho, wo, c, groups, (__nv_bfloat16*)up);
+}
+
+void ew_subsample2(const void* full, int n, int hi, int wi, int ho, int wo, int c, void* z, cudaStream_t st) {
+    const size_t groups = (size_t)n * ho * wo * (c / 8);
+    LaunchScope ls(K_EW_SUM, 4.0 * (double)n * ho * wo * c, 0.0, st);
+    launch_pdl(ew_subsample2_kernel<__nv_bfloat16, 8>, (unsigned)((groups + 255) / 256), 256, 0, st, (const __nv_bfloat16*)full, hi, wi, ho, wo, c, groups,
+               (__nv_bfloat16*)z);
+}
 
 void gap_fwd(int dtype, const ValSrc& x, int n, int hw, int c, void* out, cudaStream_t st) {
     int total = n * c;

@@ -143,6 +143,9 @@ void ew_add(int dtype, const ValSrc& a, const ValSrc& b, int act, size_t pixels,
 void ew_apply(int dtype, const ValSrc& a, size_t pixels, int c, void* out, cudaStream_t st);
 void ew_relu_mask(int dtype, const void* d, const void* out_val, size_t n, void* dst, cudaStream_t st);
 void ew_sum(int dtype, const void* a, const void* b, size_t n, void* dst, cudaStream_t st);
+// bfloat16, channel counts multiples of 8: zero-inserted gradient / subsampled output of a stride-2 3x3 conv (see conv3_s2_tc_supported)
+void ew_upsample2_grad(const GradSrc& d, int n, int hi, int wi, int ho, int wo, int c, void* up, cudaStream_t st);
+void ew_subsample2(const void* full, int n, int hi, int wi, int ho, int wo, int c, void* z, cudaStream_t st);
 void gap_fwd(int dtype, const ValSrc& x, int n, int hw, int c, void* out, cudaStream_t st);
 void gap_bwd(int dtype, const void* da, int n, int hw, int c, const void* addend, void* dx, cudaStream_t st);
 

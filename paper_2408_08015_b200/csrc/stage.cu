@@ -365,6 +365,22 @@ static void refresh_weights(asteroid_stage* s, cudaStream_t st) {
         if (u.col_kp) conv_pad_weights(s->w + u.w_off, u.g.co, u.g.k * u.g.k * u.g.ci, u.col_kp, s->wpad + u.wpad_off, st);
 }
 
+// A stride-2 3x3 conv (pad 1, bfloat16, channel counts the stride-1 tensor-core kernels take) runs on those kernels:
+// forward as the stride-1 conv on the input grid followed by a 2x subsampling, backward-data as the stride-1 input
+// gradient of the zero-inserted output gradient.  Four times the multiply-adds of the direct form, on tensor cores
+// instead of FFMA.  Both need one full-resolution tensor in the scratch arena.
+static ConvGeom s1_geom(const Unit& u) {
+    ConvGeom g = u.g;
+    g.ho = u.g.hi; g.wo = u.g.wi; g.stride = 1;
+    return g;
+}
+static bool conv3_s2_tc_supported(const asteroid_stage* s, const Unit& u) {
+    if (s->dtype != AST_BF16 || u.kind != U_CONV || u.g.k != 3 || u.g.stride != 2 || u.g.pad != 1) return false;
+    if (!conv3_tc_supported(s->dtype, s1_geom(u))) return false;
+    const size_t full = (size_t)u.g.n * u.g.hi * u.g.wi * std::max(u.g.ci, u.g.co) * 2;
+    return full <= s->scratch_floats * sizeof(float);
+}
+
 // geometry of the pointwise GEMM that stands for an im2col unit
 static ConvGeom col_geom(const Unit& u) {
     ConvGeom g = u.g;
@@ -426,6 +442,10 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
                 fused_stats = pw_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, bias, obuf, bn ? s->run + u.run_off : nullptr,
                                         bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
             else if (conv3_tc_supported(dt, u.g)) conv3_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, obuf, s->err, st);
+            else if (conv3_s2_tc_supported(s, u)) {
+                conv3_fwd_tc(s1_geom(u), val_src(s, sv, u.in), s->wb + u.w_off, s->scratch, s->err, st);
+                ew_subsample2(s->scratch, u.g.n, u.g.hi, u.g.wi, u.g.ho, u.g.wo, u.g.co, obuf, st);
+            }
             else conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, bias, obuf, st);
         } else if (u.kind == U_DW) {
             const bool bn = u.l_bn >= 0;
@@ -594,6 +614,11 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                         reduced[tgt] = 1;
                     }
                 } else if (u.kind == U_CONV && conv3_tc_supported(dt, u.g)) conv3_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
+                else if (u.kind == U_CONV && conv3_s2_tc_supported(s, u)) {
+                    ew_upsample2_grad(d, u.g.n, u.g.hi, u.g.wi, u.g.ho, u.g.wo, u.g.co, s->scratch, st);
+                    conv3_bwd_data_tc(s1_geom(u), GradSrc{s->scratch, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, ACT_NONE}, s->wtb + u.w_off, addend,
+                                      own(u.in), s->err, st);
+                }
                 else if (u.kind == U_CONV) conv_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 else dw_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 gi.state = G_OWNED;
