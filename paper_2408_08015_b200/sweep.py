@@ -7,6 +7,7 @@ at micro-batch sizes 4..64 with M = 8 in bfloat16.  Per stage: samples/s of a wh
 algorithmic GB/s of its kernels.
 
     python -m paper_2408_08015_b200.sweep [--parts 2 3 4 6] [--batches 4 8 16 32 64] [--layers] [--out FILE]
+    python -m paper_2408_08015_b200.sweep --resnet --batches 32 [--out FILE]      (ResNet-50 conv2_x+conv3_x stage, kernel trace)
 """
 import argparse
 import json
@@ -15,10 +16,10 @@ import sys
 import numpy as np
 
 
-def time_stage(P, torch, si, net, first, last, h, w, B, M, rounds=5, warm=3):
+def time_stage(P, torch, si, net, first, last, h, w, B, M, rounds=5, warm=3, trace=None, xent=None):
     dev = torch.device("cuda:0")
     bf = torch.bfloat16
-    is_last = last == len(net) - 1
+    is_last = (last == len(net) - 1) if xent is None else xent      # softmax cross-entropy head, else MSE
     hdl = P.asteroid_stage_create(net, first, last, h, w, B, M, dtype=P.AST_BF16, need_input_grad=int(first > 0))
     try:
         P.asteroid_stage_import_state(hdl, si.init_params(net, first, last, 0))
@@ -58,6 +59,12 @@ def time_stage(P, torch, si, net, first, last, h, w, B, M, rounds=5, warm=3):
         e1.record(st)
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / rounds
+        if trace is not None:
+            # per-kernel device times of the same round (every kernel alone on the stream, CUDA events around each launch)
+            P.asteroid_trace_start()
+            for _ in range(rounds):
+                one_round()
+            trace.extend(P.asteroid_trace_stop())
         return hdl, ms
     except Exception:
         P.asteroid_stage_destroy(hdl)
@@ -73,7 +80,26 @@ def main(argv=None):
     ap.add_argument("--batches", type=int, nargs="+", default=[4, 8, 16, 32, 64])
     ap.add_argument("--layers", action="store_true", help="also print the per-layer profile records")
     ap.add_argument("--out", default=None)
+    ap.add_argument("--resnet", action="store_true",
+                    help="instead of the sweep: the ResNet-50 conv2_x+conv3_x stage (56x56x64 input) as one stage at the given batches, with its kernel trace")
     args = ap.parse_args(argv)
+    if args.resnet:
+        net = si.resnet50_c2c3_net()
+        out = open(args.out, "w") if args.out else sys.stdout
+        for B in args.batches:
+            trace = []
+            hdl, ms = time_stage(P, torch, si, net, 0, len(net) - 1, 56, 56, B, 8, trace=trace, xent=False)
+            P.asteroid_stage_destroy(hdl)
+            tot = sum(k["total_ms"] for k in trace) or 1.0
+            rec = {"net": "resnet50_c2c3", "B": B, "M": 8, "ms_per_round": round(ms, 4), "samples_per_s": round(B * 8 / (ms * 1e-3), 1),
+                   "kernels": [{"name": k["name"], "launches": k["launches"], "us_per_launch": round(1e3 * k["total_ms"] / k["launches"], 1),
+                                "share": round(k["total_ms"] / tot, 4),
+                                "tflops": round(k["flops"] / (k["total_ms"] * 1e-3) / 1e12, 1) if k["total_ms"] > 0 else 0.0,
+                                "alg_gbs": round(k["alg_bytes"] / (k["total_ms"] * 1e-3) / 1e9, 1) if k["total_ms"] > 0 else 0.0}
+                               for k in sorted(trace, key=lambda k: -k["total_ms"])]}
+            out.write(json.dumps(rec) + "\n")
+            out.flush()
+        return
     net = si.mobilenetv2_net()
     units = si.mobilenetv2_units()
     shapes = si.out_shape(net, 0, len(net) - 1, 224, 224)
