@@ -88,6 +88,28 @@ def test_one_forward_one_backward_order_is_bit_identical():
     assert np.array_equal(a["G"], c["G"])          # run-to-run determinism
 
 
+def test_second_stream_round_is_bit_identical_to_a_one_stream_round():
+    """Backward runs its weight-gradient kernels on a stream of the stage's own, forked and joined inside the call.
+    While a kernel trace is recorded the same kernels all stay on the caller's stream, so both rounds must agree
+    bit for bit: a missing dependency between the two streams would show as a difference."""
+    import paper_2408_08015_b200 as P
+    net = si.stage_net_mbv2_4blocks()
+    first, last, h, w, B, M = 0, len(net) - 1, 56, 56, 8, 3
+    xs, tg, params, _ = make_inputs(net, first, last, h, w, B, M, "mse", 5, True)
+    a = gpu_round(net, first, last, h, w, B, M, "mse", xs, tg, params, True)
+    P.asteroid_trace_start()
+    try:
+        b = gpu_round(net, first, last, h, w, B, M, "mse", xs, tg, params, True)
+    finally:
+        kernels = P.asteroid_trace_stop()
+    assert sum(k["launches"] for k in kernels) > 0
+    c = gpu_round(net, first, last, h, w, B, M, "mse", xs, tg, params, True)
+    for r in (b, c):
+        assert np.array_equal(a["G"], r["G"]) and np.array_equal(a["w"], r["w"]) and np.array_equal(a["v"], r["v"])
+        for m in range(M):
+            assert np.array_equal(a["y"][m], r["y"][m]) and np.array_equal(a["dx"][m], r["dx"][m])
+
+
 def test_partitioned_stages_compose():
     """Config-5 style: a network cut at block boundaries, each stage run alone."""
     net, units = si.small_mobilenet(10)
