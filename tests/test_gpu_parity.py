@@ -24,6 +24,8 @@ SMALL = {
     "bnfree_block": (si.bnfree_net(8, 2), 9, 9, 2, 3, "mse"),
     "bottleneck_c64": (si.bottleneck_net(64, [(64, 128, 1, 1)]), 10, 9, 2, 2, "mse"),
     "bottleneck_c128": (si.bottleneck_net(128, [(128, 128, 2, 1)]), 7, 12, 2, 1, "mse"),
+    # stride-2 3x3 conv with tensor-core channel counts on an odd-sized map (zero-inserted gradient, subsampled forward)
+    "bottleneck_c64_s2_odd": (si.bottleneck_net(64, [(64, 128, 1, 2)]), 9, 7, 2, 2, "mse"),
 }
 
 
