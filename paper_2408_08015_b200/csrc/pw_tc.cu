@@ -446,6 +446,7 @@ struct PipeArgs {
     uint32_t a_bytes, b_bytes;  // one operand stage / the resident weights
     uint32_t o_bytes;           // one output staging tile [128][N] bf16 (multiple of 128)
     int OS;                     // output staging tiles: 1 or 2
+    int AS;                     // operand stages: 2, or 1 where a long reduction leaves no room for two
     const float* pivot;         // forward, optional: per-channel pivot of the fused BatchNorm statistics
     float* stat_partial;        // [CTAs][2][N]: sums of (z - pivot) and (z - pivot)^2 over the CTA's pixels
     // backward, optional: BatchNorm-backward sums of the produced gradient (the unit that made this conv's input)
@@ -469,8 +470,8 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     __shared__ int abort_store;
     volatile int* abort_flag = &abort_store;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* sA = base;                               // two operand stages
-    uint8_t* sB = base + 2 * (size_t)a.a_bytes;       // resident weights
+    uint8_t* sA = base;                               // operand stages (a.AS of them)
+    uint8_t* sB = base + (size_t)a.AS * a.a_bytes;    // resident weights
     uint8_t* sR = sB + a.b_bytes;                     // raw ring
     uint8_t* sO = sR + (size_t)a.R * a.raw_bytes;     // output staging tiles
     uint8_t* sZ = sO + (size_t)a.OS * a.o_bytes;      // backward sums: two tiles of the producing unit's raw output
@@ -583,17 +584,18 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
             const int steps = vpr_pad >> 1;
             for (int t = 0; t < my_tiles; ++t) {
-                const int st = t & 1, n = t >> 1;
-                if (!mbar_wait_abortable(a_full(st), (uint32_t)(n & 1), abort_flag)) break;
+                const int st = t & 1, n = t >> 1;                                    // accumulator stage and its use count
+                const int as = a.AS == 2 ? (t & 1) : 0, an = a.AS == 2 ? (t >> 1) : t;   // operand stage and its use count
+                if (!mbar_wait_abortable(a_full(as), (uint32_t)(an & 1), abort_flag)) break;
                 if (n > 0 && !mbar_wait_abortable(acc_empty(st), (uint32_t)((n - 1) & 1), abort_flag)) break;
                 fence_after_sync();
                 const uint32_t d = tmem + (uint32_t)(st * NT);
                 for (int k = 0; k < steps; ++k) {
                     const int kb = k >> 2, ks = k & 3;
-                    umma_bf16(d, make_desc(a0 + st * a.a_bytes + (uint32_t)kb * TM * 128u + (uint32_t)ks * 32u),
+                    umma_bf16(d, make_desc(a0 + as * a.a_bytes + (uint32_t)kb * TM * 128u + (uint32_t)ks * 32u),
                               make_desc(b0 + (uint32_t)kb * (uint32_t)NT * 128u + (uint32_t)ks * 32u), idesc, k > 0 ? 1u : 0u);
                 }
-                umma_commit(a_empty(st));
+                umma_commit(a_empty(as));
                 umma_commit(acc_full(st));
             }
         }
@@ -674,7 +676,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
-            const int st = t & 1, n = t >> 1;
+            const int st = a.AS == 2 ? (t & 1) : 0, n = a.AS == 2 ? (t >> 1) : t;    // operand stage and its use count
             if (n > 0 && !mbar_wait_abortable(a_empty(st), (uint32_t)((n - 1) & 1), abort_flag)) break;
             uint8_t* dstA = sA + (size_t)st * a.a_bytes;
             for (int sub = 0; sub < subs; ++sub, ++it) {
@@ -839,23 +841,27 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
     const size_t budget = 220 * 1024 - 1024;
     const int tensors = a.need_z ? 2 : 1;
     const size_t zp = a.r_partial ? 2 * (size_t)a.o_bytes : 0;      // two tiles of the raw output the backward sums read
-    // two output staging tiles if that still leaves room for two 64-pixel raw stages
-    a.OS = 2 * (size_t)a.a_bytes + a.b_bytes + 2 * (size_t)a.o_bytes + zp + 2 * (((size_t)64 * a.K * 2 * tensors + 127) / 128 * 128) <= budget ? 2 : 1;
-    const size_t fixed = 2 * (size_t)a.a_bytes + a.b_bytes + (size_t)a.OS * a.o_bytes + zp;
-    if (fixed >= budget) return false;
-    for (int rs = 128; rs >= 32; rs >>= 1) {
-        size_t rb = ((size_t)rs * a.K * 2 * tensors + 127) / 128 * 128;
-        size_t r = (budget - fixed) / rb;
-        if (r >= 2 || (r >= 1 && rs == 32)) {
-            // at least two stages in flight, at most MAX_RAW and no more than three tiles' worth
-            size_t cap = (size_t)3 * (TM / rs);
-            if (r > cap) r = cap;
-            if (r > MAX_RAW) r = MAX_RAW;
-            a.RS = rs;
-            a.R = (int)r;
-            a.raw_bytes = (uint32_t)rb;
-            *smem = fixed + r * rb + 1024;
-            return a.R >= 2;
+    // two operand stages if they fit; one for long reductions (the transform of tile t+1 then waits for the MMAs of t)
+    for (a.AS = 2; a.AS >= 1; --a.AS) {
+        const size_t ab = (size_t)a.AS * a.a_bytes;
+        // two output staging tiles if that still leaves room for two 64-pixel raw stages
+        a.OS = ab + a.b_bytes + 2 * (size_t)a.o_bytes + zp + 2 * (((size_t)64 * a.K * 2 * tensors + 127) / 128 * 128) <= budget ? 2 : 1;
+        const size_t fixed = ab + a.b_bytes + (size_t)a.OS * a.o_bytes + zp;
+        if (fixed >= budget) continue;
+        for (int rs = 128; rs >= 32; rs >>= 1) {
+            size_t rb = ((size_t)rs * a.K * 2 * tensors + 127) / 128 * 128;
+            size_t r = (budget - fixed) / rb;
+            if (r >= 2) {
+                // at least two stages in flight, at most MAX_RAW and no more than three tiles' worth
+                size_t cap = (size_t)3 * (TM / rs);
+                if (r > cap) r = cap;
+                if (r > MAX_RAW) r = MAX_RAW;
+                a.RS = rs;
+                a.R = (int)r;
+                a.raw_bytes = (uint32_t)rb;
+                *smem = fixed + r * rb + 1024;
+                return true;
+            }
         }
     }
     return false;
@@ -907,6 +913,7 @@ struct WgArgs {
     int mtiles, ntiles, NT, tmem_cols;
     int pa, pb;           // 64-channel panels of the two operands per stage (pa even)
     int need_z, R;
+    int OPS;              // operand stages: 2, or 1 where the raw ring needs the room
     uint32_t raw_bytes, op_bytes;
 };
 
@@ -918,8 +925,8 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
     __shared__ int abort_store;
     volatile int* abort_flag = &abort_store;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* sOp = base;                                   // two operand stages: [A panels][B panels]
-    uint8_t* sR = base + 2 * (size_t)a.op_bytes;           // raw ring
+    uint8_t* sOp = base;                                   // operand stages (a.OPS of them): [A panels][B panels]
+    uint8_t* sR = base + (size_t)a.OPS * a.op_bytes;       // raw ring
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = a.R;
     const uint32_t bar0 = smem_u32(&bars[0]);
@@ -978,7 +985,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
             const uint32_t idesc = make_idesc(a.NT) | (1u << 15) | (1u << 16);
             bool ok = true;
             for (int it = 0; it < stages && ok; ++it) {
-                const int st = it & 1, n = it >> 1;
+                const int st = a.OPS == 2 ? (it & 1) : 0, n = a.OPS == 2 ? (it >> 1) : it;
                 if (!mbar_wait_abortable(op_full(st), (uint32_t)(n & 1), abort_flag)) {
                     ok = false;
                     break;
@@ -1012,7 +1019,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
         xv.init(a.x, jb << 3);
         bool ok = true;
         for (int it = 0; it < stages; ++it) {
-            const int st = it & 1, n = it >> 1, s = it % R;
+            const int st = a.OPS == 2 ? (it & 1) : 0, n = a.OPS == 2 ? (it >> 1) : it, s = it % R;
             if (n > 0 && !mbar_wait_abortable(op_empty(st), (uint32_t)((n - 1) & 1), abort_flag)) {
                 ok = false;
                 break;
@@ -1124,7 +1131,8 @@ bool plan_wgrad(WgArgs& a, size_t* smem, size_t scratch_floats, int n_sm) {
     rb = (rb + 127) / 128 * 128;
     a.raw_bytes = (uint32_t)rb;
     const size_t budget = 220 * 1024 - 1024;
-    const size_t fixed = 2 * (size_t)a.op_bytes;
+    a.OPS = 2 * (size_t)a.op_bytes + 2 * rb <= budget ? 2 : 1;
+    const size_t fixed = (size_t)a.OPS * a.op_bytes;
     if (fixed + 2 * rb > budget) return false;
     size_t r = (budget - fixed) / rb;
     if (r > 4) r = 4;
