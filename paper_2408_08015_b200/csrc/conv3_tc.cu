@@ -31,6 +31,8 @@ struct C3Args {
     int n_img, H, W, C, N;     // C: reduction channels (multiple of 64), N: output channels (multiple of 16, <= 256)
     int tiles_per_img, rows_pad, tmem_cols;
     int flip;                  // backward: tap t uses weight tap 8 - t
+    int resident;              // all nine taps' weights fit in shared memory beside the staged rows: loaded once, before the
+                               // dependency wait, and the 9 * C/16 MMAs are issued back to back
 };
 
 // K-major, 128-byte swizzle, start address anywhere on a 128-byte row of a 1024-byte aligned
@@ -40,7 +42,8 @@ struct C3Args {
 __device__ __forceinline__ uint64_t make_desc_row(uint32_t smem_addr) { return make_desc(smem_addr); }
 
 template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kernel(const C3Args a) {
-    pdl_wait();
+    // barriers, tensor memory and (resident form) the weights, which only the refresh kernel writes, are set up before
+    // the dependency wait and overlap the previous kernel's tail
     pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2];
@@ -67,6 +70,17 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
         tmem_alloc(smem_u32(&tmem_slot), (uint32_t)a.tmem_cols);
         tmem_relinquish();
     }
+    if (a.resident) {
+        const int vprw = a.C >> 3;
+        for (int v = tid; v < 9 * a.N * vprw; v += C3_THREADS) {
+            const int t = v / (a.N * vprw), rem = v - t * (a.N * vprw);
+            const int n = rem / vprw, j = rem - n * vprw;
+            const int wt = a.flip ? 8 - t : t;
+            uint4 q = __ldg(reinterpret_cast<const uint4*>(a.w + ((size_t)n * 9 + wt) * a.C) + j);
+            *reinterpret_cast<uint4*>(sB + (size_t)t * b_stage + tile_off(n, j, a.N)) = q;
+        }
+    }
+    pdl_wait();
     // ---- stage the input rows once: position -> (hp, wp); interior positions are pixels ----
     {
         const int vpr = a.C >> 3;
@@ -97,7 +111,22 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
     uint32_t ph[2] = {0, 0};
     bool bad = false;
     const int vpr = a.C >> 3;
-    for (int t = 0; t < 9; ++t) {
+    if (a.resident) {
+        if (tid == 0) {
+            for (int t = 0; t < 9; ++t) {
+                const int r = t / 3, s = t - r * 3;
+                const uint32_t a0 = smem_u32(sA) + (uint32_t)(r * Wp + s) * 128u;
+                const uint32_t b0 = smem_u32(sB) + (uint32_t)t * b_stage;
+                for (int k = 0; k < (a.C >> 4); ++k) {
+                    const int kb = k >> 2, ks = k & 3;
+                    umma_bf16(tmem, make_desc_row(a0 + (uint32_t)kb * a_block + (uint32_t)ks * 32u),
+                              make_desc(b0 + (uint32_t)kb * (uint32_t)a.N * 128u + (uint32_t)ks * 32u), idesc, (t > 0 || k > 0) ? 1u : 0u);
+                }
+            }
+            umma_commit(bar0);
+        }
+    }
+    for (int t = 0; t < 9 && !a.resident; ++t) {
         const int st = t & 1;
         if (t >= 2) {                                   // the MMAs of tap t-2 read this weight stage
             bool ok = mbar_wait(st ? bar1 : bar0, ph[st]);
@@ -177,7 +206,9 @@ template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, cudaStream
     a.tmem_cols = 32;
     while (a.tmem_cols < a.N) a.tmem_cols <<= 1;
     const int kbs = a.C / 64;
-    size_t smem = (size_t)kbs * a.rows_pad * 128 + 2 * (size_t)kbs * a.N * 128 + 1024;
+    // all nine taps resident if two CTAs per SM still fit with them
+    a.resident = ((size_t)kbs * a.rows_pad * 128 + 9 * (size_t)kbs * a.N * 128 + 1024 <= 110 * 1024) ? 1 : 0;
+    size_t smem = (size_t)kbs * a.rows_pad * 128 + (a.resident ? 9 : 2) * (size_t)kbs * a.N * 128 + 1024;
     static bool attr_set = false;
     if (!attr_set) {
         cudaFuncSetAttribute(conv3_tc_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
