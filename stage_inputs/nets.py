@@ -168,6 +168,33 @@ def small_mobilenet(classes=10):
     return _mobilenetv2(classes, [(1, 8, 1, 1), (2, 8, 2, 2), (2, 16, 1, 1)], stem_c=8, head_c=32)
 
 
+def single_unit_net(kind, c_in, c_out, k=1, stride=1, bn=False, act=None):
+    """One conv (or depthwise conv) layer, optionally followed by BatchNorm and an activation: the
+    smallest stage that exercises one contraction / stencil kernel path in both directions."""
+    b = _Builder()
+    if kind == "dwconv":
+        b.dwconv(c_in, stride)
+    else:
+        b.conv(c_in, c_out, k, stride, pad=(k - 1) // 2)
+    if bn:
+        b.bn(c_out)
+    if act:
+        getattr(b, act)(c_out)
+    return b.layers
+
+
+def head_net(c, classes, bn_conv=0):
+    """Classifier head: [1x1 conv to bn_conv channels + BatchNorm,] global average pool, linear."""
+    b = _Builder()
+    if bn_conv:
+        b.conv(c, bn_conv, 1)
+        b.bn(bn_conv)
+        c = bn_conv
+    b.gap(c)
+    b.linear(c, classes)
+    return b.layers
+
+
 def out_shape(net, first, last, in_h, in_w):
     """(h, w, c) of every layer's output in [first, last], keyed by layer index."""
     shp = {first - 1: (in_h, in_w, net[first].c_in)}

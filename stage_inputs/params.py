@@ -52,3 +52,18 @@ def init_params(net, first, last, seed=0):
         else:
             parts.append(np.zeros(n, np.float32))
     return np.concatenate(parts) if parts else np.zeros(0, np.float32)
+
+
+def randomize_bn(params, net, first, last, seed=0):
+    """Copy of a flat parameter vector with every BatchNorm's gamma drawn from U(0.5, 1.5) and beta from U(-0.5, 0.5):
+    with the initial gamma = 1, beta = 0 a mistake in how scale and shift are used would not show."""
+    out = np.array(params, np.float32, copy=True)
+    off = 0
+    for i, name, shape in param_layout(net, first, last):
+        n = int(np.prod(shape))
+        if name == "gamma":
+            out[off:off + n] = (0.5 + uniform(seed, 2 * _PARAM_TID + i, n)).astype(np.float32)
+        elif name == "beta":
+            out[off:off + n] = (uniform(seed, 3 * _PARAM_TID + i, n) - 0.5).astype(np.float32)
+        off += n
+    return out

@@ -1,5 +1,8 @@
 """Shared test harness: run one HPP-Round on the oracle and on the CUDA library from the same
 seeded inputs, and compare tensor by tensor.  Imported by tests and the smoke check only."""
+import json
+import os
+
 import numpy as np
 
 import stage_inputs as si
@@ -120,80 +123,122 @@ def rel_err(a, b, floor=0.0):
     return float(np.abs(a - b).max() / max(np.abs(b).max(), floor, 1e-300))
 
 
-def compare(gpu, ref, net, first, last, tol, need_dx=True, outlier_frac=0.0, outlier_cap=0.25, pure=None):
-    """Per tensor (every y_m, dx_m, loss_m; accumulated gradient, momentum and weights per
-    parameter tensor, denominators floored at 1% of the largest entry of their kind so that a
-    tensor whose true value vanishes is judged on the scale of its siblings):
+PARITY_LOG = os.environ.get("ASTEROID_PARITY_LOG",
+                            os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out", "parity_table.jsonl"))
 
-      primary    max|gpu-ref| / max|ref| <= tol, where up to `outlier_frac` of the elements may
-                 exceed tol (never `outlier_cap`): a pre-activation within float rounding of a
-                 ReLU/ReLU6 kink takes a different mask on the two sides.
-      calibrated (only if `pure`, the plain float64 result, is given and the primary test
-                 fails): with bfloat16 storage one-ulp differences between two correct
-                 implementations multiply through the layers and flip masks, so deep stages
-                 cannot agree element-wise on gradients.  Then the library must be no further
-                 from the exact result than the storage format itself puts a float64
-                 implementation: max-norm error vs `pure` <= 2x, and L2 error <= 1.5x, that of
-                 `ref` (the float64 oracle rounding at the storage points).
 
-    Returns worst ratios per kind plus counts of outlier elements and calibrated tensors."""
-    worst = {"outliers": 0, "calibrated": 0}
+def _log_records(case, records):
+    """One JSON line per compared tensor, appended to the parity table a GPU run leaves behind."""
+    if not case:
+        return
+    try:
+        os.makedirs(os.path.dirname(PARITY_LOG), exist_ok=True)
+        with open(PARITY_LOG, "a") as f:
+            for r in records:
+                f.write(json.dumps(dict(case=case, **r)) + "\n")
+    except OSError:
+        pass
 
-    def note(kind, a, b, floor=0.0, p=None):
-        a = np.asarray(a, np.float64).ravel()
-        b = np.asarray(b, np.float64).ravel()
+
+CONTRACT, MIRROR, CALIBRATED = "contract", "mirror", "calibrated"
+# Calibrated criterion: factors by which a tensor's error against the plain oracle may exceed the mirroring oracle's own
+# (max-norm, L2).  Measured over all deep bfloat16 cases of this suite the ratios have median 0.99 / 1.00; tensors of at
+# least 1000 elements stay below 1.33 / 1.08, while the ratio of two error norms over a few dozen elements (BatchNorm
+# parameters of narrow layers, the 3x3x3 stem) scatters up to 2.4 / 1.7.
+CAL_BIG, CAL_SMALL, CAL_SIZE = (1.5, 1.15), (3.0, 2.0), 1000
+ALL = (CONTRACT, MIRROR, CALIBRATED)
+
+
+def compare(gpu, plain, net, first, last, tol, need_dx=True, mirror=None, allow=(CONTRACT,), outlier_frac=0.0, outlier_cap=0.05,
+            case=None, contract_kinds=("y", "loss")):
+    """Judges every tensor of a round (each y_m, dx_m, loss_m; accumulated gradient, momentum and weights, parameter
+    tensor by parameter tensor) and returns {"records": [...], "counts": {criterion: n}, kind: worst contract error}.
+
+    `plain` is the round of the plain float64 oracle: the contract.  The metric is max|gpu-ref| / max|ref| per tensor;
+    parameter tensors use a denominator floored at 1% of the largest entry of their kind, so that a tensor whose
+    true value vanishes (a beta gradient in front of another BatchNorm) is judged on the scale of its siblings.
+
+    A tensor passes by the first criterion it meets; `allow` lists the ones a test accepts; tensors of the kinds in
+    `contract_kinds` (by default the activations y and the losses) must meet the contract whatever `allow` says:
+      contract    error against `plain` <= tol.
+      mirror      (diagnostic; needs `mirror`, the float64 oracle that rounds at the bfloat16 storage points and rounds
+                  the operands of dense contractions) error against `mirror` <= tol, where up to `outlier_frac` of the
+                  elements may exceed tol but never `outlier_cap`.  ReLU/ReLU6 masks are decisions taken on stored
+                  values; this oracle takes them on the same rounded values the library sees.
+      calibrated  (diagnostic) the library is no further from `plain` than the storage format alone puts the
+                  mirroring oracle: max-norm error <= 1.5x and L2 error <= 1.15x the mirror's own (3x / 2x for tensors of fewer
+                  than 1000 elements, where a ratio of two error norms is itself noisy).
+    """
+    records, counts, worst = [], {CONTRACT: 0, MIRROR: 0, CALIBRATED: 0}, {}
+
+    def norms(a, b, floor):
         scale = max(np.abs(b).max(), floor, 1e-300)
         err = np.abs(a - b) / scale
-        assert np.isfinite(a).all(), "%s: non-finite values" % kind
-        bad = int((err > tol).sum())
-        e = float(err.max())
-        if bad and bad <= outlier_frac * err.size and e <= outlier_cap:
-            worst["outliers"] += bad
-            e = float(err[err <= tol].max())
-        if e > tol and p is not None:
-            p = np.asarray(p, np.float64).ravel()
-            ps = max(np.abs(p).max(), floor, 1e-300)
-            g_max, r_max = np.abs(a - p).max() / ps, np.abs(b - p).max() / ps
-            pn = max(np.linalg.norm(p), floor * np.sqrt(p.size), 1e-300)
-            g_l2, r_l2 = np.linalg.norm(a - p) / pn, np.linalg.norm(b - p) / pn
-            ok = g_max <= 2.0 * r_max and g_l2 <= 1.5 * r_l2
-            assert ok, ("%s: %.3e vs storage-mirroring oracle; vs float64: max %.3e (mirror %.3e), L2 %.3e (mirror %.3e)"
-                        % (kind, e, g_max, r_max, g_l2, r_l2))
-            worst["calibrated"] += 1
-            worst[kind + "_vs_f64"] = max(worst.get(kind + "_vs_f64", 0.0), float(g_max))
-            return
-        worst[kind] = max(worst.get(kind, 0.0), e)
-        assert e <= tol, "%s: relative error %.3e exceeds %.1e (%d of %d elements)" % (kind, e, tol, bad, err.size)
+        l2 = float(np.linalg.norm(a - b) / max(np.linalg.norm(b), floor * np.sqrt(b.size), 1e-300))
+        return err, l2
 
-    P = pure
-    for m in range(len(ref["y"])):
-        note("y", gpu["y"][m], ref["y"][m], p=P and P["y"][m])
+    def note(kind, name, a, p, m, floor=0.0):
+        must_contract = kind in contract_kinds
+        a = np.asarray(a, np.float64).ravel()
+        p = np.asarray(p, np.float64).ravel()
+        assert np.isfinite(a).all(), "%s: non-finite values" % name
+        err_p, l2_p = norms(a, p, floor)
+        rec = {"tensor": name, "kind": kind, "n": int(a.size), "err_plain": float(err_p.max()), "l2_plain": l2_p}
+        ok = None
+        if rec["err_plain"] <= tol:
+            ok = CONTRACT
+        if m is not None:
+            m = np.asarray(m, np.float64).ravel()
+            err_m, l2_m = norms(a, m, floor)
+            mp, l2_mp = norms(m, p, floor)
+            bad = int((err_m > tol).sum())
+            rec.update(err_mirror=float(err_m.max()), l2_mirror=l2_m, mirror_vs_plain=float(mp.max()), l2_mirror_vs_plain=l2_mp,
+                       outliers=bad)
+            if ok is None and (bad == 0 or (bad <= outlier_frac * err_m.size and float(err_m.max()) <= outlier_cap)):
+                ok = MIRROR
+            cm, cl = CAL_BIG if a.size >= CAL_SIZE else CAL_SMALL
+            if ok is None and rec["err_plain"] <= cm * rec["mirror_vs_plain"] and l2_p <= cl * l2_mp:
+                ok = CALIBRATED
+        rec["criterion"] = ok or "FAIL"
+        records.append(rec)
+        accepted = (CONTRACT,) if must_contract else allow
+        if ok in accepted:
+            counts[ok] += 1
+            worst[kind] = max(worst.get(kind, 0.0), rec["err_plain"])
+            return None
+        return "%s: %s (accepted: %s) %s" % (name, rec["criterion"], "/".join(accepted), {k: ("%.3e" % v if isinstance(v, float) else v)
+                                                                                         for k, v in rec.items() if k not in ("tensor", "kind")})
+
+    fails = []
+    M_ = mirror
+    for m in range(len(plain["y"])):
+        fails.append(note("y", "y[%d]" % m, gpu["y"][m], plain["y"][m], M_ and M_["y"][m]))
         if need_dx:
-            note("dx", gpu["dx"][m], ref["dx"][m], p=P and P["dx"][m])
-        note("loss", [gpu["loss"][m]], [ref["loss"][m]], p=P and [P["loss"][m]])
-    # parameter tensors: primary criterion tensor by tensor; if one misses and `pure` is given, the
-    # calibrated criterion is applied once to the whole flat vector of that kind (single small
-    # tensors are too few samples for a ratio of two error norms to be stable)
+            fails.append(note("dx", "dx[%d]" % m, gpu["dx"][m], plain["dx"][m], M_ and M_["dx"][m]))
+        fails.append(note("loss", "loss[%d]" % m, [gpu["loss"][m]], [plain["loss"][m]], M_ and [M_["loss"][m]]))
     for kind in ("G", "v", "w"):
-        kmax = np.abs(ref[kind]).max()
-        off, missed = 0, False
-        for i, name, shape in si.param_layout(net, first, last):
+        kmax = np.abs(plain[kind]).max()
+        off = 0
+        for i, pname, shape in si.param_layout(net, first, last):
             n = int(np.prod(shape))
             sl = slice(off, off + n)
             off += n
-            try:
-                note(kind, gpu[kind][sl], ref[kind][sl], floor=1e-2 * kmax)
-            except AssertionError:
-                if P is None:
-                    raise
-                missed = True
-        if missed:
-            note(kind, gpu[kind], ref[kind], p=P[kind])
+            fails.append(note(kind, "%s[%d.%s]" % (kind, i, pname), gpu[kind][sl], plain[kind][sl], M_ and M_[kind][sl], floor=1e-2 * kmax))
+    _log_records(case, records)
+    fails = [f for f in fails if f]
+    assert not fails, "%d tensors fail:\n%s" % (len(fails), "\n".join(fails[:12]))
+    worst["records"] = records
+    worst["counts"] = counts
     return worst
 
 
+def summary(worst):
+    """Short printable form of compare's result."""
+    return {k: ("%.2e" % v if isinstance(v, float) else v) for k, v in worst.items() if k != "records"}
+
+
 def sampled_round_check(net, first, last, h, w, B, M, loss, bf16, sample, tol, seed=0, need_dx=1, lr=0.01, mu=0.9,
-                        outlier_frac=1e-3, deep=True):
+                        outlier_frac=0.0, allow=(CONTRACT,), case=None, contract_kinds=("y", "loss")):
     """Full-size round on the GPU (all M micro-batches); the oracle computes only the micro-batches
     in `sample` (micro-batches are independent given the weights: BatchNorm statistics are per
     micro-batch), and the rest of the round is checked through what holds at any size:
@@ -211,9 +256,10 @@ def sampled_round_check(net, first, last, h, w, B, M, loss, bf16, sample, tol, s
     assert np.abs(gpu["w"] - w_expect).max() <= 2e-7 * np.abs(w_expect).max()
     S = len(sample)
     sx, st = [xs[m] for m in sample], [tg[m] for m in sample]
-    ref = oracle_round(net, first, last, B, S, loss, sx, st, params, lr=lr, mu=mu, store=bf16_store if bf16 else None)
-    pure = oracle_round(net, first, last, B, S, loss, sx, st, params, lr=lr, mu=mu) if (bf16 and deep) else None
+    plain = oracle_round(net, first, last, B, S, loss, sx, st, params, lr=lr, mu=mu)
+    mirror = oracle_round(net, first, last, B, S, loss, sx, st, params, lr=lr, mu=mu, store=bf16_store) if bf16 else None
     Gs = np.sum([gpu["g"][m].astype(np.float64) for m in sample], axis=0)
     sub = {"y": [gpu["y"][m] for m in sample], "dx": [gpu["dx"][m] for m in sample], "loss": [gpu["loss"][m] for m in sample],
            "G": Gs, "v": Gs / S, "w": params.astype(np.float64) - lr * Gs / S}
-    return compare(sub, ref, net, first, last, tol, need_dx=need_dx != 0, outlier_frac=outlier_frac, pure=pure)
+    return compare(sub, plain, net, first, last, tol, need_dx=need_dx != 0, mirror=mirror, allow=allow, outlier_frac=outlier_frac, case=case,
+                   contract_kinds=contract_kinds)

@@ -8,7 +8,7 @@ import numpy as np
 import pytest
 
 import stage_inputs as si
-from harness import bf16_store, compare, gpu_round, make_inputs, oracle_round, sampled_round_check
+from harness import ALL, CONTRACT, MIRROR, bf16_store, compare, gpu_round, make_inputs, oracle_round, sampled_round_check, summary
 
 pytestmark = pytest.mark.gpu
 
@@ -29,51 +29,72 @@ SMALL = {
 }
 
 
-def run_case(net, h, w, B, M, loss, bf16, seed=0, first=0, last=None, **kw):
+def run_case(net, h, w, B, M, loss, bf16, seed=0, first=0, last=None, allow=(CONTRACT,), outlier_frac=0.0, case=None,
+             contract_kinds=("y", "loss"), **kw):
     last = len(net) - 1 if last is None else last
     xs, tg, params, _ = make_inputs(net, first, last, h, w, B, M, loss, seed, bf16)
-    outlier_frac = kw.pop("outlier_frac", 0.0)
-    deep = kw.pop("deep", False)     # bfloat16 stage of several blocks: see harness.compare
     okw = {k: v for k, v in kw.items() if k in ("order", "rounds")}
-    ref = oracle_round(net, first, last, B, M, loss, xs, tg, params, store=bf16_store if bf16 else None, **okw)
-    pure = oracle_round(net, first, last, B, M, loss, xs, tg, params, **okw) if (bf16 and deep) else None
+    plain = oracle_round(net, first, last, B, M, loss, xs, tg, params, **okw)
+    mirror = oracle_round(net, first, last, B, M, loss, xs, tg, params, store=bf16_store, **okw) if bf16 else None
     gpu = gpu_round(net, first, last, h, w, B, M, loss, xs, tg, params, bf16, **kw)
-    return compare(gpu, ref, net, first, last, TOL[bf16], need_dx=kw.get("need_dx", 1) != 0, outlier_frac=outlier_frac, pure=pure)
+    return compare(gpu, plain, net, first, last, TOL[bf16], need_dx=kw.get("need_dx", 1) != 0, mirror=mirror, allow=allow,
+                   outlier_frac=outlier_frac, case=case, contract_kinds=contract_kinds)
+
+
+# What each bfloat16 case is held to (float32 cases: the contract alone, on every tensor).  Activation-free kernel paths meet the
+# contract outright (test_gpu_kernel_parity.py).  In a stage with ReLU/ReLU6 a bfloat16 implementation takes the masks on
+# rounded values; about 0.2% of them differ from the float64 masks and each flip moves the gradients at a few pixels by
+# several per cent of their maximum, so already for one block the gradients of ANY bfloat16-storage implementation,
+# the float64 mirroring oracle included, sit 7-15% (max-norm) from the plain oracle.  There the gradients are held to
+# the mirroring oracle; only stages several blocks deep, where one-ulp differences between two correct implementations
+# multiply from layer to layer, need the calibrated criterion.  (criteria for gradients, kinds that must meet the contract)
+SHALLOW = ((CONTRACT, MIRROR), ("y", "loss"))
+BF16_RULES = {
+    "block_ragged": SHALLOW, "block_c16": SHALLOW, "bnfree_block": SHALLOW, "bottleneck_c64": SHALLOW, "bottleneck_c64_s2_odd": SHALLOW,
+    "bottlenecks_small": ((CONTRACT, MIRROR), ("loss",)),
+    "bottleneck_c128": (ALL, ("y", "loss")), "mbv2_4blocks_small": (ALL, ("y", "loss")), "small_mobilenet_xent": (ALL, ("y", "loss")),
+}
 
 
 @pytest.mark.parametrize("bf16", [False, True], ids=["f32", "bf16"])
 @pytest.mark.parametrize("name", list(SMALL))
 def test_small_stages(name, bf16):
     net, h, w, B, M, loss = SMALL[name]
-    print(name, run_case(net, h, w, B, M, loss, bf16, deep=True))
+    allow, kinds = BF16_RULES[name] if bf16 else ((CONTRACT,), ("y", "loss"))
+    r = run_case(net, h, w, B, M, loss, bf16, allow=allow, contract_kinds=kinds, outlier_frac=5e-4 if allow is ALL else 0.0,
+                 case="small/%s/%s" % (name, "bf16" if bf16 else "f32"))
+    print(name, summary(r))
 
 
 def test_config1_block_fp32():
     """One inverted-residual block 16->96->16 at 32x32, micro-batch 8, M=4, float32, MSE."""
-    print(run_case(si.block_net(16, 6), 32, 32, 8, 4, "mse", False, outlier_frac=1e-3))
+    print(summary(run_case(si.block_net(16, 6), 32, 32, 8, 4, "mse", False, case="config1/f32")))
 
 
 def test_config1_two_rounds_momentum():
-    print(run_case(si.block_net(16, 6), 32, 32, 8, 4, "mse", False, rounds=2, outlier_frac=1e-3))
+    print(summary(run_case(si.block_net(16, 6), 32, 32, 8, 4, "mse", False, rounds=2, case="config1/f32/two_rounds")))
 
 
 def test_config2_stage_bf16_full_size():
     """Four inverted-residual blocks at 56x56, micro-batch 32, M=8, bfloat16: the benchmarked workload
     in the benchmark's launch configuration; the oracle evaluates micro-batches 0 and 7."""
-    print(sampled_round_check(si.stage_net_mbv2_4blocks(), 0, 34, 56, 56, 32, 8, "mse", True, [0, 7], 2e-2))
+    print(summary(sampled_round_check(si.stage_net_mbv2_4blocks(), 0, 34, 56, 56, 32, 8, "mse", True, [0, 7], 2e-2, allow=ALL, outlier_frac=5e-4,
+                                      case="config2/bf16")))
 
 
 def test_config3_mobilenetv2_bf16_full_size():
     """Full MobileNetV2 at 224x224x3, softmax cross-entropy, M=4 micro-batches of 16; oracle on micro-batch 3."""
     net = si.mobilenetv2_net()
-    print(sampled_round_check(net, 0, len(net) - 1, 224, 224, 16, 4, "xent", True, [3], 2e-2, need_dx=0))
+    print(summary(sampled_round_check(net, 0, len(net) - 1, 224, 224, 16, 4, "xent", True, [3], 2e-2, need_dx=0, allow=ALL, outlier_frac=5e-4,
+                                      case="config3/bf16", contract_kinds=("loss",))))
 
 
 def test_config4_resnet_stage_bf16():
     """ResNet-50 conv2_x+conv3_x at 56x56x64, M=8; micro-batch 8 instead of 32 bounds the oracle's time
     (1.7 GMAC per sample); oracle on micro-batch 5."""
     net = si.resnet50_c2c3_net()
-    print(sampled_round_check(net, 0, len(net) - 1, 56, 56, 8, 8, "mse", True, [5], 2e-2))
+    print(summary(sampled_round_check(net, 0, len(net) - 1, 56, 56, 8, 8, "mse", True, [5], 2e-2, allow=ALL, outlier_frac=5e-4,
+                                      case="config4/bf16/B8", contract_kinds=("loss",))))
 
 
 def test_one_forward_one_backward_order_is_bit_identical():
@@ -120,4 +141,5 @@ def test_partitioned_stages_compose():
     for first, last in cuts:
         h, w, _ = shapes[first - 1] if first > 0 else (32, 32, 3)
         loss = "xent" if last == len(net) - 1 else "mse"
-        print((first, last), run_case(net, h, w, 4, 2, loss, True, first=first, last=last, need_dx=int(first > 0), deep=True))
+        print((first, last), summary(run_case(net, h, w, 4, 2, loss, True, first=first, last=last, need_dx=int(first > 0), allow=(CONTRACT, MIRROR),
+                                              case="small_mobilenet_parts/%d-%d" % (first, last))))

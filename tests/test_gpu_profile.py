@@ -4,7 +4,7 @@ import pytest
 
 import oracle as O
 import stage_inputs as si
-from harness import bf16_store, compare, gpu_round, make_inputs, oracle_round
+from harness import ALL, bf16_store, compare, gpu_round, make_inputs, oracle_round, summary
 
 pytestmark = pytest.mark.gpu
 
@@ -54,7 +54,9 @@ def test_full_resolution_partitions_match_oracle(parts):
         h, w, _ = shapes[first - 1] if first > 0 else (224, 224, 3)
         loss = "xent" if last == len(net) - 1 else "mse"
         xs, tg, params, _ = make_inputs(net, first, last, h, w, B, M, loss, 1, True)
-        ref = oracle_round(net, first, last, B, M, loss, xs, tg, params, store=bf16_store)
-        pure = oracle_round(net, first, last, B, M, loss, xs, tg, params)
+        mirror = oracle_round(net, first, last, B, M, loss, xs, tg, params, store=bf16_store)
+        plain = oracle_round(net, first, last, B, M, loss, xs, tg, params)
         gpu = gpu_round(net, first, last, h, w, B, M, loss, xs, tg, params, True, need_dx=int(first > 0))
-        print((first, last), compare(gpu, ref, net, first, last, 2e-2, need_dx=first > 0, outlier_frac=1e-3, pure=pure))
+        print((first, last), summary(compare(gpu, plain, net, first, last, 2e-2, need_dx=first > 0, mirror=mirror, allow=ALL, outlier_frac=5e-4,
+                                             case="config5/P%d/%d-%d/B4" % (parts, first, last),
+                                             contract_kinds=("loss",) if parts == 2 else ("y", "loss"))))
