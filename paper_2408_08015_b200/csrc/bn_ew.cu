@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(512) chan_reduce_kernel(OP op, size_t pixels, 
         float ctx[OP::NCTX][V];
         op.template init<T, V>(c0, ctx);
         size_t pbeg = (size_t)blockIdx.y * pix_per_block, pend = min(pixels, pbeg + pix_per_block);
-#pragma unroll 4
+#pragma unroll 8
         for (size_t p = pbeg + row; p < pend; p += rows) op.template acc<T, V>(p * c + c0, ctx, a);
     }
     const int width = cw * V;
@@ -117,7 +117,7 @@ ReducePlan plan_reduce(int dtype, size_t pixels, int c, int nacc, size_t scratch
     p.cw = cg < 32 ? cg : 32;
     p.rows = 512 / p.cw;
     p.gx = (cg + p.cw - 1) / p.cw;
-    size_t by = (148 + p.gx - 1) / p.gx;            // one 512-thread block per SM: half the partials of two 256-thread blocks
+    size_t by = (sm_count() + p.gx - 1) / p.gx;            // one 512-thread block per SM: half the partials of two 256-thread blocks
     size_t max_by = (pixels + (size_t)p.rows * 4 - 1) / ((size_t)p.rows * 4);
     if (by > max_by) by = max_by;
     size_t cap = scratch_floats / ((size_t)nacc * c);
@@ -385,8 +385,9 @@ __global__ void sgd_step_kernel(float* __restrict__ w, float* __restrict__ v, fl
 
 __global__ void refresh_kernel(const float* __restrict__ w, const int32_t* __restrict__ perm, float* __restrict__ d,
                                __nv_bfloat16* __restrict__ wb, __nv_bfloat16* __restrict__ wtb, size_t n) {
-    // This kernel writes the derived weight copies that other kernels stage before their dependency wait, so it
-    // releases its dependents only after its own stores are visible device-wide.
+    // This kernel writes the derived weight copies that other kernels stage BEFORE their dependency wait.  It therefore
+    // never releases its dependents early: without a launch_dependents the next kernel in the stream starts only when this
+    // grid has completed and its stores are visible, and every later kernel is ordered behind that one.
     pdl_wait();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) {
@@ -397,8 +398,6 @@ __global__ void refresh_kernel(const float* __restrict__ w, const int32_t* __res
             wtb[i] = __float2bfloat16_rn(t);
         }
     }
-    __threadfence();
-    pdl_launch();
 }
 
 // ------------------------------------------------------------------ losses
@@ -536,9 +535,80 @@ void bn_bwd_finish_partials(const float* partial, int blocks, size_t pixels, int
     launch_pdl(bn_bwd_finish, (c + 31) / 32, 1024, 0, st, partial, blocks, c, (double)pixels, mean, rstd, gamma, o);
 }
 
+// Vector form with the per-channel coefficients in registers: the grid's threads are cut to a multiple of the vectors per
+// pixel, so that a thread striding by that count always lands on the same channels; four vectors of each operand are
+// loaded before any is used.
+template <typename T, int V>
+__global__ void __launch_bounds__(256) ew_add_vec_kernel(ValSrc a, ValSrc b, int act, size_t groups, int vpr, size_t stride, T* __restrict__ out,
+                                                          T* __restrict__ out2) {
+    pdl_wait();
+    pdl_launch();
+    const size_t id = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (id >= stride) return;
+    const int c0 = (int)(id % (size_t)vpr) * V;
+    float as[V], ah[V], bs[V], bh[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) {
+        as[q] = a.scale ? __ldg(a.scale + c0 + q) : 1.f;
+        ah[q] = a.scale ? __ldg(a.shift + c0 + q) : 0.f;
+        bs[q] = (b.p && b.scale) ? __ldg(b.scale + c0 + q) : 1.f;
+        bh[q] = (b.p && b.scale) ? __ldg(b.shift + c0 + q) : 0.f;
+    }
+    const float alo = a.act == ACT_NONE ? -INFINITY : 0.f, ahi = a.act == ACT_RELU6 ? 6.f : INFINITY;
+    const float blo = b.act == ACT_NONE ? -INFINITY : 0.f, bhi = b.act == ACT_RELU6 ? 6.f : INFINITY;
+    const float olo = act == ACT_NONE ? -INFINITY : 0.f, ohi = act == ACT_RELU6 ? 6.f : INFINITY;
+    constexpr int U = 4;
+    for (size_t i0 = id; i0 < groups; i0 += U * stride) {
+        Vec<T> va[U], vb[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t i = i0 + u * stride;
+            if (i < groups) {
+                va[u].load(a.p, i);
+                if (b.p) vb[u].load(b.p, i);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t i = i0 + u * stride;
+            if (i < groups) {
+                float x[V], y[V];
+                va[u].unpack(x);
+#pragma unroll
+                for (int q = 0; q < V; ++q) x[q] = fminf(fmaxf(fmaf(x[q], as[q], ah[q]), alo), ahi);
+                if (b.p) {
+                    vb[u].unpack(y);
+#pragma unroll
+                    for (int q = 0; q < V; ++q) x[q] += fminf(fmaxf(fmaf(y[q], bs[q], bh[q]), blo), bhi);
+                }
+#pragma unroll
+                for (int q = 0; q < V; ++q) x[q] = fminf(fmaxf(x[q], olo), ohi);
+                Vec<T> o;
+                o.pack(x);
+                o.store(out, i);
+                if (out2) o.store(out2, i);
+            }
+        }
+    }
+}
+
 template <typename T, int V> static void ew_add_launch(const ValSrc& a, const ValSrc& b, int act, size_t n, int c, void* out, void* out2, cudaStream_t st) {
     size_t groups = n / V;
     LaunchScope ls(K_EW_ADD, (double)n * sizeof(T) * (1 + (b.p ? 1 : 0) + 1 + (out2 ? 1 : 0)), (double)n, st);
+    if (V > 1) {
+        const int vpr = c / V;
+        size_t blocks = (groups + 4 * 256 - 1) / (4 * 256);
+        const size_t cap = (size_t)sm_count() * 8;
+        if (blocks > cap) blocks = cap;
+        size_t threads = blocks * 256;
+        if (threads < (size_t)vpr) {
+            blocks = ((size_t)vpr + 255) / 256;
+            threads = blocks * 256;
+        }
+        const size_t stride = threads / vpr * vpr;
+        launch_pdl(ew_add_vec_kernel<T, V>, (unsigned)blocks, 256, 0, st, a, b, act, groups, vpr, stride, (T*)out, (T*)out2);
+        return;
+    }
     launch_pdl(ew_add_kernel<T, V>, (unsigned)((groups + 255) / 256), 256, 0, st, a, b, act, groups, c, (T*)out, (T*)out2);
 }
 

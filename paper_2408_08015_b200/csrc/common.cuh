@@ -113,9 +113,9 @@ template <> struct Vec<__nv_bfloat16> {
 
 // Vector forms of ld_val / ld_grad: N consecutive channels starting at channel c0 of element
 // vector `vec_idx` (index in units of vectors).
-template <typename T> __device__ __forceinline__ void ld_val_vec(const ValSrc& s, size_t vec_idx, int c0, float* out) {
-    Vec<T> v;
-    v.load(s.p, vec_idx);
+// The transforms on vectors already in registers (so that a kernel can issue the loads of several vectors before it
+// transforms any of them).
+template <typename T> __device__ __forceinline__ void val_from_raw(const ValSrc& s, const Vec<T>& v, int c0, float* out) {
     v.unpack(out);
     if (s.scale) {
 #pragma unroll
@@ -126,15 +126,12 @@ template <typename T> __device__ __forceinline__ void ld_val_vec(const ValSrc& s
         for (int i = 0; i < Vec<T>::N; ++i) out[i] = apply_act(out[i], s.act);
     }
 }
-
-template <typename T> __device__ __forceinline__ void ld_grad_vec(const GradSrc& s, size_t vec_idx, int c0, float* out) {
-    Vec<T> v;
-    v.load(s.dy, vec_idx);
-    v.unpack(out);
-    if (s.act == ACT_NONE && s.k1 == nullptr) return;
+__device__ __forceinline__ bool grad_needs_z(const GradSrc& s) { return s.act != ACT_NONE || s.k1 != nullptr; }
+template <typename T> __device__ __forceinline__ void grad_from_raw(const GradSrc& s, const Vec<T>& dy, const Vec<T>& zv, int c0, float* out) {
+    dy.unpack(out);
+    if (!grad_needs_z(s)) return;
     float z[Vec<T>::N];
-    v.load(s.z, vec_idx);
-    v.unpack(z);
+    zv.unpack(z);
 #pragma unroll
     for (int i = 0; i < Vec<T>::N; ++i) {
         float pre = s.scale ? fmaf(z[i], __ldg(s.scale + c0 + i), __ldg(s.shift + c0 + i)) : z[i];
@@ -142,6 +139,20 @@ template <typename T> __device__ __forceinline__ void ld_grad_vec(const GradSrc&
         if (s.k1) d = fmaf(__ldg(s.k1 + c0 + i), d, fmaf(__ldg(s.k3 + c0 + i), z[i], __ldg(s.k2 + c0 + i)));
         out[i] = d;
     }
+}
+
+template <typename T> __device__ __forceinline__ void ld_val_vec(const ValSrc& s, size_t vec_idx, int c0, float* out) {
+    Vec<T> v;
+    v.load(s.p, vec_idx);
+    val_from_raw<T>(s, v, c0, out);
+}
+
+template <typename T> __device__ __forceinline__ void ld_grad_vec(const GradSrc& s, size_t vec_idx, int c0, float* out) {
+    Vec<T> v, z;
+    v.load(s.dy, vec_idx);
+    z.raw = v.raw;
+    if (grad_needs_z(s)) z.load(s.z, vec_idx);
+    grad_from_raw<T>(s, v, z, c0, out);
 }
 
 // Width-generic access: V == Vec<T>::N uses 16-byte vectors, V == 1 scalars (channel counts that

@@ -72,6 +72,7 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
     }
     if (a.resident) {
         const int vprw = a.C >> 3;
+#pragma unroll 4
         for (int v = tid; v < 9 * a.N * vprw; v += C3_THREADS) {
             const int t = v / (a.N * vprw), rem = v - t * (a.N * vprw);
             const int n = rem / vprw, j = rem - n * vprw;
@@ -82,22 +83,46 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
     }
     pdl_wait();
     // ---- stage the input rows once: position -> (hp, wp); interior positions are pixels ----
+    // A thread owns one 16-byte channel chunk (its transform coefficients stay in registers) and every (256 / chunks)-th
+    // row; the global loads of four rows are issued together before any of them is transformed, so that their
+    // latencies overlap instead of adding up.
     {
-        const int vpr = a.C >> 3;
-        for (int v = tid; v < rows * vpr; v += C3_THREADS) {
-            const int r = v / vpr, j = v - r * vpr;
-            const int f = fs0 + r;
-            const int hp = f / Wp, wp = f - hp * Wp;
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (f >= 0 && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W) {
-                float fv[8];
-                const int c0 = j << 3;
-                const size_t e = (((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.C + c0;
-                if (BWD) ld_grad_vec<__nv_bfloat16>(a.dz, e >> 3, c0, fv);
-                else ld_val_vec<__nv_bfloat16>(a.x, e >> 3, c0, fv);
-                q = pack8(fv);
+        const int vpr = a.C >> 3;                       // 8 or a multiple of 8 dividing 256
+        const int j = tid % vpr, step = C3_THREADS / vpr;
+        const int c0 = j << 3;
+        const bool need_z = BWD && (a.dz.act != ACT_NONE || a.dz.k1 != nullptr);
+        XfVal xv;
+        XfGrad xg;
+        if (BWD) xg.init(a.dz, c0);
+        else xv.init(a.x, c0);
+        const uint4* src = reinterpret_cast<const uint4*>(BWD ? a.dz.dy : a.x.p);
+        const uint4* srcz = reinterpret_cast<const uint4*>(a.dz.z);
+        constexpr int U = 4;
+        for (int rb = tid / vpr; rb < rows; rb += U * step) {
+            uint4 raw[U], rawz[U];
+            bool ok[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int r = rb + u * step;
+                const int f = fs0 + r;
+                const int hp = f / Wp, wp = f - hp * Wp;
+                ok[u] = r < rows && f >= 0 && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+                raw[u] = rawz[u] = make_uint4(0, 0, 0, 0);
+                if (ok[u]) {
+                    const size_t e = ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.C + c0) >> 3;
+                    raw[u] = __ldg(src + e);
+                    if (need_z) rawz[u] = __ldg(srcz + e);
+                }
             }
-            *reinterpret_cast<uint4*>(sA + (size_t)(j >> 3) * a_block + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int r = rb + u * step;
+                if (r < rows) {
+                    uint4 q = make_uint4(0, 0, 0, 0);
+                    if (ok[u]) q = BWD ? (need_z ? xg.apply(raw[u], rawz[u]) : raw[u]) : xv.apply(raw[u]);
+                    *reinterpret_cast<uint4*>(sA + (size_t)(j >> 3) * a_block + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+                }
+            }
         }
     }
     fence_async_smem();
@@ -138,6 +163,7 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
         }
         const int wt = a.flip ? 8 - t : t;
         uint8_t* dstB = sB + (size_t)st * b_stage;
+#pragma unroll 4
         for (int v = tid; v < a.N * vpr; v += C3_THREADS) {
             const int n = v / vpr, j = v - n * vpr;
             uint4 q = __ldg(reinterpret_cast<const uint4*>(a.w + ((size_t)n * 9 + wt) * a.C) + j);
@@ -198,7 +224,253 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
     if (warp == 0) tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
 }
 
-template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, cudaStream_t st) {
+// ---------------------------------------------------------------------------------------------
+// Persistent form of the same implicit GEMM for layers of up to 128 reduction channels on maps up to 61 pixels wide
+// (every dense 3x3 layer of the ResNet stage).  One CTA per SM walks over tiles and keeps resident, for all nine
+// taps, the weights of the 64 output channels it owns (wider layers are split over CTAs by output channel), so that
+// per tile only the halo rows are brought in.  The loop is software-pipelined with all threads in the same role:
+//
+//   iteration i:  transform the prefetched raw rows of tile i into the operand buffer -> issue its 9*C/16 MMAs into
+//                 accumulator i&1 -> issue the global loads of tile i+1's rows into registers -> wait for the MMAs of
+//                 tile i-1 and store its accumulator (i-1)&1
+//
+// so the MMAs of a tile run while the next tile's loads are in flight and the previous tile is being stored.  With 64
+// reduction channels two operand buffers fit and the transform of tile i+1 overlaps the MMAs of tile i as well.
+constexpr int C3P_THREADS = 512;
+constexpr int C3P_NH = 64;             // output channels per CTA
+
+struct C3PArgs {
+    ValSrc x;
+    GradSrc dz;
+    const __nv_bfloat16* w;    // [N][9][C]
+    const void* addend;
+    __nv_bfloat16* out;        // [n][H][W][N]
+    int* err;
+    int n_img, H, W, C, N;
+    int tiles_per_img, total_tiles, rows_pad, n_split, nbuf, flip;
+};
+
+template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) conv3_persist_kernel(const C3PArgs a) {
+    pdl_launch();
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2];
+    __shared__ uint32_t tmem_slot;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Wp = a.W + 2;
+    const int kbs = a.C >> 6;
+    const uint32_t a_block = (uint32_t)a.rows_pad * 128u;
+    const uint32_t a_buf = (uint32_t)kbs * a_block;
+    const uint32_t b_tap = (uint32_t)kbs * C3P_NH * 128u;
+    uint8_t* sA = base;
+    uint8_t* sB = base + (size_t)a.nbuf * a_buf;
+    const int half = blockIdx.x % a.n_split, n0 = half * C3P_NH;
+    const int cta = blockIdx.x / a.n_split, nctas = gridDim.x / a.n_split;
+    const int rows = TM + 2 * Wp + 2;
+    const uint32_t bar[2] = {smem_u32(&bars[0]), smem_u32(&bars[1])};
+    if (tid == 0) {
+        mbar_init(bar[0], 1);
+        mbar_init(bar[1], 1);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), 2 * C3P_NH);
+        tmem_relinquish();
+    }
+    // resident weights of this CTA's 64 output channels, all nine taps (written only by the refresh kernel, which never
+    // releases its dependents early: safe to read before the dependency wait)
+    {
+        const int vprw = a.C >> 3;
+#pragma unroll 4
+        for (int v = tid; v < 9 * C3P_NH * vprw; v += C3P_THREADS) {
+            const int t = v / (C3P_NH * vprw), rem = v - t * (C3P_NH * vprw);
+            const int n = rem / vprw, j = rem - n * vprw;
+            const int wt = a.flip ? 8 - t : t;
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(a.w + ((size_t)(n0 + n) * 9 + wt) * a.C) + j);
+            *reinterpret_cast<uint4*>(sB + (size_t)t * b_tap + tile_off(n, j, C3P_NH)) = q;
+        }
+    }
+    fence_async_smem();
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    pdl_wait();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t idesc = make_idesc(C3P_NH);
+
+    // staging role: one 16-byte channel chunk (coefficients in registers), every (512 / chunks)-th row
+    const int vpr = a.C >> 3;
+    const int j = tid % vpr, step = C3P_THREADS / vpr, r_first = tid / vpr;
+    const int c0 = j << 3;
+    const bool need_z = BWD && grad_needs_z(a.dz);
+    XfVal xv;
+    XfGrad xg;
+    if (BWD) xg.init(a.dz, c0);
+    else xv.init(a.x, c0);
+    const uint4* src = reinterpret_cast<const uint4*>(BWD ? a.dz.dy : a.x.p);
+    const uint4* srcz = reinterpret_cast<const uint4*>(a.dz.z);
+    uint4 raw[IT], rawz[IT];
+    uint32_t okmask = 0;
+
+    auto prefetch = [&](int tl) {
+        const int img = tl / a.tiles_per_img, tile = tl - img * a.tiles_per_img;
+        const int fs0 = tile * TM;                          // first staged position (first output position - Wp - 1)
+        okmask = 0;
+#pragma unroll
+        for (int u = 0; u < IT; ++u) {
+            const int r = r_first + u * step;
+            const int f = fs0 + r;
+            const int hp = f / Wp, wp = f - hp * Wp;
+            const bool ok = r < rows && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+            raw[u] = make_uint4(0, 0, 0, 0);
+            if (BWD) rawz[u] = make_uint4(0, 0, 0, 0);
+            if (ok) {
+                const size_t e = ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.C + c0) >> 3;
+                raw[u] = __ldg(src + e);
+                if (need_z) rawz[u] = __ldg(srcz + e);
+                okmask |= 1u << u;
+            }
+        }
+    };
+    auto store_stage = [&](int buf) {
+        uint8_t* dst = sA + (size_t)buf * a_buf + (size_t)(j >> 3) * a_block;
+#pragma unroll
+        for (int u = 0; u < IT; ++u) {
+            const int r = r_first + u * step;
+            if (r < rows) {
+                uint4 q = make_uint4(0, 0, 0, 0);
+                if (okmask & (1u << u)) q = BWD ? (need_z ? xg.apply(raw[u], rawz[u]) : raw[u]) : xv.apply(raw[u]);
+                *reinterpret_cast<uint4*>(dst + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+            }
+        }
+    };
+    auto issue = [&](int buf, int acc) {
+        const uint32_t abase = smem_u32(sA) + (uint32_t)buf * a_buf, bbase = smem_u32(sB);
+        const uint32_t d = tmem + (uint32_t)(acc * C3P_NH);
+        for (int t = 0; t < 9; ++t) {
+            const int r = t / 3, s = t - r * 3;
+            const uint32_t a0 = abase + (uint32_t)(r * Wp + s) * 128u;
+            const uint32_t b0 = bbase + (uint32_t)t * b_tap;
+            for (int k = 0; k < (a.C >> 4); ++k) {
+                const int kb = k >> 2, ks = k & 3;
+                umma_bf16(d, make_desc(a0 + (uint32_t)kb * a_block + (uint32_t)ks * 32u), make_desc(b0 + (uint32_t)kb * C3P_NH * 128u + (uint32_t)ks * 32u),
+                          idesc, (t > 0 || k > 0) ? 1u : 0u);
+            }
+        }
+        umma_commit(bar[acc]);
+    };
+    // 16 warps: warp & 3 = tensor-memory lane quarter (32 positions), warp >> 2 = 16 of the 64 output channels
+    auto epilogue = [&](int tl, int acc) {
+        const int img = tl / a.tiles_per_img, tile = tl - img * a.tiles_per_img;
+        const int q = warp & 3, cg = warp >> 2;
+        const int f = Wp + 1 + tile * TM + q * 32 + lane;
+        const int hp = f / Wp, wp = f - hp * Wp;
+        const bool pix = hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+        float v[16];
+        tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * C3P_NH + (cg << 4)), v);
+        if (pix) {
+            const size_t e0 = (((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.N + n0 + (cg << 4);
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                float* vv = v + (hh << 3);
+                const size_t e = e0 + (hh << 3);
+                if (BWD && a.addend) {
+                    float ad[8];
+                    Vec<__nv_bfloat16> av;
+                    av.load(a.addend, e >> 3);
+                    av.unpack(ad);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) vv[i] += ad[i];
+                }
+                *reinterpret_cast<uint4*>(a.out + e) = pack8(vv);
+            }
+        }
+    };
+
+    const int my = cta < a.total_tiles ? (a.total_tiles - cta + nctas - 1) / nctas : 0;
+    uint32_t ph[2] = {0, 0};
+    bool bad = false;
+    auto wait_mma = [&](int i) -> bool {       // block-uniform result
+        const int acc = i & 1;
+        const bool ok = mbar_wait(bar[acc], ph[acc]);
+        ph[acc] ^= 1;
+        return __syncthreads_and(ok ? 1 : 0) != 0;
+    };
+    if (my > 0) prefetch(cta);
+    for (int i = 0; i < my && !bad; ++i) {
+        const int buf = a.nbuf == 2 ? (i & 1) : 0;
+        if (a.nbuf == 1 && i > 0 && !wait_mma(i - 1)) {          // the single operand buffer is still being read
+            bad = true;
+            break;
+        }
+        store_stage(buf);
+        fence_async_smem();
+        fence_before_sync();
+        __syncthreads();
+        if (tid == 0) {
+            fence_after_sync();
+            issue(buf, i & 1);
+        }
+        if (i + 1 < my) prefetch(cta + (i + 1) * nctas);
+        if (i > 0) {
+            if (a.nbuf == 2 && !wait_mma(i - 1)) {
+                bad = true;
+                break;
+            }
+            fence_after_sync();
+            epilogue(cta + (i - 1) * nctas, (i - 1) & 1);
+        }
+    }
+    if (!bad && my > 0) {
+        if (!wait_mma(my - 1)) bad = true;
+        else {
+            fence_after_sync();
+            epilogue(cta + (my - 1) * nctas, (my - 1) & 1);
+        }
+    }
+    if (bad && tid == 0) atomicExch(a.err, 1);
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 2 * C3P_NH);
+}
+
+// true if the persistent kernel takes the layer; fills its launch geometry
+bool plan_c3p(const C3Args& a, C3PArgs& p, size_t* smem, int* it) {
+    if (a.C > 128 || a.C % 64 || a.N % C3P_NH) return false;
+    const int Wp = a.W + 2, rows = TM + 2 * Wp + 2;
+    const int kbs = a.C / 64;
+    *it = a.C == 64 ? 4 : 8;
+    if (rows > *it * (C3P_THREADS / (a.C >> 3))) return false;
+    p.x = a.x; p.dz = a.dz; p.w = a.w; p.addend = a.addend; p.out = a.out; p.err = a.err;
+    p.n_img = a.n_img; p.H = a.H; p.W = a.W; p.C = a.C; p.N = a.N; p.flip = a.flip;
+    p.tiles_per_img = ((a.H - 1) * Wp + a.W + TM - 1) / TM;
+    p.total_tiles = a.n_img * p.tiles_per_img;
+    p.rows_pad = (rows + 7) / 8 * 8;
+    p.n_split = a.N / C3P_NH;
+    const size_t wbytes = 9 * (size_t)kbs * C3P_NH * 128, abuf = (size_t)kbs * p.rows_pad * 128;
+    const size_t budget = 225 * 1024;
+    p.nbuf = wbytes + 2 * abuf + 1024 <= budget ? 2 : 1;
+    *smem = wbytes + p.nbuf * abuf + 1024;
+    return *smem <= budget;
+}
+
+template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, double useful_flops, cudaStream_t st) {
+    {
+        C3PArgs p{};
+        size_t psmem = 0;
+        int it = 0;
+        if (plan_c3p(a, p, &psmem, &it)) {
+            smem_limit_once<106>(conv3_persist_kernel<BWD, 4>, 226 * 1024);
+            smem_limit_once<107>(conv3_persist_kernel<BWD, 8>, 226 * 1024);
+            const int n_sm = sm_count();
+            int nctas = n_sm / p.n_split;
+            if (nctas < 1) nctas = 1;
+            if (nctas > p.total_tiles) nctas = p.total_tiles;
+            LaunchScope ls(kind, bytes, useful_flops > 0 ? useful_flops : 2.0 * 9.0 * a.n_img * a.H * a.W * (double)a.C * a.N, st);
+            if (it == 4) launch_pdl(conv3_persist_kernel<BWD, 4>, nctas * p.n_split, C3P_THREADS, psmem, st, p);
+            else launch_pdl(conv3_persist_kernel<BWD, 8>, nctas * p.n_split, C3P_THREADS, psmem, st, p);
+            return;
+        }
+    }
     const int Wp = a.W + 2;
     const int centers = (a.H - 1) * Wp + a.W;           // positions Wp+1 .. H*Wp+W
     a.tiles_per_img = (centers + TM - 1) / TM;
@@ -209,12 +481,8 @@ template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, cudaStream
     // all nine taps resident if two CTAs per SM still fit with them
     a.resident = ((size_t)kbs * a.rows_pad * 128 + 9 * (size_t)kbs * a.N * 128 + 1024 <= 110 * 1024) ? 1 : 0;
     size_t smem = (size_t)kbs * a.rows_pad * 128 + (a.resident ? 9 : 2) * (size_t)kbs * a.N * 128 + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(conv3_tc_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_set = true;
-    }
-    LaunchScope ls(kind, bytes, 2.0 * 9.0 * a.n_img * a.H * a.W * (double)a.C * a.N, st);
+    smem_limit_once<108>(conv3_tc_kernel<BWD>, 200 * 1024);
+    LaunchScope ls(kind, bytes, useful_flops > 0 ? useful_flops : 2.0 * 9.0 * a.n_img * a.H * a.W * (double)a.C * a.N, st);
     launch_pdl(conv3_tc_kernel<BWD>, a.n_img * a.tiles_per_img, C3_THREADS, smem, st, a);
 }
 
@@ -278,38 +546,70 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
     const int tile_beg = blockIdx.x * a.tiles_per_cta, tile_end = min(a.total_tiles, tile_beg + a.tiles_per_cta);
     uint32_t phase = 0;
     bool bad = false;
+    const int vx = a.CI >> 3, vz = a.CO >> 3;             // chunks per row: 8 or 16, both divide 256
+    const int jx = tid % vx, jz = tid % vz, stepx = C3_THREADS / vx, stepz = C3_THREADS / vz;
+    const bool need_z = a.dz.act != ACT_NONE || a.dz.k1 != nullptr;
+    const uint4* gx = reinterpret_cast<const uint4*>(a.x.p);
+    const uint4* gdy = reinterpret_cast<const uint4*>(a.dz.dy);
+    const uint4* gz = reinterpret_cast<const uint4*>(a.dz.z);
+    XfVal xv;
+    XfGrad xg;
+    xv.init(a.x, jx << 3);
+    xg.init(a.dz, jz << 3);
     for (int tl = tile_beg; tl < tile_end; ++tl) {
         const int img = tl / a.tiles_per_img, tile = tl - img * a.tiles_per_img;
         const int f0 = Wp + 1 + tile * TM, fs0 = f0 - Wp - 1;
-        // x with halo
-        const int vx = a.CI >> 3;
-        for (int v = tid; v < rows * vx; v += C3_THREADS) {
-            const int r = v / vx, j = v - r * vx;
-            const int f = fs0 + r;
-            const int hp = f / Wp, wp = f - hp * Wp;
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (f >= 0 && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W) {
-                float fv[8];
-                const int c0 = j << 3;
-                ld_val_vec<__nv_bfloat16>(a.x, ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CI + c0) >> 3, c0, fv);
-                q = pack8(fv);
+        // x with halo, then dz at the 128 centre positions: a thread owns one 16-byte channel chunk of each operand
+        // (coefficients in registers) and every (256 / chunks)-th row; the loads of four rows are issued together
+        {
+            constexpr int U = 4;
+            for (int rb = tid / vx; rb < rows; rb += U * stepx) {
+                uint4 raw[U];
+                bool ok[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = rb + u * stepx;
+                    const int f = fs0 + r;
+                    const int hp = f / Wp, wp = f - hp * Wp;
+                    ok[u] = r < rows && f >= 0 && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+                    raw[u] = make_uint4(0, 0, 0, 0);
+                    if (ok[u]) raw[u] = __ldg(gx + (((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CI + (jx << 3)) >> 3));
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = rb + u * stepx;
+                    if (r < rows) {
+                        const uint4 q = ok[u] ? xv.apply(raw[u]) : make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4*>(sX + (size_t)(jx >> 3) * x_block + (size_t)r * 128 + ((((uint32_t)jx & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+                    }
+                }
             }
-            *reinterpret_cast<uint4*>(sX + (size_t)(j >> 3) * x_block + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
-        }
-        // dz at the 128 centre positions
-        const int vz = a.CO >> 3;
-        for (int v = tid; v < TM * vz; v += C3_THREADS) {
-            const int r = v / vz, j = v - r * vz;
-            const int f = f0 + r;
-            const int hp = f / Wp, wp = f - hp * Wp;
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W) {
-                float fv[8];
-                const int c0 = j << 3;
-                ld_grad_vec<__nv_bfloat16>(a.dz, ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CO + c0) >> 3, c0, fv);
-                q = pack8(fv);
+            for (int rb = tid / vz; rb < TM; rb += U * stepz) {
+                uint4 raw[U], rawz[U];
+                bool ok[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = rb + u * stepz;
+                    const int f = f0 + r;
+                    const int hp = f / Wp, wp = f - hp * Wp;
+                    ok[u] = r < TM && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+                    raw[u] = rawz[u] = make_uint4(0, 0, 0, 0);
+                    if (ok[u]) {
+                        const size_t e = ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CO + (jz << 3)) >> 3;
+                        raw[u] = __ldg(gdy + e);
+                        if (need_z) rawz[u] = __ldg(gz + e);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = rb + u * stepz;
+                    if (r < TM) {
+                        uint4 q = make_uint4(0, 0, 0, 0);
+                        if (ok[u]) q = need_z ? xg.apply(raw[u], rawz[u]) : raw[u];
+                        *reinterpret_cast<uint4*>(sDZ + (size_t)(jz >> 3) * dz_block + (size_t)r * 128 + ((((uint32_t)jz & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
+                    }
+                }
             }
-            *reinterpret_cast<uint4*>(sDZ + (size_t)(j >> 3) * dz_block + (size_t)r * 128 + ((((uint32_t)j & 7u) ^ ((uint32_t)r & 7u)) << 4)) = q;
         }
         fence_async_smem();
         __syncthreads();
@@ -403,21 +703,22 @@ bool conv3_tc_supported(int dtype, const ConvGeom& g) {
     return (size_t)(cmax / 64) * rows_pad * 128 + 2 * (size_t)(cmax / 64) * cmax * 128 + 1024 <= 200 * 1024;
 }
 
-void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st) {
+void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st, double useful_flops) {
     C3Args a{};
     a.x = x; a.w = wb; a.out = (__nv_bfloat16*)z; a.err = err;
     a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.C = g.ci; a.N = g.co; a.flip = 0;
     double px = (double)g.n * g.hi * g.wi;
-    launch_c3<false>(a, K_CONV3_FWD_TC, 2.0 * px * (g.ci + g.co) + 2.0 * 9 * g.ci * g.co, st);
+    launch_c3<false>(a, K_CONV3_FWD_TC, 2.0 * px * (g.ci + g.co) + 2.0 * 9 * g.ci * g.co, useful_flops, st);
 }
 
-void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st) {
+void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st,
+                       double useful_flops) {
     C3Args a{};
     a.dz = dz; a.w = wtb; a.addend = addend; a.out = (__nv_bfloat16*)dx; a.err = err;
     a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.C = g.co; a.N = g.ci; a.flip = 1;
     double px = (double)g.n * g.hi * g.wi;
     launch_c3<true>(a, K_CONV3_BWD_DATA_TC,
-                    2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci * (addend ? 2.0 : 1.0) + 2.0 * 9 * g.ci * g.co, st);
+                    2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci * (addend ? 2.0 : 1.0) + 2.0 * 9 * g.ci * g.co, useful_flops, st);
 }
 
 bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g) {
@@ -425,7 +726,7 @@ bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g) {
 }
 
 void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
-                         cudaStream_t st) {
+                         cudaStream_t st, double useful_flops) {
     W3Args a{};
     a.dz = dz; a.x = x; a.partial = scratch; a.err = err;
     a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.CI = g.ci; a.CO = g.co;
@@ -433,21 +734,14 @@ void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, 
     a.tiles_per_img = ((a.H - 1) * Wp + a.W + TM - 1) / TM;
     a.total_tiles = a.n_img * a.tiles_per_img;
     a.rows_pad = (TM + 2 * Wp + 2 + 7) / 8 * 8;
-    a.taps_per_group = 512 / a.CI < 9 ? 512 / a.CI : 9;
-    if (a.taps_per_group > 5 && a.CI == 64) a.taps_per_group = 5;      // 5 + 4 taps: two balanced groups
-    if (a.CI == 128) a.taps_per_group = 3;
+    // at most 256 accumulator columns per CTA, so that two CTAs of an SM hold their tensor memory at the same time and one
+    // stages while the other multiplies: 3 taps x 64 channels (three groups) or 2 taps x 128 channels (five groups)
+    a.taps_per_group = a.CI <= 64 ? 3 : 2;
     const int groups = (9 + a.taps_per_group - 1) / a.taps_per_group;
     a.tmem_cols = 32;
     while (a.tmem_cols < a.taps_per_group * a.CI) a.tmem_cols <<= 1;
-    static int n_sm = 0;
-    static bool attr = false;
-    if (!attr) {
-        cudaFuncSetAttribute(conv3_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-        attr = true;
-    }
+    smem_limit_once<109>(conv3_wgrad_tc_kernel, 200 * 1024);
+    const int n_sm = sm_count();
     const size_t out_elems = (size_t)a.CO * 9 * a.CI;
     int ctas = (2 * n_sm) / groups;
     if (ctas > a.total_tiles) ctas = a.total_tiles;
@@ -459,7 +753,7 @@ void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, 
     double px = (double)g.n * g.hi * g.wi;
     {
         LaunchScope ls(K_CONV3_BWD_WEIGHT_TC, 2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci + 4.0 * out_elems * ctas,
-                       2.0 * 9.0 * px * g.ci * g.co, st);
+                       useful_flops > 0 ? useful_flops : 2.0 * 9.0 * px * g.ci * g.co, st);
         launch_pdl(conv3_wgrad_tc_kernel, dim3(ctas, groups), C3_THREADS, smem, st, a);
     }
     LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);

@@ -256,8 +256,7 @@ __global__ void pad_weights_kernel(const float* __restrict__ w, int co, int K, i
         const int ko = i / Kp, kk = i - ko * Kp;
         wpad[i] = __float2bfloat16_rn(kk < K ? w[(size_t)ko * K + kk] : 0.f);
     }
-    __threadfence();          // other kernels stage these weights before their dependency wait
-    pdl_launch();
+    // no early release of the dependents: other kernels stage these weights before their dependency wait (see refresh_kernel)
 }
 
 // gw[ko][kk] = gpad[ko][kk], kk < K
@@ -308,7 +307,7 @@ void conv_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValS
     a.M = g.co; a.N = g.k * g.k * g.ci; a.K = g.n * g.ho * g.wo;
     int tiles = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
     size_t out_elems = (size_t)a.M * a.N;
-    int splits = (4 * 148 + tiles - 1) / tiles;
+    int splits = (4 * sm_count() + tiles - 1) / tiles;
     int max_by_k = (a.K + 4 * BK - 1) / (4 * BK);
     if (splits > max_by_k) splits = max_by_k;
     size_t cap = scratch_floats / out_elems;

@@ -254,7 +254,7 @@ __global__ void __launch_bounds__(128) dw_roll_kernel(int n_img, int h, int w, i
     constexpr int NIN = TWR + 2;
     extern __shared__ float wsm[];            // [9][c], tap order already flipped for the adjoint
     // the weights are not written by the previous kernel in the stream (only the refresh kernel writes them, and it
-    // releases its dependents after its stores): staging them overlaps that kernel's tail
+    // never releases its dependents before it has completed): staging them overlaps that kernel's tail
     for (int i = threadIdx.x; i < 9 * c; i += blockDim.x) {
         int t = i / c, ch = i - t * c;
         wsm[i] = __ldg(w9c + (FLIP ? 8 - t : t) * c + ch);
@@ -1102,9 +1102,9 @@ void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc
     if (g.stride == 1) {
         // Long items (whole image columns when the batch gives enough of them) keep the prefetch
         // ring full; all blocks are resident at once, so there is no partial last wave.
-        const size_t resident = 3 * 148;
+        const size_t resident = 3 * (size_t)sm_count();
         int th = g.ho;
-        while (th > 7 && (size_t)g.n * ((g.ho + th - 1) / th) * sw * gx < (size_t)rows * 2 * 148) th = (th + 1) / 2;
+        while (th > 7 && (size_t)g.n * ((g.ho + th - 1) / th) * sw * gx < (size_t)rows * 2 * sm_count()) th = (th + 1) / 2;
         const size_t n_items = (size_t)g.n * ((g.ho + th - 1) / th) * sw;
         by = (n_items + rows - 1) / rows;
         if (by * gx > resident) by = resident / gx;
@@ -1126,7 +1126,7 @@ void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc
         const int th = g.ho >= 28 ? 8 : (g.ho >= 14 ? 7 : g.ho);      // rows of dz per work item
         const int nrc = (g.ho + th - 1) / th;
         const size_t n_items = (size_t)g.n * nrc * sw;
-        by = (8 * 148 + gx - 1) / gx;
+        by = (8 * sm_count() + gx - 1) / gx;
         const size_t max_by = (n_items + (size_t)rows - 1) / (size_t)rows;
         if (by > max_by) by = max_by;
         if (by > cap) by = cap;
@@ -1155,9 +1155,9 @@ bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc&
     const int sw = (g.wo + TWR - 1) / TWR;
     const size_t n_items = (size_t)g.n * sw;
     // whole image columns per thread: worth it only when that still gives every SM a few warps
-    if (n_items * gx < (size_t)rows * 2 * 148) return false;
+    if (n_items * gx < (size_t)rows * 2 * sm_count()) return false;
     const size_t cap = scratch_floats / ((size_t)9 * g.ci);
-    const size_t resident = 3 * 148;              // three blocks per SM: all blocks run at once, no partial last wave
+    const size_t resident = 3 * (size_t)sm_count();              // three blocks per SM: all blocks run at once, no partial last wave
     size_t by = (n_items + rows - 1) / rows;
     if (by * gx > resident) by = resident / gx;
     if (by > cap) by = cap;
@@ -1165,12 +1165,8 @@ bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc&
     const size_t ipb = (n_items + by - 1) / by;
     by = (n_items + ipb - 1) / ipb;
     const size_t smem = (((size_t)9 * cw * V * 4 + 15) & ~(size_t)15) + (size_t)D * NL * 128 * 8;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-        cudaFuncSetAttribute(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-        attr_set = true;
-    }
+    smem_limit_once<201>(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, true>, 96 * 1024);
+    smem_limit_once<202>(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, false>, 96 * 1024);
     double e = (double)g.n * g.hi * g.wi * g.ci;
     {
         LaunchScope ls(K_DW_BWD_FUSED, grad_src_bytes(dz, e, dtype) + e * 2.0 * (addend ? 3.0 : 2.0) + 36.0 * g.ci * (by + 1), 36.0 * e, st);

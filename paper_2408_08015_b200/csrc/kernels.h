@@ -4,6 +4,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace ast {
@@ -37,6 +39,19 @@ inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute is per device; TAG makes the bookkeeping
+// unique per call site).
+template <int TAG, typename K> inline void smem_limit_once(K* kernel, int bytes) {
+    static std::atomic<unsigned long long> done{0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(done.load(std::memory_order_acquire) & bit)) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        done.fetch_or(bit, std::memory_order_release);
+    }
+}
+
 // Brackets one kernel launch: counts it and, while a trace is active, records a CUDA event on
 // `st` before and after it together with the bytes the kernel must move (each tensor once)
 // and its floating-point operations.
@@ -47,6 +62,8 @@ struct LaunchScope {
     cudaStream_t st;
 };
 uint64_t launches();
+// number of multiprocessors of the calling thread's current device (queried once per device)
+int sm_count();
 // true while a per-launch event trace is being recorded
 bool tracing();
 // records `msg` as the calling thread's last error and returns `code`
@@ -97,12 +114,14 @@ void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, flo
 
 // ---- dense 3x3 conv (stride 1, pad 1, channels multiples of 64) on tcgen05 ----
 bool conv3_tc_supported(int dtype, const ConvGeom& g);
-// wb: bf16 weights [co][3][3][ci]; wtb: bf16 derived weights [ci][3][3][co]
-void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st);
-void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st);
+// wb: bf16 weights [co][3][3][ci]; wtb: bf16 derived weights [ci][3][3][co].  useful_flops > 0 replaces the operation count the
+// trace records (a stride-2 layer evaluated on its input grid executes four times the multiply-adds of its definition).
+void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st, double useful_flops = 0);
+void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st,
+                       double useful_flops = 0);
 bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g);
 void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
-                         cudaStream_t st);
+                         cudaStream_t st, double useful_flops = 0);
 
 // ---- depthwise 3x3 (weights tap-major: w9c[r*3+s][c]) ----
 // With `pivot` and `partial` given, the stride-1 kernel also writes the BatchNorm statistics partials of its output

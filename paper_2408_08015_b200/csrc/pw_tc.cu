@@ -75,30 +75,53 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
         const int kc = min(a.KC, a.K - k0);           // multiple of 8
         const int vpr = kc >> 3;                      // 16-byte vectors per row holding data
         const int vpr_pad = ((kc + 15) >> 4) << 1;    // rounded up to whole MMA k-steps
-        // ---- stage A: [128 pixels][kc] ----
-        for (int v = tid; v < TM * vpr_pad; v += NTHREADS) {
-            int r = v / vpr_pad, j = v - r * vpr_pad;
-            int p = p0 + r;
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (p < a.P && j < vpr) {
-                float f[8];
-                int c0 = k0 + (j << 3);
-                if (BWD) {
-                    ld_grad_vec<__nv_bfloat16>(a.dz, ((size_t)p * a.K + c0) >> 3, c0, f);
-                } else {
+        // ---- stage A: [128 pixels][kc].  The global loads of four vectors per thread are issued together before any is
+        // transformed, so that their latencies overlap instead of adding up. ----
+        constexpr int U = 4;
+        const bool need_z = BWD && grad_needs_z(a.dz);
+        const int items = TM * vpr_pad;
+        for (int v0 = tid; v0 < items; v0 += U * NTHREADS) {
+            Vec<__nv_bfloat16> raw[U], rawz[U];
+            bool ok[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * NTHREADS;
+                const int r = v / vpr_pad, j = v - r * vpr_pad;
+                const int p = p0 + r;
+                ok[u] = v < items && p < a.P && j < vpr;
+                raw[u].raw = rawz[u].raw = make_uint4(0, 0, 0, 0);
+                if (ok[u]) {
+                    const int c0 = k0 + (j << 3);
                     size_t pin = p;
-                    if (a.stride > 1) {
+                    if (!BWD && a.stride > 1) {
                         int wo = p % a.wo, t = p / a.wo;
                         int ho = t % a.ho, n = t / a.ho;
                         pin = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
                     }
-                    ld_val_vec<__nv_bfloat16>(a.x, (pin * a.K + c0) >> 3, c0, f);
+                    const size_t e = (pin * a.K + c0) >> 3;
+                    raw[u].load(BWD ? a.dz.dy : a.x.p, e);
+                    if (need_z) rawz[u].load(a.dz.z, e);
                 }
-                q = pack8(f);
             }
-            *reinterpret_cast<uint4*>(sA + tile_off(r, j, TM)) = q;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * NTHREADS;
+                if (v < items) {
+                    const int r = v / vpr_pad, j = v - r * vpr_pad;
+                    uint4 q = make_uint4(0, 0, 0, 0);
+                    if (ok[u]) {
+                        float f[8];
+                        const int c0 = k0 + (j << 3);
+                        if (BWD) grad_from_raw<__nv_bfloat16>(a.dz, raw[u], rawz[u], c0, f);
+                        else val_from_raw<__nv_bfloat16>(a.x, raw[u], c0, f);
+                        q = pack8(f);
+                    }
+                    *reinterpret_cast<uint4*>(sA + tile_off(r, j, TM)) = q;
+                }
+            }
         }
         // ---- stage B: [NT channels][kc] of the bf16 weights ----
+#pragma unroll 4
         for (int v = tid; v < NT * vpr_pad; v += NTHREADS) {
             int r = v / vpr_pad, j = v - r * vpr_pad;
             int n = n0 + r;
@@ -255,34 +278,73 @@ __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArg
             break;
         }
         const int valid = min(WSTAGE, pend - ps);
-        for (int v = tid; v < WSTAGE * ca; v += NTHREADS) {
-            int kr = v / ca, j = v - kr * ca;
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (kr < valid) {
-                float f[8];
-                int c0 = m0 + (j << 3);
-                ld_grad_vec<__nv_bfloat16>(a.dz, ((size_t)(ps + kr) * a.CO + c0) >> 3, c0, f);
-                q = pack8(f);
-            }
-            *reinterpret_cast<uint4*>(sA + (j >> 3) * PANEL + kr * 128 + (((j & 7) ^ (kr & 7)) << 4)) = q;
-        }
-        for (int v = tid; v < WSTAGE * cb; v += NTHREADS) {
-            int kr = v / cb, j = v - kr * cb;
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (kr < valid) {
-                float f[8];
-                int c0 = n0 + (j << 3);
-                size_t pin = ps + kr;
-                if (a.stride > 1) {
-                    int p = ps + kr;
-                    int wo = p % a.wo, t = p / a.wo;
-                    int ho = t % a.ho, n = t / a.ho;
-                    pin = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
+        // both operands: the loads of four vectors per thread are issued together before any is transformed
+        constexpr int U = 4;
+        const bool need_z = grad_needs_z(a.dz);
+        for (int v0 = tid; v0 < WSTAGE * ca; v0 += U * NTHREADS) {
+            Vec<__nv_bfloat16> raw[U], rawz[U];
+            bool ok[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * NTHREADS;
+                const int kr = v / ca, j = v - kr * ca;
+                ok[u] = v < WSTAGE * ca && kr < valid;
+                raw[u].raw = rawz[u].raw = make_uint4(0, 0, 0, 0);
+                if (ok[u]) {
+                    const size_t e = ((size_t)(ps + kr) * a.CO + m0 + (j << 3)) >> 3;
+                    raw[u].load(a.dz.dy, e);
+                    if (need_z) rawz[u].load(a.dz.z, e);
                 }
-                ld_val_vec<__nv_bfloat16>(a.x, (pin * a.CI + c0) >> 3, c0, f);
-                q = pack8(f);
             }
-            *reinterpret_cast<uint4*>(sB + (j >> 3) * PANEL + kr * 128 + (((j & 7) ^ (kr & 7)) << 4)) = q;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * NTHREADS;
+                if (v < WSTAGE * ca) {
+                    const int kr = v / ca, j = v - kr * ca;
+                    uint4 q = make_uint4(0, 0, 0, 0);
+                    if (ok[u]) {
+                        float f[8];
+                        grad_from_raw<__nv_bfloat16>(a.dz, raw[u], rawz[u], m0 + (j << 3), f);
+                        q = pack8(f);
+                    }
+                    *reinterpret_cast<uint4*>(sA + (j >> 3) * PANEL + kr * 128 + (((j & 7) ^ (kr & 7)) << 4)) = q;
+                }
+            }
+        }
+        for (int v0 = tid; v0 < WSTAGE * cb; v0 += U * NTHREADS) {
+            Vec<__nv_bfloat16> raw[U];
+            bool ok[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * NTHREADS;
+                const int kr = v / cb, j = v - kr * cb;
+                ok[u] = v < WSTAGE * cb && kr < valid;
+                raw[u].raw = make_uint4(0, 0, 0, 0);
+                if (ok[u]) {
+                    size_t pin = ps + kr;
+                    if (a.stride > 1) {
+                        int p = ps + kr;
+                        int wo = p % a.wo, t = p / a.wo;
+                        int ho = t % a.ho, n = t / a.ho;
+                        pin = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
+                    }
+                    raw[u].load(a.x.p, (pin * a.CI + n0 + (j << 3)) >> 3);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * NTHREADS;
+                if (v < WSTAGE * cb) {
+                    const int kr = v / cb, j = v - kr * cb;
+                    uint4 q = make_uint4(0, 0, 0, 0);
+                    if (ok[u]) {
+                        float f[8];
+                        val_from_raw<__nv_bfloat16>(a.x, raw[u], n0 + (j << 3), f);
+                        q = pack8(f);
+                    }
+                    *reinterpret_cast<uint4*>(sB + (j >> 3) * PANEL + kr * 128 + (((j & 7) ^ (kr & 7)) << 4)) = q;
+                }
+            }
         }
         fence_async_smem();
         __syncthreads();
@@ -366,66 +428,6 @@ __global__ void reduce_splits_tc(const float* __restrict__ partial, int splits, 
 // shared memory.  Every wait is bounded; a wait that runs out raises a CTA-wide abort flag, every
 // role leaves its loop, outstanding bulk copies are waited for, tensor memory is freed and the
 // error word is set.
-// Branch-free operand transforms with per-thread register coefficients.  Absent BatchNorm
-// terms take neutral values (scale 1, shift 0, k1 1, k2 = k3 0) and the activation becomes a pair
-// of bounds (ReLU6: 0..6, ReLU: 0..inf, none: -inf..inf), so that every lane runs the same
-// instruction stream whatever its operand.
-struct XfVal {
-    float cs[8], ch[8], lo, hi;
-    __device__ __forceinline__ void init(const ValSrc& s, int c0) {
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            cs[q] = s.scale ? __ldg(s.scale + c0 + q) : 1.f;
-            ch[q] = s.scale ? __ldg(s.shift + c0 + q) : 0.f;
-        }
-        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
-        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
-    }
-    __device__ __forceinline__ uint4 apply(const uint4& raw) const {
-        Vec<__nv_bfloat16> v;
-        v.raw = raw;
-        float f[8];
-        v.unpack(f);
-#pragma unroll
-        for (int q = 0; q < 8; ++q) f[q] = fminf(fmaxf(fmaf(f[q], cs[q], ch[q]), lo), hi);
-        return pack8(f);
-    }
-};
-struct XfGrad {
-    float cs[8], ch[8], k1[8], k2[8], k3[8], lo, hi;
-    __device__ __forceinline__ void init(const GradSrc& s, int c0) {
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            cs[q] = s.scale ? __ldg(s.scale + c0 + q) : 1.f;
-            ch[q] = s.scale ? __ldg(s.shift + c0 + q) : 0.f;
-            k1[q] = s.k1 ? __ldg(s.k1 + c0 + q) : 1.f;
-            k2[q] = s.k1 ? __ldg(s.k2 + c0 + q) : 0.f;
-            k3[q] = s.k1 ? __ldg(s.k3 + c0 + q) : 0.f;
-        }
-        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
-        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
-    }
-    __device__ __forceinline__ uint4 apply(const uint4& rawdy, const uint4& rawz) const {
-        Vec<__nv_bfloat16> v;
-        float f[8], z[8];
-        v.raw = rawdy;
-        v.unpack(f);
-        v.raw = rawz;
-        v.unpack(z);
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            // lo < pre < hi  <=>  (pre - lo) * (hi - pre) > 0: differences of floats keep their sign
-            // exactly, infinite bounds give +inf, and 0 * inf = NaN compares false (pre == 0 under ReLU);
-            // the test runs on the FMA pipe and guards one predicated fused multiply-add
-            const float pre = fmaf(z[q], cs[q], ch[q]);
-            float o = fmaf(k3[q], z[q], k2[q]);
-            if ((pre - lo) * (hi - pre) > 0.f) o = fmaf(k1[q], f[q], o);
-            f[q] = o;
-        }
-        return pack8(f);
-    }
-};
-
 constexpr int PIPE_THREADS = 448;     // producer, MMA issuer, 8 transform warps, 4 epilogue warps
 constexpr int PIPE_XF = 256;          // transform threads
 constexpr int MAX_RAW = 8;
@@ -460,7 +462,7 @@ struct PipeArgs {
 // parameter because even a never-taken branch around those loads slows the epilogue's inner loop.
 template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const PipeArgs a) {
     // Set-up that reads nothing the previous kernel in the stream writes (barriers, tensor memory, the resident
-    // weights: written only by the refresh kernel, which releases its dependents after its stores) runs before
+    // weights: written only by the refresh kernel, which never releases its dependents before it has completed) runs before
     // the dependency wait and so overlaps the previous kernel's tail.
     pdl_launch();
     extern __shared__ uint8_t smem_raw[];
@@ -868,16 +870,9 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
 }
 
 template <bool BWD> int launch_pipe(PipeArgs& a, size_t smem, int kind, double bytes, size_t partial_floats, cudaStream_t st) {
-    static bool attr_set = false;
-    static int n_sm = 0;
-    if (!attr_set) {
-        cudaFuncSetAttribute(pw_pipe_kernel<BWD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
-        cudaFuncSetAttribute(pw_pipe_kernel<BWD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-        attr_set = true;
-    }
+    smem_limit_once<101>(pw_pipe_kernel<BWD, false>, 222 * 1024);
+    smem_limit_once<102>(pw_pipe_kernel<BWD, true>, 222 * 1024);
+    const int n_sm = sm_count();
     int grid = a.tiles < n_sm ? a.tiles : n_sm;
     if (a.stat_partial && (size_t)grid * 2 * a.N > partial_floats) a.stat_partial = nullptr;
     if (a.r_partial && (size_t)grid * 2 * a.N > partial_floats) a.r_partial = nullptr;
@@ -1165,6 +1160,11 @@ Tiling pick_tiling(int K, int N) {
     t.KC = kpad < 256 ? kpad : 256;
     t.tmem_cols = 32;
     while (t.tmem_cols < t.NT) t.tmem_cols <<= 1;
+    // One tile per CTA, so the phases of a tile (load, multiply, store) overlap only across the CTAs of an SM: keep the
+    // staged reduction chunk small enough for three of them (or as many as the tensor-memory columns allow).
+    const int want = 512 / t.tmem_cols < 3 ? 512 / t.tmem_cols : 3;
+    while (t.KC > KB && ((size_t)(t.KC / KB) * (TM + t.NT) * 128 + 1024) * want > 220 * 1024) t.KC >>= 1;
+    t.KC = (t.KC + KB - 1) / KB * KB;
     t.smem = (size_t)(t.KC / KB) * (TM + t.NT) * 128 + 1024;
     return t;
 }
@@ -1172,11 +1172,7 @@ Tiling pick_tiling(int K, int N) {
 template <bool BWD> void launch(const PwArgs& a0, const Tiling& t, int kind, double bytes, cudaStream_t st) {
     PwArgs a = a0;
     a.NT = t.NT; a.KC = t.KC; a.tmem_cols = t.tmem_cols;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(pw_tc_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_set = true;
-    }
+    smem_limit_once<103>(pw_tc_kernel<BWD>, 200 * 1024);
     LaunchScope ls(kind, bytes, 2.0 * a.P * a.N * a.K, st);
     dim3 grid((a.P + TM - 1) / TM, t.ntiles);
     launch_pdl(pw_tc_kernel<BWD>, grid, NTHREADS, t.smem, st, a);
@@ -1252,15 +1248,8 @@ int pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wt
 void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                       cudaStream_t st) {
     if (g.stride == 1) {
-        static int n_sm = 0;
-        static bool attr = false;
-        if (!attr) {
-            cudaFuncSetAttribute(pw_wgrad_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024);
-            int dev = 0;
-            cudaGetDevice(&dev);
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-            attr = true;
-        }
+        smem_limit_once<104>(pw_wgrad_pipe_kernel, 222 * 1024);
+        const int n_sm = sm_count();
         WgArgs wa{};
         wa.dz = dz; wa.x = x; wa.partial = scratch; wa.gw = gw; wa.err = err;
         wa.P = g.n * g.ho * g.wo; wa.CO = g.co; wa.CI = g.ci;
@@ -1290,7 +1279,7 @@ void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, flo
     while (a.tmem_cols < a.NT) a.tmem_cols <<= 1;
     int mtiles = (a.CO + TM - 1) / TM;
     size_t out_elems = (size_t)a.CO * a.CI;
-    int splits = (2 * 148 + mtiles * ntiles - 1) / (mtiles * ntiles);
+    int splits = (2 * sm_count() + mtiles * ntiles - 1) / (mtiles * ntiles);
     int max_by_pix = (a.P + 4 * WSTAGE - 1) / (4 * WSTAGE);
     if (splits > max_by_pix) splits = max_by_pix;
     size_t cap = scratch_floats / out_elems;
@@ -1301,11 +1290,7 @@ void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, flo
     splits = (a.P + ppc - 1) / ppc;
     a.pix_per_cta = ppc;
     size_t smem = (size_t)2 * (2 + (a.NT + 63) / 64) * PANEL + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(pw_bwd_weight_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_set = true;
-    }
+    smem_limit_once<105>(pw_bwd_weight_tc_kernel, 200 * 1024);
     double bytes = 2.0 * (double)a.P * a.CO * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * (double)g.n * g.hi * g.wi * a.CI +
                    4.0 * out_elems * splits;
     {

@@ -65,6 +65,9 @@ struct Unit {
     int col_kp = 0;
     size_t col_off = 0;     // bytes into a slot
     size_t wpad_off = 0;    // elements into the padded bf16 weight arena
+    // stride-2 3x3 conv on the stride-1 tensor-core kernels: bytes into the arena of zero-inserted output gradients (one
+    // buffer per such unit: the weight-gradient kernel reads it on the second stream while the pass goes on), -1 = none
+    long up_off = -1;
 };
 
 struct Timing {
@@ -99,6 +102,8 @@ struct asteroid_stage {
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     float* scratch_side = nullptr;
+    char* up_mem = nullptr;                        // zero-inserted gradients of the stride-2 3x3 units
+    size_t up_bytes = 0;
     char *slot_mem = nullptr, *grad_mem = nullptr;
     size_t slot_bytes = 0, slot_stat_off = 0, grad_bytes = 0, scratch_floats = 0;
     size_t bytes_mod = 0, bytes_opt = 0, bytes_work = 0;
@@ -328,7 +333,7 @@ static void free_stage(asteroid_stage* s) {
     for (auto e : s->tm.ev) cudaEventDestroy(e);
     cudaFree(s->w); cudaFree(s->v); cudaFree(s->G); cudaFree(s->g); cudaFree(s->derived); cudaFree(s->run);
     cudaFree(s->coef); cudaFree(s->scratch); cudaFree(s->perm); cudaFree(s->slot_mem); cudaFree(s->grad_mem);
-    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err); cudaFree(s->scratch_side); cudaFree(s->wpad); cudaFree(s->gpad);
+    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err); cudaFree(s->scratch_side); cudaFree(s->wpad); cudaFree(s->gpad); cudaFree(s->up_mem);
     if (s->ev_fork) cudaEventDestroy(s->ev_fork);
     if (s->ev_join) cudaEventDestroy(s->ev_join);
     if (s->side) cudaStreamDestroy(s->side);
@@ -380,6 +385,8 @@ static bool conv3_s2_tc_supported(const asteroid_stage* s, const Unit& u) {
     const size_t full = (size_t)u.g.n * u.g.hi * u.g.wi * std::max(u.g.ci, u.g.co) * 2;
     return full <= s->scratch_floats * sizeof(float);
 }
+
+static double conv_flops(const ConvGeom& g) { return 2.0 * g.n * g.ho * g.wo * (double)g.co * g.k * g.k * g.ci; }
 
 // geometry of the pointwise GEMM that stands for an im2col unit
 static ConvGeom col_geom(const Unit& u) {
@@ -443,7 +450,7 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
                                         bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
             else if (conv3_tc_supported(dt, u.g)) conv3_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, obuf, s->err, st);
             else if (conv3_s2_tc_supported(s, u)) {
-                conv3_fwd_tc(s1_geom(u), val_src(s, sv, u.in), s->wb + u.w_off, s->scratch, s->err, st);
+                conv3_fwd_tc(s1_geom(u), val_src(s, sv, u.in), s->wb + u.w_off, s->scratch, s->err, st, conv_flops(u.g));
                 ew_subsample2(s->scratch, u.g.n, u.g.hi, u.g.wi, u.g.ho, u.g.wo, u.g.co, obuf, st);
             }
             else conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, bias, obuf, st);
@@ -576,11 +583,19 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                     continue;
                 }
             }
+            const bool s2_tc = u.kind == U_CONV && u.up_off >= 0;
+            void* up = s2_tc ? s->up_mem + u.up_off : nullptr;
+            // stride 2 on the stride-1 kernels: the zero-inserted output gradient (BatchNorm / activation backward applied
+            // on the way) serves both the weight gradient and the input gradient
+            if (s2_tc) ew_upsample2_grad(d, u.g.n, u.g.hi, u.g.wi, u.g.ho, u.g.wo, u.g.co, up, st);
+            const GradSrc dup{up, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, ACT_NONE};
             {
                 int frc = fork();
                 if (frc) return frc;
             }
-            if (u.kind == U_CONV && u.col_kp) {
+            if (s2_tc && conv3_wgrad_tc_supported(dt, s1_geom(u)))
+                conv3_bwd_weight_tc(s1_geom(u), dup, xin, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst, conv_flops(u.g));
+            else if (u.kind == U_CONV && u.col_kp) {
                 pw_bwd_weight_tc(col_geom(u), d, ValSrc{sv.base + u.col_off, nullptr, nullptr, ACT_NONE}, wscratch, s->scratch_floats, s->gpad, s->err, wst);
                 conv_unpad_grad(s->gpad, u.g.co, u.g.k * u.g.k * u.g.ci, u.col_kp, s->g + u.w_off, wst);
             } else if (u.kind == U_CONV && pw_tc_supported(dt, u.g, false))
@@ -614,11 +629,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                         reduced[tgt] = 1;
                     }
                 } else if (u.kind == U_CONV && conv3_tc_supported(dt, u.g)) conv3_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
-                else if (u.kind == U_CONV && conv3_s2_tc_supported(s, u)) {
-                    ew_upsample2_grad(d, u.g.n, u.g.hi, u.g.wi, u.g.ho, u.g.wo, u.g.co, s->scratch, st);
-                    conv3_bwd_data_tc(s1_geom(u), GradSrc{s->scratch, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, ACT_NONE}, s->wtb + u.w_off, addend,
-                                      own(u.in), s->err, st);
-                }
+                else if (s2_tc) conv3_bwd_data_tc(s1_geom(u), dup, s->wtb + u.w_off, addend, own(u.in), s->err, st, conv_flops(u.g));
                 else if (u.kind == U_CONV) conv_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 else dw_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 gi.state = G_OWNED;
@@ -697,6 +708,12 @@ static int create_impl(const ast_layer* net, int n_layers, int first, int last, 
         if (u.kind == U_CONV) s->scratch_floats = std::max(s->scratch_floats, (size_t)4 * u.g.co * u.g.k * u.g.k * u.g.ci);
     if ((rc = dev_alloc(&s->scratch, s->scratch_floats * 4, &work))) return rc;
     if ((rc = dev_alloc(&s->scratch_side, s->scratch_floats * 4, &work))) return rc;
+    for (auto& u : s->units)
+        if (conv3_s2_tc_supported(s, u)) {
+            u.up_off = (long)s->up_bytes;
+            s->up_bytes += align_up((size_t)u.g.n * u.g.hi * u.g.wi * u.g.co * 2, 256);
+        }
+    if (s->up_bytes && (rc = dev_alloc(&s->up_mem, s->up_bytes, &work))) return rc;
     CU(cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking));
     CU(cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming));
     CU(cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming));

@@ -183,6 +183,65 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Branch-free operand transforms with per-thread register coefficients.  Absent BatchNorm
+// terms take neutral values (scale 1, shift 0, k1 1, k2 = k3 0) and the activation becomes a pair
+// of bounds (ReLU6: 0..6, ReLU: 0..inf, none: -inf..inf), so that every lane runs the same
+// instruction stream whatever its operand.
+struct XfVal {
+    float cs[8], ch[8], lo, hi;
+    __device__ __forceinline__ void init(const ValSrc& s, int c0) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            cs[q] = s.scale ? __ldg(s.scale + c0 + q) : 1.f;
+            ch[q] = s.scale ? __ldg(s.shift + c0 + q) : 0.f;
+        }
+        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
+        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
+    }
+    __device__ __forceinline__ uint4 apply(const uint4& raw) const {
+        Vec<__nv_bfloat16> v;
+        v.raw = raw;
+        float f[8];
+        v.unpack(f);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) f[q] = fminf(fmaxf(fmaf(f[q], cs[q], ch[q]), lo), hi);
+        return pack8(f);
+    }
+};
+struct XfGrad {
+    float cs[8], ch[8], k1[8], k2[8], k3[8], lo, hi;
+    __device__ __forceinline__ void init(const GradSrc& s, int c0) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            cs[q] = s.scale ? __ldg(s.scale + c0 + q) : 1.f;
+            ch[q] = s.scale ? __ldg(s.shift + c0 + q) : 0.f;
+            k1[q] = s.k1 ? __ldg(s.k1 + c0 + q) : 1.f;
+            k2[q] = s.k1 ? __ldg(s.k2 + c0 + q) : 0.f;
+            k3[q] = s.k1 ? __ldg(s.k3 + c0 + q) : 0.f;
+        }
+        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
+        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
+    }
+    __device__ __forceinline__ uint4 apply(const uint4& rawdy, const uint4& rawz) const {
+        Vec<__nv_bfloat16> v;
+        float f[8], z[8];
+        v.raw = rawdy;
+        v.unpack(f);
+        v.raw = rawz;
+        v.unpack(z);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            // lo < pre < hi  <=>  (pre - lo) * (hi - pre) > 0: differences of floats keep their sign
+            // exactly, infinite bounds give +inf, and 0 * inf = NaN compares false (pre == 0 under ReLU);
+            // the test runs on the FMA pipe and guards one predicated fused multiply-add
+            const float pre = fmaf(z[q], cs[q], ch[q]);
+            float o = fmaf(k3[q], z[q], k2[q]);
+            if ((pre - lo) * (hi - pre) > 0.f) o = fmaf(k1[q], f[q], o);
+            f[q] = o;
+        }
+        return pack8(f);
+    }
+};
 
 }  // namespace tc
 }  // namespace ast

@@ -1,5 +1,6 @@
 // Launch accounting: every kernel launch of the library passes through a LaunchScope, which
 // counts it and, while a trace is active, brackets it with CUDA events on the launching stream.
+#include <atomic>
 #include <cstdio>
 #include <mutex>
 #include <vector>
@@ -37,6 +38,18 @@ const char* const kNames[K_KINDS] = {
     "dw_bwd_weight_finish", "bn_stats", "bn_stats_finish", "bn_bwd_reduce", "bn_bwd_finish", "ew_add", "ew_relu_mask", "ew_sum",
     "gap_fwd", "gap_bwd", "accumulate", "sgd_step", "refresh_derived", "loss_mse", "loss_softmax_xent", "pw_fwd_tcgen05", "pw_bwd_data_tcgen05", "pw_bwd_weight_tcgen05", "conv3x3_fwd_tcgen05", "conv3x3_bwd_data_tcgen05", "conv3x3_bwd_weight_tcgen05", "dw_bwd_fused", "conv_im2col", "conv_pad_unpad"};
 }  // namespace
+
+int sm_count() {
+    static std::atomic<int> cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n <= 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
 
 const char* kernel_name(int kind) { return (kind >= 0 && kind < K_KINDS) ? kNames[kind] : "?"; }
 uint64_t launches() { return g_launches; }
