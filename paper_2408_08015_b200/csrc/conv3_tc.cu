@@ -459,8 +459,8 @@ template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, double use
         size_t psmem = 0;
         int it = 0;
         if (plan_c3p(a, p, &psmem, &it)) {
-            smem_limit_once<106>(conv3_persist_kernel<BWD, 4>, 226 * 1024);
-            smem_limit_once<107>(conv3_persist_kernel<BWD, 8>, 226 * 1024);
+            smem_limit_once<106 + (BWD ? 50 : 0)>(conv3_persist_kernel<BWD, 4>, 226 * 1024);
+            smem_limit_once<107 + (BWD ? 50 : 0)>(conv3_persist_kernel<BWD, 8>, 226 * 1024);
             const int n_sm = sm_count();
             int nctas = n_sm / p.n_split;
             if (nctas < 1) nctas = 1;
@@ -481,7 +481,7 @@ template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, double use
     // all nine taps resident if two CTAs per SM still fit with them
     a.resident = ((size_t)kbs * a.rows_pad * 128 + 9 * (size_t)kbs * a.N * 128 + 1024 <= 110 * 1024) ? 1 : 0;
     size_t smem = (size_t)kbs * a.rows_pad * 128 + (a.resident ? 9 : 2) * (size_t)kbs * a.N * 128 + 1024;
-    smem_limit_once<108>(conv3_tc_kernel<BWD>, 200 * 1024);
+    smem_limit_once<108 + (BWD ? 50 : 0)>(conv3_tc_kernel<BWD>, 200 * 1024);
     LaunchScope ls(kind, bytes, useful_flops > 0 ? useful_flops : 2.0 * 9.0 * a.n_img * a.H * a.W * (double)a.C * a.N, st);
     launch_pdl(conv3_tc_kernel<BWD>, a.n_img * a.tiles_per_img, C3_THREADS, smem, st, a);
 }

@@ -1165,8 +1165,8 @@ bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc&
     const size_t ipb = (n_items + by - 1) / by;
     by = (n_items + ipb - 1) / ipb;
     const size_t smem = (((size_t)9 * cw * V * 4 + 15) & ~(size_t)15) + (size_t)D * NL * 128 * 8;
-    smem_limit_once<201>(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, true>, 96 * 1024);
-    smem_limit_once<202>(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, false>, 96 * 1024);
+    smem_limit_once<201 + V * 10000 + TWR * 1000 + D * 100>(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, true>, 96 * 1024);
+    smem_limit_once<202 + V * 10000 + TWR * 1000 + D * 100>(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, false>, 96 * 1024);
     double e = (double)g.n * g.hi * g.wi * g.ci;
     {
         LaunchScope ls(K_DW_BWD_FUSED, grad_src_bytes(dz, e, dtype) + e * 2.0 * (addend ? 3.0 : 2.0) + 36.0 * g.ci * (by + 1), 36.0 * e, st);

@@ -870,8 +870,8 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
 }
 
 template <bool BWD> int launch_pipe(PipeArgs& a, size_t smem, int kind, double bytes, size_t partial_floats, cudaStream_t st) {
-    smem_limit_once<101>(pw_pipe_kernel<BWD, false>, 222 * 1024);
-    smem_limit_once<102>(pw_pipe_kernel<BWD, true>, 222 * 1024);
+    smem_limit_once<101 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, false>, 222 * 1024);
+    smem_limit_once<102 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, true>, 222 * 1024);
     const int n_sm = sm_count();
     int grid = a.tiles < n_sm ? a.tiles : n_sm;
     if (a.stat_partial && (size_t)grid * 2 * a.N > partial_floats) a.stat_partial = nullptr;
@@ -1172,7 +1172,7 @@ Tiling pick_tiling(int K, int N) {
 template <bool BWD> void launch(const PwArgs& a0, const Tiling& t, int kind, double bytes, cudaStream_t st) {
     PwArgs a = a0;
     a.NT = t.NT; a.KC = t.KC; a.tmem_cols = t.tmem_cols;
-    smem_limit_once<103>(pw_tc_kernel<BWD>, 200 * 1024);
+    smem_limit_once<103 + (BWD ? 50 : 0)>(pw_tc_kernel<BWD>, 200 * 1024);
     LaunchScope ls(kind, bytes, 2.0 * a.P * a.N * a.K, st);
     dim3 grid((a.P + TM - 1) / TM, t.ntiles);
     launch_pdl(pw_tc_kernel<BWD>, grid, NTHREADS, t.smem, st, a);
