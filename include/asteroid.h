@@ -137,7 +137,11 @@ int asteroid_stage_step(asteroid_stage* s, float lr, float momentum, void* strea
 /* Per-layer cost record at batch size `batch` (Section 3.3: FP/BP time of each layer for various
  * batch sizes, output size and weight size in bytes).  Runs the stage's own kernels on zero-filled
  * buffers of that batch size (3 warm-up + 7 timed rounds, CUDA events), synchronises.
- * `layer` is an index in [first,last]. */
+ * `layer` is an index in [first,last].  The timed launch plan is the one a round uses (BatchNorm
+ * statistics and backward sums taken inside the neighbouring kernels wherever the round does so),
+ * except that every kernel stays on one stream, so that a layer's time is that of its own kernels.
+ * A BatchNorm whose sums were taken by another layer's kernel reports only its finishing kernel
+ * (alg_bytes of a few kB, or 0) and names that layer in fused_into. */
 int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_profile* out);
 
 /* Loss heads (used by the last stage and by tests).  All pointers are DEVICE pointers.
@@ -154,7 +158,9 @@ int asteroid_loss_mse(const void* y, const void* target, size_t n, int dtype, vo
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress) with
  *    that device current; make that first call before starting any stream capture.
  *  - All calls on a device share the one array: each call clears the ticket word on `stream` before
- *    its kernel, and two calls whose kernels may overlap on the GPU (different streams) race. */
+ *    its kernel, and two calls whose kernels may overlap on the GPU (different streams) race.
+ *  - Concurrent first calls on one device from several host threads are safe (each stores the same address).
+ *    Device ordinals of 64 and above are refused with AST_ERR_ARG. */
 int asteroid_loss_mse_noalloc(const void* y, const void* target, size_t n, int dtype, void* dy, float* loss, void* stream);
 /* Softmax cross-entropy: *loss = mean_r(-log softmax(logits_r)[labels_r]),
  * dlogits = (softmax - onehot) / rows.  rows <= 65536. */
@@ -176,6 +182,14 @@ typedef struct {
 } ast_kernel_stat;
 int asteroid_trace_start(void);
 int asteroid_trace_stop(ast_kernel_stat* out, int capacity, int* n_out);
+
+/* Self-test of the bounded device-side waits (the paper has no counterpart).  Every hand-off wait inside the
+ * tensor-core kernels gives up after a fixed number of polls, sets the stage's error word and lets the kernel
+ * return, which export_state then reports as AST_ERR_TIMEOUT.  This call runs that mechanism on purpose: one
+ * warp waits 1024 polls on a barrier at which nobody arrives.  Returns AST_ERR_TIMEOUT when the wait gave up and
+ * the kernel returned (the expected outcome), AST_OK if the wait reported success, AST_ERR_CUDA on a runtime
+ * error.  Synchronises the device; the context stays usable. */
+int asteroid_selftest_bounded_wait(void);
 
 /* Count of kernel launches this library has enqueued in the calling process. */
 uint64_t asteroid_launch_count(void);

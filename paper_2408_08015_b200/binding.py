@@ -14,7 +14,7 @@ EXPORTS = ["asteroid_stage_create", "asteroid_stage_destroy", "asteroid_stage_pa
            "asteroid_stage_export_bn_running", "asteroid_stage_forward", "asteroid_stage_backward",
            "asteroid_stage_accumulate", "asteroid_stage_step", "asteroid_stage_profile",
            "asteroid_loss_mse", "asteroid_loss_mse_noalloc", "asteroid_loss_softmax_xent", "asteroid_trace_start", "asteroid_trace_stop",
-           "asteroid_launch_count", "asteroid_last_error"]
+           "asteroid_selftest_bounded_wait", "asteroid_launch_count", "asteroid_last_error"]
 
 
 class ast_layer(C.Structure):
@@ -76,6 +76,7 @@ def lib():
         L.asteroid_loss_softmax_xent.argtypes = [vp, vp, i, i, i, vp, vp, vp]
         L.asteroid_trace_start.argtypes = []
         L.asteroid_trace_stop.argtypes = [C.POINTER(ast_kernel_stat), i, C.POINTER(i)]
+        L.asteroid_selftest_bounded_wait.argtypes = []
         L.asteroid_launch_count.argtypes = []
         L.asteroid_launch_count.restype = C.c_uint64
         L.asteroid_last_error.argtypes = []
@@ -185,6 +186,11 @@ def asteroid_trace_stop():
     _check(lib().asteroid_trace_stop(buf, 64, C.byref(n)))
     return [{"name": buf[j].name.decode(), "launches": buf[j].launches, "total_ms": buf[j].total_ms,
              "alg_bytes": buf[j].alg_bytes, "flops": buf[j].flops} for j in range(n.value)]
+
+
+def asteroid_selftest_bounded_wait():
+    """Return code of the bounded-wait self-test (AST_ERR_TIMEOUT is the expected outcome); does not raise."""
+    return lib().asteroid_selftest_bounded_wait()
 
 
 def asteroid_launch_count():

@@ -734,7 +734,9 @@ extern "C" int asteroid_loss_mse_noalloc(const void* y, const void* target, size
     if (n > NOALLOC_MAX_ELEMS)
         return report_error(-1, "asteroid_loss_mse_noalloc: n exceeds the 67108864-element limit of the allocation-free variant; use asteroid_loss_mse");
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return report_error(-5, "asteroid_loss_mse_noalloc: cudaGetDevice failed");
+    if (cudaGetDevice(&dev) != cudaSuccess) return report_error(-5, "asteroid_loss_mse_noalloc: cudaGetDevice failed");
+    if (dev < 0 || dev >= 64) return report_error(-1, "asteroid_loss_mse_noalloc: device ordinals of 64 and above are not supported");
+    // two host threads making the first call on a device at once both look up and store the same address: harmless
     if (!g_noalloc_ptr[dev]) {
         float* p = nullptr;
         cudaError_t e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);

@@ -179,4 +179,7 @@ void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float
 void loss_xent(int dtype, const void* logits, const int32_t* labels, int rows, int classes, void* dlogits, float* loss,
                float* scratch, cudaStream_t st);
 
+// one warp waits `limit` polls on an mbarrier nobody arrives at; sets *err = 1 when the wait gave up
+void launch_bounded_wait_probe(int* err, unsigned limit, cudaStream_t st);
+
 }  // namespace ast

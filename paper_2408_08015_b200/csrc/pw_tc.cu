@@ -428,8 +428,8 @@ __global__ void reduce_splits_tc(const float* __restrict__ partial, int splits, 
 // shared memory.  Every wait is bounded; a wait that runs out raises a CTA-wide abort flag, every
 // role leaves its loop, outstanding bulk copies are waited for, tensor memory is freed and the
 // error word is set.
-constexpr int PIPE_THREADS = 448;     // producer, MMA issuer, 8 transform warps, 4 epilogue warps
-constexpr int PIPE_XF = 256;          // transform threads
+constexpr int PIPE_WORKERS = 12;      // transform + epilogue warps
+constexpr int PIPE_THREADS = (2 + PIPE_WORKERS) * 32;     // producer, MMA issuer, workers
 constexpr int MAX_RAW = 8;
 
 struct PipeArgs {
@@ -449,6 +449,8 @@ struct PipeArgs {
     uint32_t o_bytes;           // one output staging tile [128][N] bf16 (multiple of 128)
     int OS;                     // output staging tiles: 1 or 2
     int AS;                     // operand stages: 2, or 1 where a long reduction leaves no room for two
+    int xf_warps;               // of the 12 worker warps, how many transform (4 or 8); the rest run the epilogue: a tile
+                                // costs the transform warps ~K and the epilogue warps ~N instructions per row
     const float* pivot;         // forward, optional: per-channel pivot of the fused BatchNorm statistics
     float* stat_partial;        // [CTAs][2][N]: sums of (z - pivot) and (z - pivot)^2 over the CTA's pixels
     // backward, optional: BatchNorm-backward sums of the produced gradient (the unit that made this conv's input)
@@ -481,6 +483,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     const bool csum = bred || (!BWD && a.stat_partial != nullptr);   // the transform warps take column sums of every output tile
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = a.R, RS = a.RS, subs = TM / RS;
+    const int nxf = a.xf_warps * 32, nepi = (PIPE_WORKERS - a.xf_warps) * 32, epi_warp0 = 2 + a.xf_warps;
     const uint32_t bar0 = smem_u32(&bars[0]);
     auto raw_full = [&](int s) { return bar0 + 8u * s; };
     auto raw_empty = [&](int s) { return bar0 + 8u * (MAX_RAW + s); };
@@ -496,17 +499,17 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     if (tid == 0) {
         for (int s = 0; s < R; ++s) {
             mbar_init(raw_full(s), 1);
-            mbar_init(raw_empty(s), PIPE_XF);
+            mbar_init(raw_empty(s), nxf);
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(a_full(s), PIPE_XF);
+            mbar_init(a_full(s), nxf);
             mbar_init(a_empty(s), 1);
             mbar_init(acc_full(s), 1);
-            mbar_init(acc_empty(s), 128);
+            mbar_init(acc_empty(s), nepi);
             mbar_init(zp_full(s), 1);
-            mbar_init(zp_empty(s), PIPE_XF);
+            mbar_init(zp_empty(s), nxf);
             mbar_init(so_full(s), 1);
-            mbar_init(so_free(s), PIPE_XF);
+            mbar_init(so_free(s), nxf);
         }
         abort_store = 0;
     }
@@ -601,10 +604,10 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
                 umma_commit(acc_full(st));
             }
         }
-    } else if (warp < 10) {
+    } else if (warp < epi_warp0) {
         // ------------------------------------------------------------ transformers
         const int tix = tid - 64;
-        const int groups = PIPE_XF / vpr_pad;             // row groups; thread (grp, j) owns chunk j of rows grp, grp+groups, ...
+        const int groups = nxf / vpr_pad;                 // row groups; thread (grp, j) owns chunk j of rows grp, grp+groups, ...
         const int j = tix % vpr_pad, grp = tix / vpr_pad;
         const bool active = grp < groups;
         const bool data = j < vpr;                        // chunks beyond K are zero padding
@@ -618,7 +621,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
         //   forward:  sums of (z - pivot) and (z - pivot)^2, the BatchNorm statistics partials of the output;
         //   backward: sums of dpre = dx * [pre inside the activation's linear region] and dpre * xhat, with pre = z*rcs + rch
         //             and xhat = z*rrs + rms taken from the matching tile of the producing unit's raw output z.
-        const int r_units = a.N >> 2, r_split = PIPE_XF / r_units;
+        const int r_units = a.N >> 2, r_split = nxf / r_units;
         const int cu = tix % r_units, rh = tix / r_units;
         const bool ractive = csum && rh < r_split;
         float s1[4], s2[4], rcs[4], rch[4], rrs[4], rms[4];     // forward: rcs holds the pivot
@@ -729,7 +732,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             // combine the r_split row classes of every column group in fixed order (every transform thread gets here,
             // also after an abort: all waits are bounded); the operand stages are free now: the last tile's sums were
             // taken after its epilogue, hence after its MMAs
-            named_bar_sync(2, PIPE_XF);
+            named_bar_sync(2, nxf);
             float* red = reinterpret_cast<float*>(sA);        // [r_split][2][N]
             if (ractive) {
 #pragma unroll
@@ -738,8 +741,8 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
                     red[(rh * 2 + 1) * a.N + cu * 4 + i] = s2[i];
                 }
             }
-            named_bar_sync(2, PIPE_XF);
-            for (int e = tix; e < 2 * a.N; e += PIPE_XF) {
+            named_bar_sync(2, nxf);
+            for (int e = tix; e < 2 * a.N; e += nxf) {
                 float acc = 0.f;
                 for (int k = 0; k < r_split; ++k) acc += red[k * 2 * a.N + e];
                 (BWD ? a.r_partial : a.stat_partial)[(size_t)blockIdx.x * 2 * a.N + e] = acc;
@@ -752,7 +755,8 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
         // are one contiguous byte range; one thread then stores the tile with a single bulk copy.
         const int q = warp & 3;                            // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
-        const int et = tid - (PIPE_THREADS - 128);
+        const int et = tid - epi_warp0 * 32;
+        const int half = (warp - epi_warp0) >> 2, nhalf = nepi >> 7;      // several threads share a row: they alternate column batches
         const uint32_t row_out = (uint32_t)a.N * 2u;
         int issued = 0;
         for (int t = 0; t < my_tiles; ++t) {
@@ -768,13 +772,13 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
                 if (a.OS == 2) bulk_wait_read<1>();
                 else bulk_wait_read<0>();
             }
-            ok = named_bar_and(1, 128, ok);
+            ok = named_bar_and(1, nepi, ok);
             if (!ok) break;
             fence_after_sync();
             const int p = tile * TM + row;
             // accumulator columns in batches of up to 64: the batch's tcgen05.ld are all issued
             // before the one wait, so their latencies overlap
-            for (int g0 = 0; g0 < (NT >> 4); g0 += 4) {
+            for (int g0 = half * 4; g0 < (NT >> 4); g0 += 4 * nhalf) {
                 uint32_t rr[4][16];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
@@ -810,7 +814,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             fence_before_sync();
             mbar_arrive(acc_empty(st));
             fence_async_smem();
-            named_bar_sync(1, 128);
+            named_bar_sync(1, nepi);
             const int valid = min(TM, a.P - tile * TM);
             if (et == 0) {
                 bulk_s2g(a.out + (size_t)tile * TM * a.N, smem_u32(so), (uint32_t)valid * row_out);
@@ -844,6 +848,22 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
     const int tensors = a.need_z ? 2 : 1;
     const size_t zp = a.r_partial ? 2 * (size_t)a.o_bytes : 0;      // two tiles of the raw output the backward sums read
     // two operand stages if they fit; one for long reductions (the transform of tile t+1 then waits for the MMAs of t)
+    {
+        // split of the twelve worker warps: estimated instructions per tile of the two roles, spread over their warps
+        const double vpr_pad = ((a.K + 15) / 16) * 2;
+        const bool csum = a.stat_partial != nullptr || a.r_partial != nullptr;
+        const double xf_work = 128.0 * vpr_pad * (a.need_z ? 60.0 : 30.0) + (csum ? 128.0 * (a.N / 4) * (a.r_partial ? 25.0 : 15.0) : 0.0);
+        const double epi_work = 128.0 * (a.N / 8.0) * ((a.addend || a.bias) ? 35.0 : 22.0);
+        double best = 0;
+        a.xf_warps = 8;
+        for (int x = 4; x <= PIPE_WORKERS - 4; x += 4) {
+            const double t = xf_work / x > epi_work / (PIPE_WORKERS - x) ? xf_work / x : epi_work / (PIPE_WORKERS - x);
+            if (x == 4 || t < best) {
+                best = t;
+                a.xf_warps = x;
+            }
+        }
+    }
     for (a.AS = 2; a.AS >= 1; --a.AS) {
         const size_t ab = (size_t)a.AS * a.a_bytes;
         // two output staging tiles if that still leaves room for two 64-pixel raw stages

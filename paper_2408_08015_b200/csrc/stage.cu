@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <string>
 #include <vector>
@@ -70,6 +71,17 @@ struct Unit {
     long up_off = -1;
 };
 
+// Arenas of a stage carry a guard band of GUARD bytes of a fixed pattern on both sides.  With the environment variable
+// ASTEROID_CHECK_GUARDS=1 export_state reads the bands back and reports an arena whose band was overwritten (an
+// out-of-bounds write of some kernel) as AST_ERR_CUDA.  The check runs on the host, between rounds.
+constexpr size_t GUARD = 256;
+constexpr unsigned char GUARD_BYTE = 0xA5;
+struct Arena {
+    char* base;
+    size_t bytes;      // payload bytes (the guards lie at base and base + GUARD + bytes)
+    const char* name;
+};
+
 struct Timing {
     bool on = false;
     std::vector<cudaEvent_t> ev;    // per unit: f0 f1 f2 b0 b1 b2
@@ -111,8 +123,13 @@ struct asteroid_stage {
     std::vector<int> slot_of_mb, mb_of_slot;
     int pending_g = -1, n_acc = 0;
     Timing tm;
+    std::vector<ast::Arena> arenas;                // every device allocation of the stage, with its guard bands
+    bool check_guards = false;
     std::vector<asteroid_stage*> prof_cache;
     std::vector<std::vector<double>> prof_ms;   // per cached stage: 4 per unit (f_main, f_bn, b_bn, b_main)
+    // what the last forward / backward did, per unit: statistics partials written by the producing kernel (their count, 0 =
+    // standalone pass); unit whose backward-data kernel took this unit's BatchNorm-backward sums (-1 = standalone pass)
+    std::vector<int> fwd_stats_blocks, bwd_sums_by;
 };
 
 namespace ast {
@@ -331,14 +348,15 @@ static void free_stage(asteroid_stage* s) {
     if (!s) return;
     for (auto* p : s->prof_cache) free_stage(p);
     for (auto e : s->tm.ev) cudaEventDestroy(e);
-    cudaFree(s->w); cudaFree(s->v); cudaFree(s->G); cudaFree(s->g); cudaFree(s->derived); cudaFree(s->run);
-    cudaFree(s->coef); cudaFree(s->scratch); cudaFree(s->perm); cudaFree(s->slot_mem); cudaFree(s->grad_mem);
-    cudaFree(s->wb); cudaFree(s->wtb); cudaFree(s->err); cudaFree(s->scratch_side); cudaFree(s->wpad); cudaFree(s->gpad); cudaFree(s->up_mem);
+    for (const Arena& a : s->arenas) cudaFree(a.base);
     if (s->ev_fork) cudaEventDestroy(s->ev_fork);
     if (s->ev_join) cudaEventDestroy(s->ev_join);
     if (s->side) cudaStreamDestroy(s->side);
     delete s;
 }
+
+
+template <typename P> static int arena_alloc(asteroid_stage* s, const char* name, P** p, size_t bytes, size_t* tally);
 
 template <typename P> static int dev_alloc(P** p, size_t bytes, size_t* tally) {
     if (bytes == 0) bytes = 256;
@@ -350,6 +368,37 @@ template <typename P> static int dev_alloc(P** p, size_t bytes, size_t* tally) {
     e = cudaMemset(*p, 0, bytes);
     if (e != cudaSuccess) return fail(AST_ERR_CUDA, "cudaMemset: %s", cudaGetErrorString(e));
     *tally += bytes;
+    return AST_OK;
+}
+
+template <typename P> static int arena_alloc(asteroid_stage* s, const char* name, P** p, size_t bytes, size_t* tally) {
+    if (bytes == 0) bytes = 256;
+    bytes = align_up(bytes, 256);
+    char* base = nullptr;
+    cudaError_t e = cudaMalloc((void**)&base, bytes + 2 * GUARD);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(AST_ERR_ALLOC, "cudaMalloc of %zu bytes (%s) failed: %s", bytes, name, cudaGetErrorString(e));
+    }
+    s->arenas.push_back(Arena{base, bytes, name});
+    e = cudaMemset(base, GUARD_BYTE, GUARD);
+    if (e == cudaSuccess) e = cudaMemset(base + GUARD, 0, bytes);
+    if (e == cudaSuccess) e = cudaMemset(base + GUARD + bytes, GUARD_BYTE, GUARD);
+    if (e != cudaSuccess) return fail(AST_ERR_CUDA, "cudaMemset: %s", cudaGetErrorString(e));
+    *p = reinterpret_cast<P*>(base + GUARD);
+    *tally += bytes + 2 * GUARD;
+    return AST_OK;
+}
+
+static int check_guards(asteroid_stage* s) {
+    unsigned char h[2 * GUARD];
+    for (const Arena& a : s->arenas) {
+        CU(cudaMemcpy(h, a.base, GUARD, cudaMemcpyDeviceToHost));
+        CU(cudaMemcpy(h + GUARD, a.base + GUARD + a.bytes, GUARD, cudaMemcpyDeviceToHost));
+        for (size_t i = 0; i < 2 * GUARD; ++i)
+            if (h[i] != GUARD_BYTE)
+                return fail(AST_ERR_CUDA, "guard band of arena '%s' overwritten %s the arena (byte %zu)", a.name, i < GUARD ? "before" : "after", i % GUARD);
+    }
     return AST_OK;
 }
 
@@ -465,6 +514,7 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
             gap_fwd(dt, val_src(s, sv, u.in), s->B, a.h * a.w, a.c, obuf, st);
         }
         tick(s, ui, 1, st);
+        s->fwd_stats_blocks[ui] = fused_stats;
         if (u.l_bn >= 0) {
             float* stt = sv.stats + o.stat_off;
             BnFwdOut bo{stt, stt + o.c, stt + 2 * (size_t)o.c, stt + 3 * (size_t)o.c, s->run + u.run_off, s->run + u.run_off + o.c};
@@ -529,6 +579,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
     gs.back().state = G_ALIAS;
     gs.back().ptr = dy;
     std::vector<char> reduced(s->units.size(), 0);   // BatchNorm-backward sums already taken by the kernel that wrote dy
+    std::fill(s->bwd_sums_by.begin(), s->bwd_sums_by.end(), -1);
     // weight gradients go to the second stream (not while a profile run times the units one by one, nor while a
     // per-launch trace brackets every kernel with events: a kernel's duration is then that of the kernel running alone)
     const bool use_side = s->side != nullptr && !s->tm.on && !tracing();
@@ -609,7 +660,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                 const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
                 // this kernel writes the complete gradient of its input value: let it also take the BatchNorm-backward
                 // sums of the unit that gradient belongs to
-                const int tgt = (s->vals[u.in].first_cons == ui && !s->tm.on) ? bn_reduce_target(s, u.in) : -1;
+                const int tgt = s->vals[u.in].first_cons == ui ? bn_reduce_target(s, u.in) : -1;
                 if (u.kind == U_CONV && pw_tc_supported(dt, u.g, true)) {
                     BnRed red{};
                     if (tgt >= 0) {
@@ -627,6 +678,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                         BnBwdOut tbo{s->g + tu.gamma_off, s->g + tu.beta_off, tk, tk + tv.c, tk + 2 * (size_t)tv.c};
                         bn_bwd_finish_partials(s->scratch, blocks, tv.elems / tv.c, tv.c, ts, ts + tv.c, s->w + tu.gamma_off, tbo, st);
                         reduced[tgt] = 1;
+                        s->bwd_sums_by[tgt] = ui;
                     }
                 } else if (u.kind == U_CONV && conv3_tc_supported(dt, u.g)) conv3_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
                 else if (s2_tc) conv3_bwd_data_tc(s1_geom(u), dup, s->wtb + u.w_off, addend, own(u.in), s->err, st, conv_flops(u.g));
@@ -679,41 +731,45 @@ static int create_impl(const ast_layer* net, int n_layers, int first, int last, 
     s->need_dx = opts ? (opts->need_input_grad != 0) : 1;
     s->eps = (opts && opts->bn_eps > 0.f) ? opts->bn_eps : 1e-5f;
     s->bn_mom = (opts && opts->bn_momentum > 0.f) ? opts->bn_momentum : 0.1f;
+    {
+        const char* e = getenv("ASTEROID_CHECK_GUARDS");
+        s->check_guards = e && e[0] == '1';
+    }
     int rc = build_plan(s);
     if (rc) return rc;
 
     const size_t np = s->n_params;
     size_t mod = 0, opt = 0, act = 0, work = 0;
-    if ((rc = dev_alloc(&s->w, np * 4, &mod))) return rc;
-    if ((rc = dev_alloc(&s->G, np * 4, &mod))) return rc;
-    if ((rc = dev_alloc(&s->g, np * 4, &mod))) return rc;
-    if ((rc = dev_alloc(&s->derived, np * 4, &mod))) return rc;
-    if ((rc = dev_alloc(&s->perm, np * 4, &mod))) return rc;
-    if ((rc = dev_alloc(&s->run, s->n_run * 4, &mod))) return rc;
+    if ((rc = arena_alloc(s, "parameters", &s->w, np * 4, &mod))) return rc;
+    if ((rc = arena_alloc(s, "accumulated gradients", &s->G, np * 4, &mod))) return rc;
+    if ((rc = arena_alloc(s, "micro-batch gradients", &s->g, np * 4, &mod))) return rc;
+    if ((rc = arena_alloc(s, "derived weights", &s->derived, np * 4, &mod))) return rc;
+    if ((rc = arena_alloc(s, "permutation", &s->perm, np * 4, &mod))) return rc;
+    if ((rc = arena_alloc(s, "running statistics", &s->run, s->n_run * 4, &mod))) return rc;
     if (s->dtype == AST_BF16) {
-        if ((rc = dev_alloc(&s->wb, np * 2, &mod))) return rc;
-        if ((rc = dev_alloc(&s->wtb, np * 2, &mod))) return rc;
+        if ((rc = arena_alloc(s, "bf16 weights", &s->wb, np * 2, &mod))) return rc;
+        if ((rc = arena_alloc(s, "bf16 derived weights", &s->wtb, np * 2, &mod))) return rc;
     }
     if (s->n_wpad) {
-        if ((rc = dev_alloc(&s->wpad, s->n_wpad * 2, &mod))) return rc;
-        if ((rc = dev_alloc(&s->gpad, s->n_gpad * 4, &work))) return rc;
+        if ((rc = arena_alloc(s, "padded weights", &s->wpad, s->n_wpad * 2, &mod))) return rc;
+        if ((rc = arena_alloc(s, "padded weight gradient", &s->gpad, s->n_gpad * 4, &work))) return rc;
     }
-    if ((rc = dev_alloc(&s->err, 256, &work))) return rc;
-    if ((rc = dev_alloc(&s->v, np * 4, &opt))) return rc;
-    if ((rc = dev_alloc(&s->slot_mem, s->slot_bytes * s->slots, &act))) return rc;
-    if ((rc = dev_alloc(&s->grad_mem, s->grad_bytes, &work))) return rc;
-    if ((rc = dev_alloc(&s->coef, s->n_coef * 4, &work))) return rc;
+    if ((rc = arena_alloc(s, "error word", &s->err, 256, &work))) return rc;
+    if ((rc = arena_alloc(s, "momentum", &s->v, np * 4, &opt))) return rc;
+    if ((rc = arena_alloc(s, "activation slots", &s->slot_mem, s->slot_bytes * s->slots, &act))) return rc;
+    if ((rc = arena_alloc(s, "gradient workspace", &s->grad_mem, s->grad_bytes, &work))) return rc;
+    if ((rc = arena_alloc(s, "BatchNorm-backward coefficients", &s->coef, s->n_coef * 4, &work))) return rc;
     s->scratch_floats = (size_t)8 << 20;
     for (const auto& u : s->units)
         if (u.kind == U_CONV) s->scratch_floats = std::max(s->scratch_floats, (size_t)4 * u.g.co * u.g.k * u.g.k * u.g.ci);
-    if ((rc = dev_alloc(&s->scratch, s->scratch_floats * 4, &work))) return rc;
-    if ((rc = dev_alloc(&s->scratch_side, s->scratch_floats * 4, &work))) return rc;
+    if ((rc = arena_alloc(s, "scratch", &s->scratch, s->scratch_floats * 4, &work))) return rc;
+    if ((rc = arena_alloc(s, "scratch of the second stream", &s->scratch_side, s->scratch_floats * 4, &work))) return rc;
     for (auto& u : s->units)
         if (conv3_s2_tc_supported(s, u)) {
             u.up_off = (long)s->up_bytes;
             s->up_bytes += align_up((size_t)u.g.n * u.g.hi * u.g.wi * u.g.co * 2, 256);
         }
-    if (s->up_bytes && (rc = dev_alloc(&s->up_mem, s->up_bytes, &work))) return rc;
+    if (s->up_bytes && (rc = arena_alloc(s, "zero-inserted gradients", &s->up_mem, s->up_bytes, &work))) return rc;
     CU(cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking));
     CU(cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming));
     CU(cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming));
@@ -724,6 +780,8 @@ static int create_impl(const ast_layer* net, int n_layers, int first, int last, 
     if ((rc = reset_bn_running(s))) return rc;
     s->slot_of_mb.assign(M, -1);
     s->mb_of_slot.assign(s->slots, -1);
+    s->fwd_stats_blocks.assign(s->units.size(), 0);
+    s->bwd_sums_by.assign(s->units.size(), -1);
     return AST_OK;
 }
 
@@ -798,6 +856,10 @@ int asteroid_stage_export_state(asteroid_stage* s, float* params, float* momentu
     if (errw) {
         CU(cudaMemset(s->err, 0, sizeof errw));
         return fail(AST_ERR_TIMEOUT, "a bounded device-side wait expired in a tensor-core kernel; results of this round are invalid");
+    }
+    if (s->check_guards) {
+        int grc = check_guards(s);
+        if (grc) return grc;
     }
     if (n) {
         if (params) CU(cudaMemcpy(params, s->w, n * 4, cudaMemcpyDeviceToHost));
@@ -1009,14 +1071,37 @@ int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_pr
         } else if (layer == u.l_bn) {
             out->t_f_ms = ms[ui * 4 + 1];
             out->t_b_ms = ms[ui * 4 + 2];
-            out->alg_bytes_f = zo;          // statistics pass over z
-            out->alg_bytes_b = 2 * zo;      // the two reductions read dy and z
+            // Statistics: a standalone pass over z, or - taken inside the producing kernel - only the finishing of that
+            // kernel's per-CTA partials.  Backward sums: a standalone pass over dy and z, or nothing here when the
+            // backward-data kernel of the consuming unit took them (its record carries the time; fused_into names it).
+            const int fb = t->fwd_stats_blocks[ui];
+            out->alg_bytes_f = fb > 0 ? 8ull * vout.c * (uint64_t)(fb + 4) : zo;
+            if (fb > 0) out->fused_into = u.l_main;
+            const int by = t->bwd_sums_by[ui];
+            out->alg_bytes_b = by >= 0 ? 0 : 2 * zo;
+            if (by >= 0) out->fused_into = t->units[by].l_main;
         } else {                            // activation: applied inside the neighbouring kernels
             out->fused_into = u.l_bn >= 0 ? u.l_bn : u.l_main;
         }
         return AST_OK;
     }
     return fail(AST_ERR_ARG, "layer %d not found in the plan", layer);
+}
+
+int asteroid_selftest_bounded_wait(void) {
+    int* err = nullptr;
+    CU(cudaMalloc((void**)&err, sizeof(int)));
+    cudaError_t e = cudaMemset(err, 0, sizeof(int));
+    int h = 0;
+    if (e == cudaSuccess) {
+        launch_bounded_wait_probe(err, 1024u, 0);
+        e = cudaDeviceSynchronize();
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(&h, err, sizeof h, cudaMemcpyDeviceToHost);
+    cudaFree(err);
+    if (e != cudaSuccess) return fail(AST_ERR_CUDA, "bounded-wait self-test: %s", cudaGetErrorString(e));
+    if (h) return fail(AST_ERR_TIMEOUT, "a bounded device-side wait expired (self-test: expected)");
+    return AST_OK;
 }
 
 uint64_t asteroid_launch_count(void) { return launches(); }

@@ -25,6 +25,10 @@ def test_profile_record_closed_forms_and_memory_terms():
             assert r["a_l_bytes"] == ref["a_l"] and r["w_l_bytes"] == ref["w_l"] and r["flops"] == ref["flops"], (l, r, ref)
             if net[l].op in ("conv", "dwconv"):
                 assert r["t_f_ms"] > 0 and r["t_b_ms"] > 0 and r["alg_bytes_f"] > 0 and r["alg_bytes_b"] > r["alg_bytes_f"]
+            # no record may claim more than the memory system can deliver (a fused BatchNorm reports its finishing kernel only)
+            for t, nb in ((r["t_f_ms"], r["alg_bytes_f"]), (r["t_b_ms"], r["alg_bytes_b"])):
+                if t > 0:
+                    assert nb / (t * 1e-3) < 8e12, (l, net[l].op, r)
             if net[l].op in ("relu6", "relu"):
                 assert r["t_f_ms"] == 0 and r["fused_into"] == l - 1
         r0 = recs[first]

@@ -37,6 +37,30 @@ def test_noalloc_mse_matches_allocating_entry_point_twice(bf16):
         assert abs(lb - ref) <= tol * ref
 
 
+def test_noalloc_calls_leave_the_free_device_memory_unchanged_and_work_on_a_second_stream():
+    import torch
+    import paper_2408_08015_b200 as P
+    dev = torch.device("cuda:0")
+    n = 1 << 20
+    y = torch.from_numpy(si.normal(6, 1, (n,)).astype(np.float32)).to(dev)
+    t = torch.from_numpy(si.normal(6, 2, (n,)).astype(np.float32)).to(dev)
+    dy, loss = torch.empty_like(y), torch.zeros(2, device=dev)
+    side = torch.cuda.Stream(device=dev)
+    P.asteroid_loss_mse_noalloc(y.data_ptr(), t.data_ptr(), n, P.AST_F32, dy.data_ptr(), loss.data_ptr())     # warm-up: address look-up
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(20):
+        P.asteroid_loss_mse_noalloc(y.data_ptr(), t.data_ptr(), n, P.AST_F32, dy.data_ptr(), loss.data_ptr())
+    torch.cuda.synchronize()
+    # a call on another stream once the first stream's calls have finished (the shared ticket word is cleared per call)
+    P.asteroid_loss_mse_noalloc(y.data_ptr(), t.data_ptr(), n, P.AST_F32, dy.data_ptr(), loss.data_ptr() + 4, side.cuda_stream)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0            # no allocation by the entry point (torch allocated nothing in between)
+    la, lb = loss.cpu().numpy().tolist()
+    ref = ((y.double() - t.double()) ** 2).mean().item()
+    assert abs(la - ref) <= 1e-5 * ref and la == lb
+
+
 def test_noalloc_rejects_sizes_beyond_its_limit():
     import torch
     import paper_2408_08015_b200 as P
