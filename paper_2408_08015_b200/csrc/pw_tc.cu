@@ -80,6 +80,50 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
         constexpr int U = 4;
         const bool need_z = BWD && grad_needs_z(a.dz);
         const int items = TM * vpr_pad;
+        if (NTHREADS % vpr_pad == 0) {
+            // usual case: the chunks per row divide the thread count, so a thread keeps one 16-byte channel chunk for the
+            // whole reduction chunk and holds that chunk's transform coefficients in registers
+            const int j = tid % vpr_pad, rstep = NTHREADS / vpr_pad;
+            const bool data = j < vpr;
+            const int c0 = k0 + ((data ? j : 0) << 3);
+            XfVal xv;
+            XfGrad xg;
+            if (BWD) xg.init(a.dz, c0);
+            else xv.init(a.x, c0);
+            const uint4* src = reinterpret_cast<const uint4*>(BWD ? a.dz.dy : a.x.p);
+            const uint4* srcz = reinterpret_cast<const uint4*>(a.dz.z);
+            for (int rb = tid / vpr_pad; rb < TM; rb += U * rstep) {
+                uint4 raw[U], rawz[U];
+                bool ok[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = rb + u * rstep;
+                    const int p = p0 + r;
+                    ok[u] = r < TM && p < a.P && data;
+                    raw[u] = rawz[u] = make_uint4(0, 0, 0, 0);
+                    if (ok[u]) {
+                        size_t pin = p;
+                        if (!BWD && a.stride > 1) {
+                            int wo = p % a.wo, t = p / a.wo;
+                            int ho = t % a.ho, n = t / a.ho;
+                            pin = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
+                        }
+                        const size_t e = (pin * a.K + c0) >> 3;
+                        raw[u] = src[e];
+                        if (need_z) rawz[u] = srcz[e];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = rb + u * rstep;
+                    if (r < TM) {
+                        uint4 q = make_uint4(0, 0, 0, 0);
+                        if (ok[u]) q = BWD ? (need_z ? xg.apply(raw[u], rawz[u]) : raw[u]) : xv.apply(raw[u]);
+                        *reinterpret_cast<uint4*>(sA + tile_off(r, j, TM)) = q;
+                    }
+                }
+            }
+        } else
         for (int v0 = tid; v0 < items; v0 += U * NTHREADS) {
             Vec<__nv_bfloat16> raw[U], rawz[U];
             bool ok[U];
@@ -264,6 +308,12 @@ __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArg
     uint32_t ph[2] = {0, 0};
     int issued[2] = {0, 0};
     bool ok = true, bad = false;       // `bad` is decided by a block-wide vote: uniform across threads
+    const bool fast = ca > 0 && cb > 0 && NTHREADS % ca == 0 && NTHREADS % cb == 0;
+    const int fja = fast ? tid % ca : 0, fjb = fast ? tid % cb : 0;
+    XfGrad fxg;
+    XfVal fxv;
+    fxg.init(a.dz, m0 + (fja << 3));
+    fxv.init(a.x, n0 + (fjb << 3));
     int stage = 0;
     for (int ps = pbeg; ps < pend; ps += WSTAGE, ++stage) {
         const int b = stage & 1;
@@ -281,6 +331,60 @@ __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArg
         // both operands: the loads of four vectors per thread are issued together before any is transformed
         constexpr int U = 4;
         const bool need_z = grad_needs_z(a.dz);
+        if (fast) {
+            // a thread keeps one channel chunk of each operand; its coefficients were loaded into registers once
+            const uint4* gdy = reinterpret_cast<const uint4*>(a.dz.dy);
+            const uint4* gz = reinterpret_cast<const uint4*>(a.dz.z);
+            const uint4* gx = reinterpret_cast<const uint4*>(a.x.p);
+            for (int rb = tid / ca; rb < WSTAGE; rb += U * (NTHREADS / ca)) {
+                uint4 raw[U], rawz[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int kr = rb + u * (NTHREADS / ca);
+                    raw[u] = rawz[u] = make_uint4(0, 0, 0, 0);
+                    if (kr < valid) {
+                        const size_t e = ((size_t)(ps + kr) * a.CO + m0 + (fja << 3)) >> 3;
+                        raw[u] = gdy[e];
+                        if (need_z) rawz[u] = gz[e];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int kr = rb + u * (NTHREADS / ca);
+                    if (kr < WSTAGE) {
+                        uint4 q = make_uint4(0, 0, 0, 0);
+                        if (kr < valid) q = need_z ? fxg.apply(raw[u], rawz[u]) : raw[u];
+                        *reinterpret_cast<uint4*>(sA + (fja >> 3) * PANEL + kr * 128 + (((fja & 7) ^ (kr & 7)) << 4)) = q;
+                    }
+                }
+            }
+            for (int rb = tid / cb; rb < WSTAGE; rb += U * (NTHREADS / cb)) {
+                uint4 raw[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int kr = rb + u * (NTHREADS / cb);
+                    raw[u] = make_uint4(0, 0, 0, 0);
+                    if (kr < valid) {
+                        size_t pin = ps + kr;
+                        if (a.stride > 1) {
+                            int p = ps + kr;
+                            int wo = p % a.wo, t = p / a.wo;
+                            int ho = t % a.ho, n = t / a.ho;
+                            pin = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
+                        }
+                        raw[u] = gx[(pin * a.CI + n0 + (fjb << 3)) >> 3];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int kr = rb + u * (NTHREADS / cb);
+                    if (kr < WSTAGE) {
+                        const uint4 q = kr < valid ? fxv.apply(raw[u]) : make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4*>(sB + (fjb >> 3) * PANEL + kr * 128 + (((fjb & 7) ^ (kr & 7)) << 4)) = q;
+                    }
+                }
+            }
+        } else {
         for (int v0 = tid; v0 < WSTAGE * ca; v0 += U * NTHREADS) {
             Vec<__nv_bfloat16> raw[U], rawz[U];
             bool ok[U];
@@ -345,6 +449,7 @@ __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArg
                     *reinterpret_cast<uint4*>(sB + (j >> 3) * PANEL + kr * 128 + (((j & 7) ^ (kr & 7)) << 4)) = q;
                 }
             }
+        }
         }
         fence_async_smem();
         __syncthreads();
