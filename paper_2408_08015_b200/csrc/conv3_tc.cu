@@ -311,23 +311,32 @@ template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) co
     uint4 raw[IT], rawz[IT];
     uint32_t okmask = 0;
 
+    // Positions advance by `step` rows per item: (hp, wp) of a row follow from the previous row's by additions, so that a
+    // tile costs one integer division per thread; element indices stay in 32 bits, in units of 16-byte vectors.
+    const int step_q = step / Wp, step_r = step - step_q * Wp;
+    const uint32_t W_u = (uint32_t)a.W, H_u = (uint32_t)a.H;
     auto prefetch = [&](int tl) {
         const int img = tl / a.tiles_per_img, tile = tl - img * a.tiles_per_img;
-        const int fs0 = tile * TM;                          // first staged position (first output position - Wp - 1)
+        const int f0 = tile * TM + r_first;                 // first staged position of this thread (first output position - Wp - 1)
+        int hp = f0 / Wp, wp = f0 - hp * Wp;
+        const uint32_t img_row0 = (uint32_t)img * H_u;
         okmask = 0;
 #pragma unroll
         for (int u = 0; u < IT; ++u) {
-            const int r = r_first + u * step;
-            const int f = fs0 + r;
-            const int hp = f / Wp, wp = f - hp * Wp;
-            const bool ok = r < rows && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+            const bool ok = r_first + u * step < rows && (uint32_t)(hp - 1) < H_u && (uint32_t)(wp - 1) < W_u;
             raw[u] = make_uint4(0, 0, 0, 0);
             if (BWD) rawz[u] = make_uint4(0, 0, 0, 0);
             if (ok) {
-                const size_t e = ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.C + c0) >> 3;
+                const uint32_t e = ((img_row0 + (uint32_t)(hp - 1)) * W_u + (uint32_t)(wp - 1)) * (uint32_t)vpr + (uint32_t)j;
                 raw[u] = __ldg(src + e);
                 if (need_z) rawz[u] = __ldg(srcz + e);
                 okmask |= 1u << u;
+            }
+            wp += step_r;
+            hp += step_q;
+            if (wp >= Wp) {
+                wp -= Wp;
+                ++hp;
             }
         }
     };
@@ -346,14 +355,18 @@ template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) co
     auto issue = [&](int buf, int acc) {
         const uint32_t abase = smem_u32(sA) + (uint32_t)buf * a_buf, bbase = smem_u32(sB);
         const uint32_t d = tmem + (uint32_t)(acc * C3P_NH);
+        // descriptor = constant fields + (address >> 4): all addresses here are 16-byte multiples below 256 KB
+        const uint64_t dconst = make_desc(0);
+#pragma unroll
         for (int t = 0; t < 9; ++t) {
             const int r = t / 3, s = t - r * 3;
-            const uint32_t a0 = abase + (uint32_t)(r * Wp + s) * 128u;
-            const uint32_t b0 = bbase + (uint32_t)t * b_tap;
-            for (int k = 0; k < (a.C >> 4); ++k) {
-                const int kb = k >> 2, ks = k & 3;
-                umma_bf16(d, make_desc(a0 + (uint32_t)kb * a_block + (uint32_t)ks * 32u), make_desc(b0 + (uint32_t)kb * C3P_NH * 128u + (uint32_t)ks * 32u),
-                          idesc, (t > 0 || k > 0) ? 1u : 0u);
+            const uint32_t a0 = (abase + (uint32_t)(r * Wp + s) * 128u) >> 4;
+            const uint32_t b0 = (bbase + (uint32_t)t * b_tap) >> 4;
+            for (int kb = 0; kb < kbs; ++kb) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16(d, dconst + (uint64_t)(a0 + (((uint32_t)kb * a_block + (uint32_t)ks * 32u) >> 4)),
+                              dconst + (uint64_t)(b0 + (((uint32_t)kb * C3P_NH * 128u + (uint32_t)ks * 32u) >> 4)), idesc, (t > 0 || kb > 0 || ks > 0) ? 1u : 0u);
             }
         }
         umma_commit(bar[acc]);
@@ -440,6 +453,7 @@ bool plan_c3p(const C3Args& a, C3PArgs& p, size_t* smem, int* it) {
     const int kbs = a.C / 64;
     *it = a.C == 64 ? 4 : 8;
     if (rows > *it * (C3P_THREADS / (a.C >> 3))) return false;
+    if ((double)a.n_img * a.H * a.W * (a.C > a.N ? a.C : a.N) / 8.0 >= 4.0e9) return false;      // 32-bit vector indices
     p.x = a.x; p.dz = a.dz; p.w = a.w; p.addend = a.addend; p.out = a.out; p.err = a.err;
     p.n_img = a.n_img; p.H = a.H; p.W = a.W; p.C = a.C; p.N = a.N; p.flip = a.flip;
     p.tiles_per_img = ((a.H - 1) * Wp + a.W + TM - 1) / TM;
@@ -548,6 +562,7 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
     bool bad = false;
     const int vx = a.CI >> 3, vz = a.CO >> 3;             // chunks per row: 8 or 16, both divide 256
     const int jx = tid % vx, jz = tid % vz, stepx = C3_THREADS / vx, stepz = C3_THREADS / vz;
+    const int sxq = stepx / Wp, sxr = stepx - sxq * Wp, szq = stepz / Wp, szr = stepz - szq * Wp;
     const bool need_z = a.dz.act != ACT_NONE || a.dz.k1 != nullptr;
     const uint4* gx = reinterpret_cast<const uint4*>(a.x.p);
     const uint4* gdy = reinterpret_cast<const uint4*>(a.dz.dy);
@@ -563,17 +578,24 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
         // (coefficients in registers) and every (256 / chunks)-th row; the loads of four rows are issued together
         {
             constexpr int U = 4;
+            // (hp, wp) of consecutive items follow by additions (one division per tile and operand); 32-bit vector indices
+            const uint32_t img_row0 = (uint32_t)img * (uint32_t)a.H;
+            int hp = (fs0 + tid / vx) / Wp, wp = (fs0 + tid / vx) - hp * Wp;
             for (int rb = tid / vx; rb < rows; rb += U * stepx) {
                 uint4 raw[U];
                 bool ok[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const int r = rb + u * stepx;
-                    const int f = fs0 + r;
-                    const int hp = f / Wp, wp = f - hp * Wp;
-                    ok[u] = r < rows && f >= 0 && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+                    ok[u] = r < rows && (uint32_t)(hp - 1) < (uint32_t)a.H && (uint32_t)(wp - 1) < (uint32_t)a.W;
                     raw[u] = make_uint4(0, 0, 0, 0);
-                    if (ok[u]) raw[u] = __ldg(gx + (((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CI + (jx << 3)) >> 3));
+                    if (ok[u]) raw[u] = __ldg(gx + ((img_row0 + (uint32_t)(hp - 1)) * (uint32_t)a.W + (uint32_t)(wp - 1)) * (uint32_t)vx + (uint32_t)jx);
+                    wp += sxr;
+                    hp += sxq;
+                    if (wp >= Wp) {
+                        wp -= Wp;
+                        ++hp;
+                    }
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
@@ -584,20 +606,26 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
                     }
                 }
             }
+            hp = (f0 + tid / vz) / Wp;
+            wp = (f0 + tid / vz) - hp * Wp;
             for (int rb = tid / vz; rb < TM; rb += U * stepz) {
                 uint4 raw[U], rawz[U];
                 bool ok[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const int r = rb + u * stepz;
-                    const int f = f0 + r;
-                    const int hp = f / Wp, wp = f - hp * Wp;
-                    ok[u] = r < TM && hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+                    ok[u] = r < TM && (uint32_t)(hp - 1) < (uint32_t)a.H && (uint32_t)(wp - 1) < (uint32_t)a.W;
                     raw[u] = rawz[u] = make_uint4(0, 0, 0, 0);
                     if (ok[u]) {
-                        const size_t e = ((((size_t)img * a.H + (hp - 1)) * a.W + (wp - 1)) * a.CO + (jz << 3)) >> 3;
+                        const uint32_t e = ((img_row0 + (uint32_t)(hp - 1)) * (uint32_t)a.W + (uint32_t)(wp - 1)) * (uint32_t)vz + (uint32_t)jz;
                         raw[u] = __ldg(gdy + e);
                         if (need_z) rawz[u] = __ldg(gz + e);
+                    }
+                    wp += szr;
+                    hp += szq;
+                    if (wp >= Wp) {
+                        wp -= Wp;
+                        ++hp;
                     }
                 }
 #pragma unroll
@@ -620,9 +648,10 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
                 const int t = t_first + tt, r = t / 3, s = t - r * 3;
                 const uint32_t xs = x0 + (uint32_t)(r * Wp + s) * 128u;
                 const uint32_t d = tmem + (uint32_t)(tt * a.CI);
+                const uint64_t dz_const = make_desc_mn_lbo(0, dz_block), x_const = make_desc_mn_lbo(0, x_block);
 #pragma unroll
                 for (int k = 0; k < TM / 16; ++k)
-                    umma_bf16(d, make_desc_mn_lbo(z0 + k * 2048, dz_block), make_desc_mn_lbo(xs + k * 2048, x_block), idesc,
+                    umma_bf16(d, dz_const + (uint64_t)((z0 + k * 2048) >> 4), x_const + (uint64_t)((xs + k * 2048) >> 4), idesc,
                               (tl > tile_beg || k > 0) ? 1u : 0u);
             }
             umma_commit(bar);
@@ -722,7 +751,8 @@ void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16
 }
 
 bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g) {
-    return conv3_tc_supported(dtype, g) && g.ci <= 128 && g.co <= 128;
+    // the kernel indexes 16-byte vectors with 32 bits
+    return conv3_tc_supported(dtype, g) && g.ci <= 128 && g.co <= 128 && (double)g.n * g.hi * g.wi * 16.0 < 4.0e9;
 }
 
 void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
