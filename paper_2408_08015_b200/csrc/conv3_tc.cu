@@ -236,7 +236,6 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
 //
 // so the MMAs of a tile run while the next tile's loads are in flight and the previous tile is being stored.  With 64
 // reduction channels two operand buffers fit and the transform of tile i+1 overlaps the MMAs of tile i as well.
-constexpr int C3P_THREADS = 512;
 constexpr int C3P_NH = 64;             // output channels per CTA
 
 struct C3PArgs {
@@ -250,7 +249,9 @@ struct C3PArgs {
     int tiles_per_img, total_tiles, rows_pad, n_split, nbuf, flip;
 };
 
-template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) conv3_persist_kernel(const C3PArgs a) {
+// NTHR = 512 with one CTA per SM (128 reduction channels: the resident weights take 147 KB), or 256 with two CTAs per SM (64
+// channels: 74 KB of weights and a 31 KB operand buffer each), which then overlap each other's load and barrier waits.
+template <bool BWD, int IT, int NTHR> __global__ void __launch_bounds__(NTHR, NTHR == 256 ? 2 : 1) conv3_persist_kernel(const C3PArgs a) {
     pdl_launch();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2];
@@ -281,7 +282,7 @@ template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) co
     {
         const int vprw = a.C >> 3;
 #pragma unroll 4
-        for (int v = tid; v < 9 * C3P_NH * vprw; v += C3P_THREADS) {
+        for (int v = tid; v < 9 * C3P_NH * vprw; v += NTHR) {
             const int t = v / (C3P_NH * vprw), rem = v - t * (C3P_NH * vprw);
             const int n = rem / vprw, j = rem - n * vprw;
             const int wt = a.flip ? 8 - t : t;
@@ -299,7 +300,7 @@ template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) co
 
     // staging role: one 16-byte channel chunk (coefficients in registers), every (512 / chunks)-th row
     const int vpr = a.C >> 3;
-    const int j = tid % vpr, step = C3P_THREADS / vpr, r_first = tid / vpr;
+    const int j = tid % vpr, step = NTHR / vpr, r_first = tid / vpr;
     const int c0 = j << 3;
     const bool need_z = BWD && grad_needs_z(a.dz);
     XfVal xv;
@@ -371,13 +372,17 @@ template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) co
         }
         umma_commit(bar[acc]);
     };
-    // 16 warps: warp & 3 = tensor-memory lane quarter (32 positions), warp >> 2 = 16 of the 64 output channels
+    // warp & 3 = tensor-memory lane quarter (32 positions), warp >> 2 = which share of the 64 output channels (16 or 32 of them)
     auto epilogue = [&](int tl, int acc) {
         const int img = tl / a.tiles_per_img, tile = tl - img * a.tiles_per_img;
-        const int q = warp & 3, cg = warp >> 2;
+        const int q = warp & 3;
         const int f = Wp + 1 + tile * TM + q * 32 + lane;
         const int hp = f / Wp, wp = f - hp * Wp;
         const bool pix = hp >= 1 && hp <= a.H && wp >= 1 && wp <= a.W;
+        constexpr int CHUNKS = C3P_NH / 16 / (NTHR / 128);       // 16-column chunks per warp
+#pragma unroll
+        for (int ch = 0; ch < CHUNKS; ++ch) {
+        const int cg = (warp >> 2) * CHUNKS + ch;
         float v[16];
         tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * C3P_NH + (cg << 4)), v);
         if (pix) {
@@ -396,6 +401,7 @@ template <bool BWD, int IT> __global__ void __launch_bounds__(C3P_THREADS, 1) co
                 }
                 *reinterpret_cast<uint4*>(a.out + e) = pack8(vv);
             }
+        }
         }
     };
 
@@ -451,8 +457,9 @@ bool plan_c3p(const C3Args& a, C3PArgs& p, size_t* smem, int* it) {
     if (a.C > 128 || a.C % 64 || a.N % C3P_NH) return false;
     const int Wp = a.W + 2, rows = TM + 2 * Wp + 2;
     const int kbs = a.C / 64;
-    *it = a.C == 64 ? 4 : 8;
-    if (rows > *it * (C3P_THREADS / (a.C >> 3))) return false;
+    *it = 8;                                            // items per thread: 256 threads x 8 chunks (C = 64) or 512 x 16 (C = 128)
+    const int nthr = a.C == 64 ? 256 : 512;
+    if (rows > *it * (nthr / (a.C >> 3))) return false;
     if ((double)a.n_img * a.H * a.W * (a.C > a.N ? a.C : a.N) / 8.0 >= 4.0e9) return false;      // 32-bit vector indices
     p.x = a.x; p.dz = a.dz; p.w = a.w; p.addend = a.addend; p.out = a.out; p.err = a.err;
     p.n_img = a.n_img; p.H = a.H; p.W = a.W; p.C = a.C; p.N = a.N; p.flip = a.flip;
@@ -462,9 +469,9 @@ bool plan_c3p(const C3Args& a, C3PArgs& p, size_t* smem, int* it) {
     p.n_split = a.N / C3P_NH;
     const size_t wbytes = 9 * (size_t)kbs * C3P_NH * 128, abuf = (size_t)kbs * p.rows_pad * 128;
     const size_t budget = 225 * 1024;
-    p.nbuf = wbytes + 2 * abuf + 1024 <= budget ? 2 : 1;
+    p.nbuf = 1;
     *smem = wbytes + p.nbuf * abuf + 1024;
-    return *smem <= budget;
+    return *smem <= (a.C == 64 ? budget / 2 : budget);
 }
 
 template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, double useful_flops, cudaStream_t st) {
@@ -473,15 +480,16 @@ template <bool BWD> void launch_c3(C3Args& a, int kind, double bytes, double use
         size_t psmem = 0;
         int it = 0;
         if (plan_c3p(a, p, &psmem, &it)) {
-            smem_limit_once<106 + (BWD ? 50 : 0)>(conv3_persist_kernel<BWD, 4>, 226 * 1024);
-            smem_limit_once<107 + (BWD ? 50 : 0)>(conv3_persist_kernel<BWD, 8>, 226 * 1024);
+            smem_limit_once<106 + (BWD ? 50 : 0)>(conv3_persist_kernel<BWD, 8, 256>, 113 * 1024);
+            smem_limit_once<107 + (BWD ? 50 : 0)>(conv3_persist_kernel<BWD, 8, 512>, 226 * 1024);
             const int n_sm = sm_count();
-            int nctas = n_sm / p.n_split;
+            const bool two = a.C == 64;                     // two 256-thread CTAs per SM
+            int nctas = (two ? 2 * n_sm : n_sm) / p.n_split;
             if (nctas < 1) nctas = 1;
             if (nctas > p.total_tiles) nctas = p.total_tiles;
             LaunchScope ls(kind, bytes, useful_flops > 0 ? useful_flops : 2.0 * 9.0 * a.n_img * a.H * a.W * (double)a.C * a.N, st);
-            if (it == 4) launch_pdl(conv3_persist_kernel<BWD, 4>, nctas * p.n_split, C3P_THREADS, psmem, st, p);
-            else launch_pdl(conv3_persist_kernel<BWD, 8>, nctas * p.n_split, C3P_THREADS, psmem, st, p);
+            if (two) launch_pdl(conv3_persist_kernel<BWD, 8, 256>, nctas * p.n_split, 256, psmem, st, p);
+            else launch_pdl(conv3_persist_kernel<BWD, 8, 512>, nctas * p.n_split, 512, psmem, st, p);
             return;
         }
     }
