@@ -319,7 +319,7 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
         one_round(sets[0])
     # repeats: the timed region lasts about MIN_TIMED_S (every rank takes the same count: it comes from rank 0's probe)
     probe = timed(lambda: one_round(sets[0]), 2) / 2
-    rep = max(1, int(np.ceil(MIN_TIMED_S * 1e3 / max(probe * args.steps, 1e-3))))
+    rep = max(1, int(np.ceil(args.min_seconds * 1e3 / max(probe * args.steps, 1e-3))))
     if dist is not None:
         t = torch.tensor([rep], device=dev)
         dist.broadcast(t, 0)
@@ -396,7 +396,7 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
             "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
             "config": {"workload": wl.name, "samples_per_step_per_gpu": Bn * Mn, "parallelism": "replicas only" if world > 1 else "single GPU",
                        "steps_timed": steps_timed,
-                       "timed_region": "%d x %d steps so that it lasts about %.0f s; ms_per_step is their mean" % (rep, args.steps, MIN_TIMED_S),
+                       "timed_region": "%d x %d steps so that it lasts about %.0f s; ms_per_step is their mean" % (rep, args.steps, args.min_seconds),
                        "l2": ("no flush: each step streams its activation slots and gradients, far beyond the 126 MB L2" if wl.cfg != 1 else
                               "no flush and smaller than L2: a step touches about 30 MB, so this workload is launch- and latency-bound by construction")},
             "clocks": clocks,
@@ -448,6 +448,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="all", choices=["1", "2", "3", "4", "all"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
+                    help="the K timed steps are repeated until the timed region lasts about this long (0: exactly K steps)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

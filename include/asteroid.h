@@ -183,6 +183,45 @@ typedef struct {
 int asteroid_trace_start(void);
 int asteroid_trace_stop(ast_kernel_stat* out, int capacity, int* n_out);
 
+/* ---- Parallelism planning (Section 3.3, "Parallelism Planning"), host only --------------------------------------------
+ * Input: the profiler's cost tables per device type (FP / BP milliseconds of every layer at the profiled batch sizes;
+ * times between profiled sizes are interpolated linearly, 0 at batch 0, the last segment continued beyond the largest),
+ * per layer the output bytes per sample a_l, the parameter bytes w_l and the bytes kept per sample for BP; the device
+ * pool (type and memory budget of each device, pairwise bandwidth in bytes per millisecond); micro-batch size B,
+ * micro-batches per round M, and the block of samples the offloading phase moves at a time.
+ * All pointers are HOST pointers owned by the caller.  Layouts: t_f, t_b [n_types][L][n_bs]; bw [N][N].
+ * Memory of a device holding layers i..j with y samples as the stage K-th from the end (Eq. (3)):
+ *     (mod_factor + opt_factor) * sum w_l + (2K - 1) * y * sum act_l  <=  dev_mem.                                  */
+#define AST_PLAN_MAX_DEVICES 64
+typedef struct {
+    int32_t L, n_types, n_bs, N, B, M, block;
+    const int32_t* bs;
+    const double *t_f, *t_b;
+    const double *a, *w, *act;
+    double mod_factor, opt_factor;
+    const int32_t* dev_type;
+    const double* dev_mem;
+    const double* bw;
+} ast_plan_problem;
+
+/* The chosen hybrid pipeline: n_stages stages in pipeline order; stage s runs layers first_layer[s]..last_layer[s]
+ * data-parallel on devices[dev_begin[s] .. dev_begin[s+1]) (indices into the caller's device arrays), device
+ * devices[q] taking samples[q] of every micro-batch.  e_f/e_b/t_a: FP, BP and AllReduce milliseconds of the stage
+ * (Eq. (5), (8)); dominant_step indexes the step list exec, comm, exec, ... (Eq. (11)); latency_ms is the estimated
+ * HPP-Round latency (Eq. (4)).  n_stages == 0 with infinite latency: no configuration fits the memory budgets. */
+typedef struct {
+    double latency_ms;
+    int32_t n_stages, n_steps, dominant_step, reserved;
+    int32_t first_layer[AST_PLAN_MAX_DEVICES], last_layer[AST_PLAN_MAX_DEVICES], dev_begin[AST_PLAN_MAX_DEVICES + 1];
+    int32_t devices[AST_PLAN_MAX_DEVICES], samples[AST_PLAN_MAX_DEVICES];
+    double e_f_ms[AST_PLAN_MAX_DEVICES], e_b_ms[AST_PLAN_MAX_DEVICES], t_a_ms[AST_PLAN_MAX_DEVICES];
+} ast_plan_result;
+
+/* Algorithm 2 (dynamic programming over layers, devices in descending order of memory, and stage count; Eq. (10)) with
+ * Algorithm 1 (memory-aware balancing, then straggler offloading; Eq. (7)-(9)) for every candidate stage.
+ * Errors: AST_ERR_ARG (null table, non-positive size, more than 64 devices, batch sizes not ascending, bad device type). */
+int asteroid_plan(const ast_plan_problem* problem, ast_plan_result* result);
+
 /* Self-test of the bounded device-side waits (the paper has no counterpart).  Every hand-off wait inside the
  * tensor-core kernels gives up after a fixed number of polls, sets the stage's error word and lets the kernel
  * return, which export_state then reports as AST_ERR_TIMEOUT.  This call runs that mechanism on purpose: one

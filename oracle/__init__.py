@@ -15,7 +15,10 @@ Pins (tests/test_oracle_*.py): brute-force direct convolution, central finite
 differences, adjoint identities, BatchNorm closed forms and invariants, loss
 special cases, closed-form SGD steps, the micro-batch accumulation invariant,
 agreement with torch.autograd in float64 on whole stages, and the K_p values the
-paper prints for a three-stage pipeline.  No function here is unpinned.
+paper prints for a three-stage pipeline; the storage-mirroring mode by tests/test_oracle_mirror.py;
+the planner (oracle/planner.py) by closed forms and exhaustive search on tiny instances
+(tests/test_oracle_planner.py).  No function here is unpinned.
 """
 from .layers import *      # noqa: F401,F403
 from .stage import *       # noqa: F401,F403
+from . import planner       # noqa: F401

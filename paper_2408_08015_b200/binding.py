@@ -14,7 +14,7 @@ EXPORTS = ["asteroid_stage_create", "asteroid_stage_destroy", "asteroid_stage_pa
            "asteroid_stage_export_bn_running", "asteroid_stage_forward", "asteroid_stage_backward",
            "asteroid_stage_accumulate", "asteroid_stage_step", "asteroid_stage_profile",
            "asteroid_loss_mse", "asteroid_loss_mse_noalloc", "asteroid_loss_softmax_xent", "asteroid_trace_start", "asteroid_trace_stop",
-           "asteroid_selftest_bounded_wait", "asteroid_launch_count", "asteroid_last_error"]
+           "asteroid_selftest_bounded_wait", "asteroid_plan", "asteroid_launch_count", "asteroid_last_error"]
 
 
 class ast_layer(C.Structure):
@@ -36,6 +36,24 @@ class ast_layer_profile(C.Structure):
 class ast_kernel_stat(C.Structure):
     _fields_ = [("name", C.c_char * 48), ("launches", C.c_uint64), ("total_ms", C.c_double),
                 ("alg_bytes", C.c_double), ("flops", C.c_double)]
+
+
+PLAN_MAX_DEVICES = 64
+
+
+class ast_plan_problem(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("L", "n_types", "n_bs", "N", "B", "M", "block")] + \
+               [("bs", C.POINTER(C.c_int32)), ("t_f", C.POINTER(C.c_double)), ("t_b", C.POINTER(C.c_double)),
+                ("a", C.POINTER(C.c_double)), ("w", C.POINTER(C.c_double)), ("act", C.POINTER(C.c_double)),
+                ("mod_factor", C.c_double), ("opt_factor", C.c_double), ("dev_type", C.POINTER(C.c_int32)),
+                ("dev_mem", C.POINTER(C.c_double)), ("bw", C.POINTER(C.c_double))]
+
+
+class ast_plan_result(C.Structure):
+    _fields_ = [("latency_ms", C.c_double), ("n_stages", C.c_int32), ("n_steps", C.c_int32), ("dominant_step", C.c_int32), ("reserved", C.c_int32),
+                ("first_layer", C.c_int32 * PLAN_MAX_DEVICES), ("last_layer", C.c_int32 * PLAN_MAX_DEVICES), ("dev_begin", C.c_int32 * (PLAN_MAX_DEVICES + 1)),
+                ("devices", C.c_int32 * PLAN_MAX_DEVICES), ("samples", C.c_int32 * PLAN_MAX_DEVICES),
+                ("e_f_ms", C.c_double * PLAN_MAX_DEVICES), ("e_b_ms", C.c_double * PLAN_MAX_DEVICES), ("t_a_ms", C.c_double * PLAN_MAX_DEVICES)]
 
 
 class AsteroidError(RuntimeError):
@@ -77,6 +95,7 @@ def lib():
         L.asteroid_trace_start.argtypes = []
         L.asteroid_trace_stop.argtypes = [C.POINTER(ast_kernel_stat), i, C.POINTER(i)]
         L.asteroid_selftest_bounded_wait.argtypes = []
+        L.asteroid_plan.argtypes = [C.POINTER(ast_plan_problem), C.POINTER(ast_plan_result)]
         L.asteroid_launch_count.argtypes = []
         L.asteroid_launch_count.restype = C.c_uint64
         L.asteroid_last_error.argtypes = []
@@ -191,6 +210,34 @@ def asteroid_trace_stop():
 def asteroid_selftest_bounded_wait():
     """Return code of the bounded-wait self-test (AST_ERR_TIMEOUT is the expected outcome); does not raise."""
     return lib().asteroid_selftest_bounded_wait()
+
+
+def asteroid_plan(prob):
+    """`prob`: the dict form of a planning problem (keys L, B, M, block, bs, t_f[type][l][k], t_b, a, w, act, mod_factor, opt_factor,
+    devices [{type, mem}], bw[d][d']).  Returns {"latency", "dm", "stages": [{"layers": (i, j), "devices": [...], "y": [...],
+    "ef", "eb", "ta"}]} or None when nothing fits.  Marshalling only: the planning runs in the library."""
+    import numpy as np
+    L, N = int(prob["L"]), len(prob["devices"])
+    bs = np.ascontiguousarray(prob["bs"], np.int32)
+    tf = np.ascontiguousarray(prob["t_f"], np.float64)
+    tb = np.ascontiguousarray(prob["t_b"], np.float64)
+    a, w, act = (np.ascontiguousarray(prob[k], np.float64) for k in ("a", "w", "act"))
+    dt = np.ascontiguousarray([d["type"] for d in prob["devices"]], np.int32)
+    dm = np.ascontiguousarray([d["mem"] for d in prob["devices"]], np.float64)
+    bw = np.ascontiguousarray(prob["bw"], np.float64)
+    dp, ip = (lambda x: x.ctypes.data_as(C.POINTER(C.c_double))), (lambda x: x.ctypes.data_as(C.POINTER(C.c_int32)))
+    p = ast_plan_problem(L, tf.shape[0], bs.size, N, int(prob["B"]), int(prob["M"]), int(prob["block"]), ip(bs), dp(tf), dp(tb), dp(a), dp(w), dp(act),
+                         float(prob["mod_factor"]), float(prob["opt_factor"]), ip(dt), dp(dm), dp(bw))
+    r = ast_plan_result()
+    _check(lib().asteroid_plan(C.byref(p), C.byref(r)))
+    if r.n_stages == 0:
+        return None
+    stages = []
+    for s in range(r.n_stages):
+        q0, q1 = r.dev_begin[s], r.dev_begin[s + 1]
+        stages.append({"layers": (r.first_layer[s], r.last_layer[s]), "devices": list(r.devices[q0:q1]), "y": list(r.samples[q0:q1]),
+                       "ef": r.e_f_ms[s], "eb": r.e_b_ms[s], "ta": r.t_a_ms[s]})
+    return {"latency": r.latency_ms, "dm": r.dominant_step, "n_steps": r.n_steps, "stages": stages}
 
 
 def asteroid_launch_count():

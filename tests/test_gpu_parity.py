@@ -33,7 +33,7 @@ def run_case(net, h, w, B, M, loss, bf16, seed=0, first=0, last=None, allow=(CON
              contract_kinds=("y", "loss"), **kw):
     last = len(net) - 1 if last is None else last
     xs, tg, params, _ = make_inputs(net, first, last, h, w, B, M, loss, seed, bf16)
-    okw = {k: v for k, v in kw.items() if k in ("order", "rounds")}
+    okw = {k: v for k, v in kw.items() if k in ("order", "rounds", "lr")}
     plain = oracle_round(net, first, last, B, M, loss, xs, tg, params, **okw)
     mirror = oracle_round(net, first, last, B, M, loss, xs, tg, params, store=bf16_store, **okw) if bf16 else None
     gpu = gpu_round(net, first, last, h, w, B, M, loss, xs, tg, params, bf16, **kw)
@@ -73,6 +73,19 @@ def test_config1_block_fp32():
 
 def test_config1_two_rounds_momentum():
     print(summary(run_case(si.block_net(16, 6), 32, 32, 8, 4, "mse", False, rounds=2, case="config1/f32/two_rounds")))
+
+
+@pytest.mark.parametrize("name", ["stem_c3", "block_c16", "c3_64_64"])
+def test_two_rounds_bf16_second_round_sees_the_updated_weights(name):
+    """Several kernels stage their weights before they wait for the previous kernel in the stream; the kernels that rewrite
+    the weight copies after an update therefore never release their dependents early.  Two rounds back to back, on a stage
+    whose first kernel after the update is a memcpy + the im2col kernel (3 input channels), a slot-copy kernel (16) or a
+    resident-weight 3x3 pipeline (64): the second round must have used the updated weights."""
+    net, h, w = {"stem_c3": (si.single_unit_net("conv", 3, 32, k=3, stride=2, bn=True, act="relu6"), 33, 31),
+                 "block_c16": (si.block_net(16, 6), 12, 12),
+                 "c3_64_64": (si.single_unit_net("conv", 64, 64, k=3, bn=True, act="relu"), 14, 13)}[name]
+    r = run_case(net, h, w, 3, 2, "mse", True, rounds=2, allow=(CONTRACT, MIRROR), case="two_rounds/%s/bf16" % name, lr=5.0)
+    print(name, summary(r))
 
 
 def test_config2_stage_bf16_full_size():

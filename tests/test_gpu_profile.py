@@ -64,3 +64,24 @@ def test_full_resolution_partitions_match_oracle(parts):
         print((first, last), summary(compare(gpu, plain, net, first, last, 2e-2, need_dx=first > 0, mirror=mirror, allow=ALL, outlier_frac=5e-4,
                                              case="config5/P%d/%d-%d/B4" % (parts, first, last),
                                              contract_kinds=("loss",) if parts == 2 else ("y", "loss"))))
+
+
+def test_planner_on_measured_cost_tables_equals_the_oracle():
+    """Section 3.3 end to end: profile a small network's block-level units on this GPU at three batch sizes, hand the tables
+    to the library's planner and to the planning oracle with the same synthetic device pool: same pipeline, same latency."""
+    import paper_2408_08015_b200 as P
+    from paper_2408_08015_b200.sweep import plan_problem, unit_cost_tables
+    from oracle import planner as PL
+    net, units = si.small_mobilenet(10)
+    batches = [2, 4, 8]
+    tabs = unit_cost_tables(P, si, net, units, 32, 32, batches)
+    assert all(t > 0 for row in tabs[0] for t in row) and all(t > 0 for row in tabs[1] for t in row)
+    for kw in ({"devices": ((0, 1e9), (1, 1e9), (2, 1e9)), "B": 8, "M": 4, "block": 1},
+               {"devices": ((0, 2e5), (1, 1.5e5), (1, 1.5e5), (2, 1e5)), "B": 8, "M": 4, "block": 1, "bytes_per_ms": 1e3}):
+        prob = plan_problem(*tabs, batches, **kw)
+        got, ref = P.asteroid_plan(prob), PL.plan(prob)
+        assert (got is None) == (ref is None)
+        if ref is not None:
+            assert got["latency"] == pytest.approx(ref["latency"], rel=1e-12)
+            assert [(tuple(s["layers"]), s["devices"], s["y"]) for s in got["stages"]] == [(tuple(s["layers"]), s["devices"], s["y"]) for s in ref["stages"]]
+            print(kw["devices"], "->", [(s["layers"], s["devices"], s["y"]) for s in got["stages"]], "%.3f ms" % got["latency"])
