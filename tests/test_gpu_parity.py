@@ -84,7 +84,9 @@ def test_two_rounds_bf16_second_round_sees_the_updated_weights(name):
     net, h, w = {"stem_c3": (si.single_unit_net("conv", 3, 32, k=3, stride=2, bn=True, act="relu6"), 33, 31),
                  "block_c16": (si.block_net(16, 6), 12, 12),
                  "c3_64_64": (si.single_unit_net("conv", 64, 64, k=3, bn=True, act="relu"), 14, 13)}[name]
-    r = run_case(net, h, w, 3, 2, "mse", True, rounds=2, allow=(CONTRACT, MIRROR), case="two_rounds/%s/bf16" % name, lr=5.0)
+    # lr = 5 moves the weights by tens of per cent, so stale weights in round 2 would miss the contract on y outright; the
+    # same step also multiplies round 1's rounding-level gradient differences into round 2, hence all criteria for gradients
+    r = run_case(net, h, w, 3, 2, "mse", True, rounds=2, allow=ALL, outlier_frac=5e-4, case="two_rounds/%s/bf16" % name, lr=5.0)
     print(name, summary(r))
 
 
