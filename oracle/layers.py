@@ -9,7 +9,7 @@ import numpy as np
 __all__ = ["conv2d_forward", "conv2d_backward", "dwconv2d_forward", "dwconv2d_backward",
            "bn_forward", "bn_backward", "act_forward", "act_backward", "gap_forward",
            "gap_backward", "linear_forward", "linear_backward", "mse_loss",
-           "softmax_xent_loss", "sgd_momentum_step", "warmup_forwards", "stage_memory"]
+           "softmax_xent_loss", "sgd_momentum_step", "warmup_forwards", "stage_memory", "sigmoid", "se_forward", "se_backward"]
 
 
 def _out_size(n, k, stride, pad):
@@ -111,16 +111,56 @@ def act_forward(kind, pre):
         return np.minimum(np.maximum(pre, 0.0), 6.0)
     if kind == "relu":
         return np.maximum(pre, 0.0)
+    if kind == "silu":
+        return pre * sigmoid(pre)
     raise ValueError(kind)
 
 
+def sigmoid(x):
+    return 1.0 / (1.0 + np.exp(-x))
+
+
 def act_backward(kind, dy, pre):
-    """Gradient passes only strictly inside the linear region (0 at the kinks)."""
+    """ReLU / ReLU6: gradient passes only strictly inside the linear region (0 at the kinks).
+    SiLU x*sigmoid(x): derivative sigmoid(x) * (1 + x * (1 - sigmoid(x)))."""
     if kind == "relu6":
         return dy * ((pre > 0.0) & (pre < 6.0))
     if kind == "relu":
         return dy * (pre > 0.0)
+    if kind == "silu":
+        sg = sigmoid(pre)
+        return dy * sg * (1.0 + pre * (1.0 - sg))
     raise ValueError(kind)
+
+
+def se_forward(x, w1, b1, w2, b2):
+    """Squeeze-and-excitation of the EfficientNet block (one of the paper's vision workloads, Section 5.1): per sample
+    s[n,c] = mean_{h,w} x;  h = silu(s w1^T + b1);  g = sigmoid(h w2^T + b2);  out[n,h,w,c] = x[n,h,w,c] * g[n,c].
+    Returns (out, cache)."""
+    s = x.mean(axis=(1, 2))
+    p1 = s @ w1.T + b1
+    h = p1 * sigmoid(p1)
+    p2 = h @ w2.T + b2
+    g = sigmoid(p2)
+    return x * g[:, None, None, :], (s, p1, h, g)
+
+
+def se_backward(x, w1, w2, cache, dout):
+    """Adjoint of se_forward: returns (dx, dw1, db1, dw2, db2)."""
+    s, p1, h, g = cache
+    hw = x.shape[1] * x.shape[2]
+    dg = (dout * x).sum(axis=(1, 2))
+    dp2 = dg * g * (1.0 - g)
+    dw2 = dp2.T @ h
+    db2 = dp2.sum(axis=0)
+    dh = dp2 @ w2
+    sg = sigmoid(p1)
+    dp1 = dh * sg * (1.0 + p1 * (1.0 - sg))
+    dw1 = dp1.T @ s
+    db1 = dp1.sum(axis=0)
+    ds = dp1 @ w1
+    dx = dout * g[:, None, None, :] + (ds / hw)[:, None, None, :]
+    return dx, dw1, db1, dw2, db2
 
 
 def gap_forward(x):

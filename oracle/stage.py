@@ -7,7 +7,7 @@ from the definitions in `layers.py`; nothing is fused, blocked or reordered.
 
 Flat parameter order (the interchange format with any other implementation): layers in list
 order; conv weight [c_out][k][k][c_in]; depthwise weight [c][k][k]; bn gamma, beta; linear
-weight [c_out][c_in], bias.
+weight [c_out][c_in], bias; squeeze-excite w1 [k][c], b1 [k], w2 [c][k], b2 [c].
 """
 import numpy as np
 from . import layers as L
@@ -25,6 +25,8 @@ def _layer_param_shapes(layer):
         return [("gamma", (layer.c_out,)), ("beta", (layer.c_out,))]
     if op == "linear":
         return [("weight", (layer.c_out, layer.c_in)), ("bias", (layer.c_out,))]
+    if op == "se":                # squeeze width in the layer's k field
+        return [("w1", (layer.k, layer.c_out)), ("b1", (layer.k,)), ("w2", (layer.c_out, layer.k)), ("b2", (layer.c_out,))]
     return []
 
 
@@ -41,8 +43,10 @@ class Stage:
     BatchNorm), the output of a residual add (after the ReLU that directly follows it, if any),
     the pooled features, the stage output, and the gradient with respect to each of those
     stored-or-recomputed unit outputs and to the stage input (rounded after every term added
-    to it).  BatchNorm and activation outputs inside a conv->BN->activation chain are never
-    stored.  store=None is the plain float64 definition.
+    to it).  BatchNorm and ReLU/ReLU6 outputs inside a conv->BN->activation chain are never
+    stored; a SiLU is not part of a chain: its output and the output of a squeeze-excite layer are
+    stored tensors (the squeeze-excite layer's per-sample vectors are not rounded).
+    store=None is the plain float64 definition.
 
     `operand`: optional rounding applied to both operands of every dense contraction (conv and
     linear layers, in FP, in the input-gradient product and in the weight-gradient product; not the
@@ -84,7 +88,7 @@ class Stage:
         if b.src != i:
             return False
         if a.op in _CONVLIKE:
-            return b.op == "bn" or b.op in _ACTS
+            return b.op == "bn" or b.op in _ACTS      # _ACTS holds the chain-fused activations only (not silu)
         if a.op == "bn":
             return b.op in _ACTS and i - 1 >= self.first and self.net[i - 1].op in _CONVLIKE and a.src == i - 1
         if a.op == "add":
@@ -99,6 +103,8 @@ class Stage:
             return not self._chains_into_next(i)
         if op == "relu":
             return i - 1 >= self.first and self.net[i - 1].op == "add" and self.net[i].src == i - 1
+        if op in ("silu", "se"):
+            return True
         return False
 
     # ---- flat views -------------------------------------------------------------------
@@ -138,8 +144,10 @@ class Stage:
                 rm, rv = self.running[i]
                 self.running[i] = [(1 - self.bn_momentum) * rm + self.bn_momentum * mu,
                                    (1 - self.bn_momentum) * rv + self.bn_momentum * var * cnt / max(cnt - 1, 1)]
-            elif ly.op in ("relu6", "relu"):
+            elif ly.op in ("relu6", "relu", "silu"):
                 val[i] = L.act_forward(ly.op, a)
+            elif ly.op == "se":
+                val[i], cache[i] = L.se_forward(a, self.p[(i, "w1")], self.p[(i, "b1")], self.p[(i, "w2")], self.p[(i, "b2")])
             elif ly.op == "add":
                 val[i] = a + val[ly.add_from]
             elif ly.op == "gap":
@@ -180,8 +188,11 @@ class Stage:
             elif ly.op == "bn":
                 dz, g[(i, "gamma")], g[(i, "beta")] = L.bn_backward(d, cache[i], self.p[(i, "gamma")], self.eps)
                 give(ly.src, dz)
-            elif ly.op in ("relu6", "relu"):
+            elif ly.op in ("relu6", "relu", "silu"):
                 give(ly.src, L.act_backward(ly.op, d, a))
+            elif ly.op == "se":
+                dx, g[(i, "w1")], g[(i, "b1")], g[(i, "w2")], g[(i, "b2")] = L.se_backward(a, self.p[(i, "w1")], self.p[(i, "w2")], cache[i], d)
+                give(ly.src, dx)
             elif ly.op == "add":
                 give(ly.src, d)
                 give(ly.add_from, d)

@@ -15,7 +15,7 @@ from collections import namedtuple
 Layer = namedtuple("Layer", "op c_in c_out k stride pad src add_from")
 
 # integer codes shared with the C header's enum (values fixed by that header)
-OPS = {"conv": 0, "dwconv": 1, "bn": 2, "relu6": 3, "relu": 4, "add": 5, "gap": 6, "linear": 7}
+OPS = {"conv": 0, "dwconv": 1, "bn": 2, "relu6": 3, "relu": 4, "add": 5, "gap": 6, "linear": 7, "silu": 8, "se": 9}
 
 
 class _Builder:
@@ -35,8 +35,15 @@ class _Builder:
     def conv(self, c_in, c_out, k, stride=1, pad=None, src=None):
         return self._push("conv", c_in, c_out, k, stride, (k - 1) // 2 if pad is None else pad, src)
 
-    def dwconv(self, c, stride=1, src=None):
-        return self._push("dwconv", c, c, 3, stride, 1, src)
+    def dwconv(self, c, stride=1, src=None, k=3):
+        return self._push("dwconv", c, c, k, stride, (k - 1) // 2, src)
+
+    def silu(self, c):
+        return self._push("silu", c, c)
+
+    def se(self, c, squeeze):
+        """Squeeze-excite over c channels with `squeeze` hidden units (kept in the record's k field)."""
+        return self._push("se", c, c, squeeze)
 
     def bn(self, c):
         return self._push("bn", c, c)
@@ -76,6 +83,36 @@ def inverted_residual(b, c_in, c_out, stride, t, use_bn=True, act="relu6"):
     if stride == 1 and c_in == c_out:
         b.add(c_out, src=b.last, add_from=x)
     return b.last
+
+
+def mbconv(b, c_in, c_out, stride, t, k, se_ratio=0.25):
+    """Append one EfficientNet MBConv block: 1x1 expand + BN + SiLU, k x k depthwise + BN + SiLU, squeeze-excite with
+    max(1, c_in * se_ratio) hidden units, 1x1 project + BN, residual add when the shapes allow."""
+    x = b.last
+    hid = c_in * t
+    if t != 1:
+        b.conv(c_in, hid, 1); b.bn(hid); b.silu(hid)
+    b.dwconv(hid, stride, k=k); b.bn(hid); b.silu(hid)
+    b.se(hid, max(1, int(c_in * se_ratio)))
+    b.conv(hid, c_out, 1); b.bn(c_out)
+    if stride == 1 and c_in == c_out:
+        b.add(c_out, src=b.last, add_from=x)
+    return b.last
+
+
+def mbconv_net(c_in, blocks):
+    """A stage of MBConv blocks [(c_out, stride, expand, kernel)]."""
+    b = _Builder()
+    for c_out, stride, t, k in blocks:
+        mbconv(b, c_in, c_out, stride, t, k)
+        c_in = c_out
+    return b.layers
+
+
+def efficientnet_b1_stage_net():
+    """EfficientNet-B1-style stage (the paper's third vision workload, Section 5.1): the 5x5 and the first 3x3 MBConv6 groups,
+    24 -> 40 (stride 2, then two more) -> 80 (stride 2, then one more), for a 56x56x24 input."""
+    return mbconv_net(24, [(40, 2, 6, 5), (40, 1, 6, 5), (40, 1, 6, 5), (80, 2, 6, 3), (80, 1, 6, 3)])
 
 
 def block_net(c=16, t=6):
@@ -168,18 +205,20 @@ def small_mobilenet(classes=10):
     return _mobilenetv2(classes, [(1, 8, 1, 1), (2, 8, 2, 2), (2, 16, 1, 1)], stem_c=8, head_c=32)
 
 
-def single_unit_net(kind, c_in, c_out, k=1, stride=1, bn=False, act=None):
+def single_unit_net(kind, c_in, c_out, k=1, stride=1, bn=False, act=None, se=0):
     """One conv (or depthwise conv) layer, optionally followed by BatchNorm and an activation: the
     smallest stage that exercises one contraction / stencil kernel path in both directions."""
     b = _Builder()
     if kind == "dwconv":
-        b.dwconv(c_in, stride)
+        b.dwconv(c_in, stride, k=k if k > 1 else 3)
     else:
         b.conv(c_in, c_out, k, stride, pad=(k - 1) // 2)
     if bn:
         b.bn(c_out)
     if act:
         getattr(b, act)(c_out)
+    if se:
+        b.se(c_out, se)
     return b.layers
 
 

@@ -5,8 +5,9 @@ Flat order: layers in list order; per layer (weight, [bias], gamma, beta):
   dwconv  weight [c][k][k]
   bn      gamma [c], beta [c]
   linear  weight [c_out][c_in], bias [c_out]
-Conv and linear weights ~ U(-b, b), b = sqrt(6 / fan_in), fan_in = k*k*c_in/groups;
-gamma = 1, beta = 0, bias = 0.  The stream of a layer's weight is keyed by its index
+  se      w1 [k][c], b1 [k], w2 [c][k], b2 [c]      (k = squeeze width)
+Conv, linear and squeeze-excite weights ~ U(-b, b), b = sqrt(6 / fan_in), fan_in = k*k*c_in/groups;
+gamma = 1, beta = 0, biases = 0.  The stream of a layer's weight is keyed by its index
 in the whole network, so a stage cut out of a network sees the same values.
 """
 import numpy as np
@@ -30,6 +31,11 @@ def param_layout(net, first, last):
         elif L.op == "linear":
             out.append((i, "weight", (L.c_out, L.c_in)))
             out.append((i, "bias", (L.c_out,)))
+        elif L.op == "se":
+            out.append((i, "w1", (L.k, L.c_out)))
+            out.append((i, "b1", (L.k,)))
+            out.append((i, "w2", (L.c_out, L.k)))
+            out.append((i, "b2", (L.c_out,)))
     return out
 
 
@@ -47,6 +53,9 @@ def init_params(net, first, last, seed=0):
             fan_in = {"conv": L.k * L.k * L.c_in, "dwconv": L.k * L.k, "linear": L.c_in}[L.op]
             b = np.sqrt(6.0 / fan_in)
             parts.append(((2.0 * uniform(seed, _PARAM_TID + i, n) - 1.0) * b).astype(np.float32))
+        elif name in ("w1", "w2"):
+            b = np.sqrt(6.0 / shape[1])
+            parts.append(((2.0 * uniform(seed, (4 if name == "w1" else 5) * _PARAM_TID + i, n) - 1.0) * b).astype(np.float32))
         elif name == "gamma":
             parts.append(np.ones(n, np.float32))
         else:

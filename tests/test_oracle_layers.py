@@ -244,3 +244,44 @@ def test_warmup_forwards_matches_paper_example():
         assert O.warmup_forwards(int(P), int(p)) == int(k)
     assert O.warmup_forwards(1, 0) == 1          # a single stage keeps one micro-batch resident
     assert O.stage_memory(10, 4, 7, 5) == 10 + 4 + 5 * 7      # Eq. (3)
+
+
+def test_silu_values_and_fd():
+    x = np.array([-30.0, -1.0, 0.0, 1.0, 30.0])
+    y = O.act_forward("silu", x)
+    assert abs(y[0]) < 1e-10 and y[2] == 0.0 and abs(y[4] - 30.0) < 1e-10
+    assert np.allclose(y[[1, 3]], [-1.0 / (1.0 + np.e), 1.0 / (1.0 + 1.0 / np.e)], rtol=0, atol=1e-15)       # x * sigmoid(x) at -1 and 1
+    assert np.allclose(O.act_forward("silu", x) - O.act_forward("silu", -x), x, rtol=0, atol=1e-12)           # silu(x) - silu(-x) = x
+    rng = np.random.default_rng(3)
+    pre = rng.normal(size=(2, 3, 3, 4)) * 3
+    dy = rng.normal(size=pre.shape)
+    g = fd_grad(lambda: float((O.act_forward("silu", pre) * dy).sum()), pre)
+    assert_close_rel(O.act_backward("silu", dy, pre), g)
+    assert O.act_backward("silu", np.ones(1), np.zeros(1))[0] == 0.5                                            # derivative at 0
+
+
+def test_squeeze_excite_closed_forms_and_fd():
+    rng = np.random.default_rng(4)
+    n, h, w, c, k = 2, 3, 4, 5, 2
+    x = rng.normal(size=(n, h, w, c))
+    w1, b1, w2, b2 = rng.normal(size=(k, c)), rng.normal(size=k), rng.normal(size=(c, k)), rng.normal(size=c)
+    out, cache = O.se_forward(x, w1, b1, w2, b2)
+    # hand loop of the definition
+    for nn in range(n):
+        s = [sum(x[nn, i, j, cc] for i in range(h) for j in range(w)) / (h * w) for cc in range(c)]
+        hid = []
+        for q in range(k):
+            p = sum(w1[q, cc] * s[cc] for cc in range(c)) + b1[q]
+            hid.append(p / (1.0 + np.exp(-p)))
+        for cc in range(c):
+            p2 = sum(w2[cc, q] * hid[q] for q in range(k)) + b2[cc]
+            g = 1.0 / (1.0 + np.exp(-p2))
+            assert np.allclose(out[nn, :, :, cc], x[nn, :, :, cc] * g, rtol=0, atol=1e-14)
+    # zero second-layer weights: the gate is sigmoid(b2), the same for every sample
+    o0, _ = O.se_forward(x, w1, b1, np.zeros_like(w2), b2)
+    assert np.allclose(o0, x * (1.0 / (1.0 + np.exp(-b2))), rtol=0, atol=1e-14)
+    dout = rng.normal(size=out.shape)
+    dx, dw1, db1, dw2, db2 = O.se_backward(x, w1, w2, cache, dout)
+    L = lambda: float((O.se_forward(x, w1, b1, w2, b2)[0] * dout).sum())       # fd_grad perturbs its array in place
+    for got, arr in ((dx, x), (dw1, w1), (db1, b1), (dw2, w2), (db2, b2)):
+        assert_close_rel(got, fd_grad(L, arr))

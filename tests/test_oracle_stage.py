@@ -35,6 +35,12 @@ def torch_stage(net, first, last, params, x_nhwc, eps=1e-5):
             val[i] = F.relu6(a)
         elif ly.op == "relu":
             val[i] = F.relu(a)
+        elif ly.op == "silu":
+            val[i] = F.silu(a)
+        elif ly.op == "se":
+            sq = a.mean(dim=(2, 3))
+            hid = F.silu(F.linear(sq, per_layer[(i, "w1")], per_layer[(i, "b1")]))
+            val[i] = a * torch.sigmoid(F.linear(hid, per_layer[(i, "w2")], per_layer[(i, "b2")]))[:, :, None, None]
         elif ly.op == "add":
             val[i] = a + val[ly.add_from]
         elif ly.op == "gap":
@@ -53,6 +59,7 @@ CASES = {
     "mbv2_4blocks": (si.stage_net_mbv2_4blocks(), 8, 8, "mse"),
     "bottlenecks": (si.bottleneck_net(4, [(2, 8, 2, 1), (4, 16, 2, 2)]), 8, 8, "mse"),
     "small_mobilenet": (si.small_mobilenet(10)[0], 16, 16, "xent"),
+    "mbconv_k5_se": (si.mbconv_net(4, [(4, 1, 3, 5), (8, 2, 2, 3)]), 9, 9, "mse"),
 }
 
 
