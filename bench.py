@@ -4,13 +4,14 @@
 One step = one HPP-Round of the stage on one batch of synthetic input: M forwards (+ the loss head), M backwards,
 M gradient accumulations and one SGD-momentum update, all enqueued on one stream through the C ABI.
 
-    python bench.py [--config 1|2|3|4|all] [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--config 1|2|3|4|6|all] [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 Workloads (synthetic tensors of the shapes of the paper's compact vision models):
   1  one inverted-residual block 16->96->16 at 32x32, float32, micro-batch 8, M=4, MSE
   2  MobileNetV2-style stage of four inverted-residual blocks at 56x56x24, bfloat16, micro-batch 32, M=8, MSE
   3  full MobileNetV2 at 224x224x3, bfloat16, micro-batch 16, M=4, softmax cross-entropy
   4  ResNet-50 conv2_x + conv3_x bottleneck stage at 56x56x64, bfloat16, micro-batch 32, M=8, MSE
+  6  EfficientNet-B1-style stage of five MBConv6 blocks at 56x56x24, bfloat16, micro-batch 32, M=8, MSE (only on request)
 `--config all` (the default) prints one JSON line per workload; the LAST line is the headline: workload 4, the
 largest of the single-GPU workloads.  The timed region is repeated until it lasts about two seconds
 (`steps_timed` = steps x repeats; `ms_per_step` is the mean over all of them).
@@ -62,8 +63,13 @@ class Workload:
             self.net, self.H, self.W, self.B, self.M, self.bf16, self.loss = si.resnet50_c2c3_net(), 56, 56, 32, 8, True, "mse"
             self.name = "config 4: ResNet-50 conv2_x+conv3_x bottleneck stage at 56x56x64, micro-batch 32, M=8, bf16, MSE"
             self.cpu_sample, self.ref_sample = 8, 1
+        elif cfg == 6:
+            self.net, self.H, self.W, self.B, self.M, self.bf16, self.loss = si.efficientnet_b1_stage_net(), 56, 56, 32, 8, True, "mse"
+            self.name = ("EfficientNet-B1-style stage: 5 MBConv6 blocks (5x5 then 3x3 depthwise, squeeze-excite, SiLU) at 56x56x24, "
+                         "micro-batch 32, M=8, bf16, MSE")
+            self.cpu_sample, self.ref_sample = 16, 4
         else:
-            raise ValueError("config must be 1..4")
+            raise ValueError("config must be 1, 2, 3, 4 or 6")
         self.first, self.last = 0, len(self.net) - 1
         self.need_dx = 0 if cfg == 3 else 1          # the full network is the first stage of itself: no input gradient
         self.shp = si.out_shape(self.net, self.first, self.last, self.H, self.W)[self.last]
@@ -446,7 +452,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="all", choices=["1", "2", "3", "4", "all"])
+    ap.add_argument("--config", default="all", choices=["1", "2", "3", "4", "6", "all"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
                     help="the K timed steps are repeated until the timed region lasts about this long (0: exactly K steps)")

@@ -23,6 +23,7 @@
  *    dwconv  weight [c][k][k]
  *    bn      gamma [c], beta [c]
  *    linear  weight [c_out][c_in], bias [c_out]
+ *    se      w1 [k][c], b1 [k], w2 [c][k], b2 [c]      (k = squeeze width)
  */
 #ifndef ASTEROID_H
 #define ASTEROID_H
@@ -36,7 +37,7 @@ extern "C" {
 
 typedef struct asteroid_stage asteroid_stage;
 
-enum { AST_CONV = 0, AST_DWCONV = 1, AST_BN = 2, AST_RELU6 = 3, AST_RELU = 4, AST_ADD = 5, AST_GAP = 6, AST_LINEAR = 7 };
+enum { AST_CONV = 0, AST_DWCONV = 1, AST_BN = 2, AST_RELU6 = 3, AST_RELU = 4, AST_ADD = 5, AST_GAP = 6, AST_LINEAR = 7, AST_SILU = 8, AST_SE = 9 };
 enum { AST_F32 = 0, AST_BF16 = 1 };
 enum {
     AST_OK = 0,
@@ -53,8 +54,11 @@ enum {
  * reads, `add_from` (AST_ADD only) the index of the second operand; index -1 is the network
  * input.  Inside a stage [first,last] an index equal to first-1 denotes the stage input;
  * smaller indices are rejected.  Conv: cross-correlation, zero padding `pad`, no bias, weights
- * [c_out][k][k][c_in].  Dwconv: k=3, pad=1, c_in==c_out.  BN: training mode, statistics over
- * the micro-batch.  Add: out = value[src] + value[add_from]. */
+ * [c_out][k][k][c_in].  Dwconv: k = 3, 5 or 7, pad = (k-1)/2, c_in==c_out.  BN: training mode, statistics over
+ * the micro-batch.  Add: out = value[src] + value[add_from].  ReLU6 / ReLU directly after a conv (or its BN) are applied
+ * while the next layer loads; SiLU (x * sigmoid(x)) and SE are layers of their own whose output is stored.
+ * SE (squeeze-excite of the EfficientNet block, one of the paper's vision workloads, Section 5.1), c_in == c_out == c,
+ * `k` = squeeze width: s = mean over h,w; h = silu(w1 s + b1); g = sigmoid(w2 h + b2); out = x * g per sample and channel. */
 typedef struct {
     int32_t op, c_in, c_out, k, stride, pad, src, add_from;
 } ast_layer;

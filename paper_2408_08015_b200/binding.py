@@ -7,7 +7,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libasteroid.so")
 
 AST_F32, AST_BF16 = 0, 1
 AST_OK, AST_ERR_ARG, AST_ERR_UNSUPPORTED, AST_ERR_ORDER, AST_ERR_ALLOC, AST_ERR_CUDA, AST_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
-OP_CODES = {"conv": 0, "dwconv": 1, "bn": 2, "relu6": 3, "relu": 4, "add": 5, "gap": 6, "linear": 7}
+OP_CODES = {"conv": 0, "dwconv": 1, "bn": 2, "relu6": 3, "relu": 4, "add": 5, "gap": 6, "linear": 7, "silu": 8, "se": 9}
 
 EXPORTS = ["asteroid_stage_create", "asteroid_stage_destroy", "asteroid_stage_param_count",
            "asteroid_stage_output_elems", "asteroid_stage_import_state", "asteroid_stage_export_state",

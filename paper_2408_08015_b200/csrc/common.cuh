@@ -126,7 +126,7 @@ template <typename T> __device__ __forceinline__ void val_from_raw(const ValSrc&
         for (int i = 0; i < Vec<T>::N; ++i) out[i] = apply_act(out[i], s.act);
     }
 }
-__device__ __forceinline__ bool grad_needs_z(const GradSrc& s) { return s.act != ACT_NONE || s.k1 != nullptr; }
+__host__ __device__ __forceinline__ bool grad_needs_z(const GradSrc& s) { return s.act != ACT_NONE || s.k1 != nullptr; }
 template <typename T> __device__ __forceinline__ void grad_from_raw(const GradSrc& s, const Vec<T>& dy, const Vec<T>& zv, int c0, float* out) {
     dy.unpack(out);
     if (!grad_needs_z(s)) return;

@@ -18,7 +18,7 @@ struct ConvGeom {
 enum KernelKind {
     K_CONV_FWD = 0, K_CONV_BWD_DATA, K_CONV_BWD_WEIGHT, K_REDUCE_SPLITS, K_DW_FWD, K_DW_BWD_DATA, K_DW_BWD_WEIGHT,
     K_DW_BWD_WEIGHT_FINISH, K_BN_STATS, K_BN_STATS_FINISH, K_BN_BWD_REDUCE, K_BN_BWD_FINISH, K_EW_ADD, K_EW_MASK, K_EW_SUM,
-    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_CONV3_BWD_WEIGHT_TC, K_DW_BWD_FUSED, K_IM2COL, K_COL_AUX, K_KINDS
+    K_GAP_FWD, K_GAP_BWD, K_ACCUMULATE, K_SGD_STEP, K_REFRESH, K_LOSS_MSE, K_LOSS_XENT, K_PW_FWD_TC, K_PW_BWD_DATA_TC, K_PW_BWD_WEIGHT_TC, K_CONV3_FWD_TC, K_CONV3_BWD_DATA_TC, K_CONV3_BWD_WEIGHT_TC, K_DW_BWD_FUSED, K_IM2COL, K_COL_AUX, K_SILU, K_SE, K_KINDS
 };
 const char* kernel_name(int kind);
 
@@ -167,6 +167,22 @@ void ew_upsample2_grad(const GradSrc& d, int n, int hi, int wi, int ho, int wo, 
 void ew_subsample2(const void* full, int n, int hi, int wi, int ho, int wo, int c, void* z, cudaStream_t st);
 void gap_fwd(int dtype, const ValSrc& x, int n, int hw, int c, void* out, cudaStream_t st);
 void gap_bwd(int dtype, const void* da, int n, int hw, int c, const void* addend, void* dx, cudaStream_t st);
+
+// ---- EfficientNet MBConv pieces (mbconv.cu) ----
+// SiLU as a materialising unit: out = silu(value(x)); dx = dy * silu'(value(x)) (+ addend)
+void silu_fwd(int dtype, const ValSrc& x, size_t pixels, int c, void* out, void* out2, cudaStream_t st);
+void silu_bwd(int dtype, const void* dy, const ValSrc& x, const void* addend, size_t pixels, int c, void* dx, cudaStream_t st);
+// squeeze-excite over [n][hw][c] with k hidden units; s [n][c], p1 [n][k], gate [n][c] are float vectors kept for the backward pass;
+// work: >= n*(3c+k) floats
+void se_forward(int dtype, const ValSrc& x, int n, int hw, int c, int k, const float* w1, const float* b1, const float* w2, const float* b2,
+                float* s, float* p1, float* gate, void* out, void* out2, cudaStream_t st);
+void se_backward(int dtype, const void* dout, const ValSrc& x, int n, int hw, int c, int k, const float* w1, const float* w2, const float* s,
+                 const float* p1, const float* gate, float* work, const void* addend, void* dx, float* gw1, float* gb1, float* gw2, float* gb2,
+                 cudaStream_t st);
+// depthwise conv of odd kernel size k <= 7, pad (k-1)/2, stride 1 or 2; weights tap-major wkc[r*k+s][c]; gw[c][k][k]
+void dwk_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* wkc, void* z, cudaStream_t st);
+void dwk_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* wkc, const void* addend, void* dx, cudaStream_t st);
+void dwk_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, cudaStream_t st);
 
 // ---- parameters ----
 void accumulate(float* G, const float* g, size_t n, cudaStream_t st);

@@ -33,7 +33,7 @@ int report_error(int code, const char* msg) { return fail(code, "%s", msg); }
         if (e_ != cudaSuccess) return fail(AST_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_));   \
     } while (0)
 
-enum { U_CONV = 0, U_DW = 1, U_ADD = 2, U_GAP = 3 };
+enum { U_CONV = 0, U_DW = 1, U_ADD = 2, U_GAP = 3, U_SILU = 4, U_SE = 5 };
 enum { G_NONE = 0, G_ALIAS = 1, G_OWNED = 2 };
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -69,6 +69,10 @@ struct Unit {
     // stride-2 3x3 conv on the stride-1 tensor-core kernels: bytes into the arena of zero-inserted output gradients (one
     // buffer per such unit: the weight-gradient kernel reads it on the second stream while the pass goes on), -1 = none
     long up_off = -1;
+    // squeeze-excite: hidden width, floats into a slot's statistics area of the saved vectors (s [B][c], p1 [B][k], gate [B][c]),
+    // floats into the backward-coefficient arena of its work vectors (B*(3c+k))
+    int se_k = 0;
+    size_t se_off = 0, se_work_off = 0;
 };
 
 // Arenas of a stage carry a guard band of GUARD bytes of a fixed pattern on both sides.  With the environment variable
@@ -99,7 +103,11 @@ struct asteroid_stage {
     std::vector<Val> vals;          // vals[0] = stage input
     std::vector<Unit> units;
     std::vector<int> val_of_layer;  // layer index - (first-1) -> value id or -1
-    size_t n_params = 0, n_run = 0, n_coef = 0;
+    // n_params: values of the caller's flat state (layers back to back); n_pad: floats of the internal parameter arenas, where
+    // every layer starts on a multiple of 8 floats (16-byte aligned in the bfloat16 copies, whatever precedes it)
+    size_t n_params = 0, n_pad = 0, n_run = 0, n_coef = 0;
+    struct Seg { size_t pub, in, n; };
+    std::vector<Seg> segs;
     // device arenas
     float *w = nullptr, *v = nullptr, *G = nullptr, *g = nullptr, *derived = nullptr, *run = nullptr, *coef = nullptr, *scratch = nullptr;
     int32_t* perm = nullptr;
@@ -153,6 +161,7 @@ static int n_layer_params(const ast_layer& L) {
         case AST_DWCONV: return L.c_out * L.k * L.k;
         case AST_BN: return 2 * L.c_out;
         case AST_LINEAR: return L.c_out * L.c_in + L.c_out;
+        case AST_SE: return 2 * L.k * L.c_out + L.k + L.c_out;
         default: return 0;
     }
 }
@@ -165,12 +174,16 @@ static int build_plan(asteroid_stage* s) {
     const int first = s->first, last = s->last;
     const int vecw = s->dtype == AST_F32 ? 4 : 8;
     std::vector<long> poff(net.size(), -1);
-    long off = 0;
+    long off = 0, pub = 0;
     for (int i = first; i <= last; ++i) {
+        const long n = n_layer_params(net[i]);
         poff[i] = off;
-        off += n_layer_params(net[i]);
+        if (n) s->segs.push_back({(size_t)pub, (size_t)off, (size_t)n});
+        pub += n;
+        off = (off + n + 7) / 8 * 8;
     }
-    s->n_params = (size_t)off;
+    s->n_params = (size_t)pub;
+    s->n_pad = (size_t)off;
     s->val_of_layer.assign(last - first + 2, -1);
     auto vol = [&](int layer) -> int& { return s->val_of_layer[layer - (first - 1)]; };
 
@@ -210,8 +223,8 @@ static int build_plan(asteroid_stage* s) {
                 if (g.k < 1 || g.stride < 1 || g.pad < 0) return fail(AST_ERR_ARG, "layer %d: bad k/stride/pad", i);
             }
             if (L.op == AST_DWCONV) {
-                if (L.k != 3 || L.pad != 1 || L.c_in != L.c_out || (L.stride != 1 && L.stride != 2))
-                    return fail(AST_ERR_UNSUPPORTED, "layer %d: depthwise conv must be 3x3, pad 1, stride 1 or 2", i);
+                if ((L.k != 3 && L.k != 5 && L.k != 7) || L.pad != (L.k - 1) / 2 || L.c_in != L.c_out || (L.stride != 1 && L.stride != 2))
+                    return fail(AST_ERR_UNSUPPORTED, "layer %d: depthwise conv must be 3x3, 5x5 or 7x7 with pad (k-1)/2 and stride 1 or 2", i);
                 if (L.c_in % vecw) return fail(AST_ERR_UNSUPPORTED, "layer %d: depthwise channels must be a multiple of %d", i, vecw);
             }
             g.ho = (g.hi + 2 * g.pad - g.k) / g.stride + 1;
@@ -262,6 +275,29 @@ static int build_plan(asteroid_stage* s) {
             s->vals.push_back(o);
             vol(j - 1) = u.out;
             i = j;
+        } else if (L.op == AST_SILU || L.op == AST_SE) {
+            // materialising units: the value they read keeps its on-load BatchNorm; their own output is a plain stored tensor
+            if ((rc = resolve(L.src, i, &u.in))) return rc;
+            const Val& a = s->vals[u.in];
+            if (a.c != L.c_in || L.c_in != L.c_out) return fail(AST_ERR_ARG, "layer %d: channel count %d does not match its input's %d", i, L.c_in, a.c);
+            if (L.op == AST_SE) {
+                if (L.k < 1 || L.k > 1024) return fail(AST_ERR_ARG, "layer %d: squeeze width must be in [1,1024]", i);
+                if (a.c > 8192) return fail(AST_ERR_UNSUPPORTED, "layer %d: squeeze-excite takes at most 8192 channels", i);
+                u.kind = U_SE;
+                u.se_k = L.k;
+                u.w_off = poff[i];
+                u.g.n = s->B; u.g.hi = u.g.ho = a.h; u.g.wi = u.g.wo = a.w; u.g.ci = u.g.co = a.c;
+            } else {
+                u.kind = U_SILU;
+            }
+            Val o;
+            o.h = a.h; o.w = a.w; o.c = a.c;
+            o.unit = (int)s->units.size();
+            o.elems = a.elems;
+            u.out = (int)s->vals.size();
+            s->vals.push_back(o);
+            vol(i) = u.out;
+            i = i + 1;
         } else if (L.op == AST_GAP) {
             if ((rc = resolve(L.src, i, &u.in))) return rc;
             const Val& a = s->vals[u.in];
@@ -320,6 +356,13 @@ static int build_plan(asteroid_stage* s) {
             nrun += 2 * (size_t)o.c;
         }
     }
+    for (auto& u : s->units)
+        if (u.kind == U_SE) {
+            u.se_off = nstat;
+            nstat += (size_t)s->B * (2 * (size_t)u.g.ci + u.se_k);
+            u.se_work_off = ncoef;
+            ncoef += (size_t)s->B * (3 * (size_t)u.g.ci + u.se_k);
+        }
     s->slot_bytes = align_up(sb + nstat * sizeof(float), 256);
     s->grad_bytes = gb;
     s->n_coef = ncoef;
@@ -328,7 +371,7 @@ static int build_plan(asteroid_stage* s) {
 }
 
 static void fill_perm(const asteroid_stage* s, std::vector<int32_t>& perm) {
-    perm.resize(s->n_params);
+    perm.resize(s->n_pad);
     for (size_t i = 0; i < perm.size(); ++i) perm[i] = (int32_t)i;
     for (const auto& u : s->units) {
         if (u.kind == U_CONV) {          // derived: wt[c][r][s][ko] <- w[ko][r][s][c]
@@ -337,9 +380,10 @@ static void fill_perm(const asteroid_stage* s, std::vector<int32_t>& perm) {
                 for (int rs = 0; rs < g.k * g.k; ++rs)
                     for (int c = 0; c < g.ci; ++c)
                         perm[u.w_off + ((size_t)c * g.k * g.k + rs) * g.co + ko] = (int32_t)(u.w_off + ((size_t)ko * g.k * g.k + rs) * g.ci + c);
-        } else if (u.kind == U_DW) {     // derived: w9c[t][c] <- w[c][t]
+        } else if (u.kind == U_DW) {     // derived: tap-major wkc[t][c] <- w[c][t]
+            const int taps = u.g.k * u.g.k;
             for (int c = 0; c < u.g.ci; ++c)
-                for (int t = 0; t < 9; ++t) perm[u.w_off + (size_t)t * u.g.ci + c] = (int32_t)(u.w_off + (size_t)c * 9 + t);
+                for (int t = 0; t < taps; ++t) perm[u.w_off + (size_t)t * u.g.ci + c] = (int32_t)(u.w_off + (size_t)c * taps + t);
         }
     }
 }
@@ -414,7 +458,7 @@ static int reset_bn_running(asteroid_stage* s) {
 
 // derived weight copies of every kind, after the master weights changed
 static void refresh_weights(asteroid_stage* s, cudaStream_t st) {
-    refresh_derived(s->w, s->perm, s->derived, s->wb, s->wtb, s->n_params, st);
+    refresh_derived(s->w, s->perm, s->derived, s->wb, s->wtb, s->n_pad, st);
     for (const auto& u : s->units)
         if (u.col_kp) conv_pad_weights(s->w + u.w_off, u.g.co, u.g.k * u.g.k * u.g.ci, u.col_kp, s->wpad + u.wpad_off, st);
 }
@@ -505,8 +549,18 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
             else conv_fwd(dt, u.g, val_src(s, sv, u.in), s->w + u.w_off, bias, obuf, st);
         } else if (u.kind == U_DW) {
             const bool bn = u.l_bn >= 0;
-            fused_stats = dw_fwd(dt, u.g, val_src(s, sv, u.in), s->derived + u.w_off, obuf, bn ? s->run + u.run_off : nullptr, bn ? s->scratch : nullptr,
-                                 s->scratch_floats, st);
+            if (u.g.k != 3) dwk_fwd(dt, u.g, val_src(s, sv, u.in), s->derived + u.w_off, obuf, st);
+            else
+                fused_stats = dw_fwd(dt, u.g, val_src(s, sv, u.in), s->derived + u.w_off, obuf, bn ? s->run + u.run_off : nullptr, bn ? s->scratch : nullptr,
+                                     s->scratch_floats, st);
+        } else if (u.kind == U_SILU) {
+            silu_fwd(dt, val_src(s, sv, u.in), o.elems / o.c, o.c, obuf, is_last ? y : nullptr, st);
+        } else if (u.kind == U_SE) {
+            const int c = o.c, k = u.se_k;
+            const float* wp = s->w + u.w_off;        // w1 [k][c], b1 [k], w2 [c][k], b2 [c]
+            float* sev = sv.stats + u.se_off;        // s [B][c], p1 [B][k], gate [B][c]
+            se_forward(dt, val_src(s, sv, u.in), s->B, o.h * o.w, c, k, wp, wp + (size_t)k * c, wp + (size_t)k * c + k, wp + 2 * (size_t)k * c + k, sev,
+                       sev + (size_t)s->B * c, sev + (size_t)s->B * (c + k), obuf, is_last ? y : nullptr, st);
         } else if (u.kind == U_ADD) {
             ew_add(dt, val_src(s, sv, u.in), val_src(s, sv, u.in2), u.act, o.elems / o.c, o.c, obuf, is_last ? y : nullptr, st);
         } else {
@@ -624,7 +678,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             }
             tick(s, ui, 4, st);
             ValSrc xin = val_src(s, sv, u.in);
-            if (u.kind == U_DW && want_in) {
+            if (u.kind == U_DW && want_in && u.g.k == 3) {
                 GradState& gi = gs[u.in];
                 const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
                 if (dw_bwd_fused(dt, u.g, d, xin, s->derived + u.w_off, addend, own(u.in), s->scratch, s->scratch_floats, s->g + u.w_off, st)) {
@@ -654,6 +708,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             else if (u.kind == U_CONV && conv3_wgrad_tc_supported(dt, u.g))
                 conv3_bwd_weight_tc(u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst);
             else if (u.kind == U_CONV) conv_bwd_weight(dt, u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, wst);
+            else if (u.g.k != 3) dwk_bwd_weight(dt, u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, wst);
             else dw_bwd_weight(dt, u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, wst);
             if (want_in) {
                 GradState& gi = gs[u.in];
@@ -683,6 +738,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                 } else if (u.kind == U_CONV && conv3_tc_supported(dt, u.g)) conv3_bwd_data_tc(u.g, d, s->wtb + u.w_off, addend, own(u.in), s->err, st);
                 else if (s2_tc) conv3_bwd_data_tc(s1_geom(u), dup, s->wtb + u.w_off, addend, own(u.in), s->err, st, conv_flops(u.g));
                 else if (u.kind == U_CONV) conv_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
+                else if (u.g.k != 3) dwk_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 else dw_bwd_data(dt, u.g, d, s->derived + u.w_off, addend, own(u.in), st);
                 gi.state = G_OWNED;
                 gi.ptr = own(u.in);
@@ -696,6 +752,26 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             }
             if (u.in != 0 || s->need_dx) pass(u.in, go.ptr);
             if (u.in2 != 0 || s->need_dx) pass(u.in2, go.ptr);
+        } else if (u.kind == U_SILU || u.kind == U_SE) {
+            tick(s, ui, 4, st);
+            GradState& gi = gs[u.in];
+            const void* addend = gi.state == G_NONE ? nullptr : gi.ptr;
+            if (u.kind == U_SE) {
+                // the parameter gradients are wanted even when the input gradient is not; the kernel sequence computes both
+                const int c = o.c, k = u.se_k;
+                const float* wp = s->w + u.w_off;
+                float* gp = s->g + u.w_off;
+                const float* sev = sv.stats + u.se_off;
+                se_backward(dt, go.ptr, val_src(s, sv, u.in), s->B, o.h * o.w, c, k, wp, wp + (size_t)k * c + k, sev, sev + (size_t)s->B * c,
+                            sev + (size_t)s->B * (c + k), s->coef + u.se_work_off, addend, want_in ? own(u.in) : nullptr, gp, gp + (size_t)k * c, gp + (size_t)k * c + k,
+                            gp + 2 * (size_t)k * c + k, st);
+            } else if (want_in) {
+                silu_bwd(dt, go.ptr, val_src(s, sv, u.in), addend, o.elems / o.c, o.c, own(u.in), st);
+            }
+            if (want_in) {
+                gi.state = G_OWNED;
+                gi.ptr = own(u.in);
+            }
         } else {  // U_GAP
             tick(s, ui, 4, st);
             if (want_in) {
@@ -738,7 +814,7 @@ static int create_impl(const ast_layer* net, int n_layers, int first, int last, 
     int rc = build_plan(s);
     if (rc) return rc;
 
-    const size_t np = s->n_params;
+    const size_t np = s->n_pad;
     size_t mod = 0, opt = 0, act = 0, work = 0;
     if ((rc = arena_alloc(s, "parameters", &s->w, np * 4, &mod))) return rc;
     if ((rc = arena_alloc(s, "accumulated gradients", &s->G, np * 4, &mod))) return rc;
@@ -833,10 +909,14 @@ int asteroid_stage_import_state(asteroid_stage* s, const float* params, const fl
     if (n != s->n_params) return fail(AST_ERR_ARG, "state has %zu values, the stage has %zu parameters", n, s->n_params);
     CU(cudaDeviceSynchronize());
     if (n) {
-        CU(cudaMemcpy(s->w, params, n * 4, cudaMemcpyHostToDevice));
-        if (momentum) CU(cudaMemcpy(s->v, momentum, n * 4, cudaMemcpyHostToDevice));
-        else CU(cudaMemset(s->v, 0, n * 4));
-        CU(cudaMemset(s->G, 0, n * 4));
+        std::vector<float> h(s->n_pad, 0.f);
+        for (const auto& g : s->segs) memcpy(h.data() + g.in, params + g.pub, g.n * 4);
+        CU(cudaMemcpy(s->w, h.data(), s->n_pad * 4, cudaMemcpyHostToDevice));
+        if (momentum) {
+            for (const auto& g : s->segs) memcpy(h.data() + g.in, momentum + g.pub, g.n * 4);
+            CU(cudaMemcpy(s->v, h.data(), s->n_pad * 4, cudaMemcpyHostToDevice));
+        } else CU(cudaMemset(s->v, 0, s->n_pad * 4));
+        CU(cudaMemset(s->G, 0, s->n_pad * 4));
         refresh_weights(s, 0);
     }
     int rc = reset_bn_running(s);
@@ -862,10 +942,13 @@ int asteroid_stage_export_state(asteroid_stage* s, float* params, float* momentu
         if (grc) return grc;
     }
     if (n) {
-        if (params) CU(cudaMemcpy(params, s->w, n * 4, cudaMemcpyDeviceToHost));
-        if (momentum) CU(cudaMemcpy(momentum, s->v, n * 4, cudaMemcpyDeviceToHost));
-        if (grad_accum) CU(cudaMemcpy(grad_accum, s->G, n * 4, cudaMemcpyDeviceToHost));
-        if (micro_grad) CU(cudaMemcpy(micro_grad, s->g, n * 4, cudaMemcpyDeviceToHost));
+        std::vector<float> h(s->n_pad);
+        const std::pair<float*, const float*> outs[4] = {{params, s->w}, {momentum, s->v}, {grad_accum, s->G}, {micro_grad, s->g}};
+        for (const auto& o : outs) {
+            if (!o.first) continue;
+            CU(cudaMemcpy(h.data(), o.second, s->n_pad * 4, cudaMemcpyDeviceToHost));
+            for (const auto& g : s->segs) memcpy(o.first + g.pub, h.data() + g.in, g.n * 4);
+        }
     }
     return AST_OK;
 }
@@ -923,7 +1006,7 @@ int asteroid_stage_accumulate(asteroid_stage* s, int mb, void* stream) {
     if (!s) return fail(AST_ERR_ARG, "null argument");
     if (s->pending_g != mb) return fail(AST_ERR_ORDER, "accumulate(%d): the last backward was of micro-batch %d", mb, s->pending_g);
     if (s->n_acc >= s->M) return fail(AST_ERR_ORDER, "already accumulated %d micro-batches this round", s->M);
-    accumulate(s->G, s->g, s->n_params, (cudaStream_t)stream);
+    accumulate(s->G, s->g, s->n_pad, (cudaStream_t)stream);
     CU(cudaGetLastError());
     s->pending_g = -1;
     s->n_acc++;
@@ -934,7 +1017,7 @@ int asteroid_stage_step(asteroid_stage* s, float lr, float momentum, void* strea
     if (!s) return fail(AST_ERR_ARG, "null argument");
     if (s->n_acc != s->M) return fail(AST_ERR_ORDER, "step after %d of %d micro-batches accumulated", s->n_acc, s->M);
     cudaStream_t st = (cudaStream_t)stream;
-    sgd_step(s->w, s->v, s->G, s->n_params, 1.f / (float)s->M, lr, momentum, st);
+    sgd_step(s->w, s->v, s->G, s->n_pad, 1.f / (float)s->M, lr, momentum, st);
     refresh_weights(s, st);
     CU(cudaGetLastError());
     s->n_acc = 0;
@@ -988,12 +1071,12 @@ int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_pr
         const size_t nu = t->units.size();
         t->tm.ev.resize(nu * 6);
         for (auto& e : t->tm.ev) CU(cudaEventCreate(&e));
-        if (s->n_params) {
-            CU(cudaMemcpy(t->w, s->w, s->n_params * 4, cudaMemcpyDeviceToDevice));
-            CU(cudaMemcpy(t->derived, s->derived, s->n_params * 4, cudaMemcpyDeviceToDevice));
+        if (s->n_pad) {
+            CU(cudaMemcpy(t->w, s->w, s->n_pad * 4, cudaMemcpyDeviceToDevice));
+            CU(cudaMemcpy(t->derived, s->derived, s->n_pad * 4, cudaMemcpyDeviceToDevice));
             if (s->wb) {
-                CU(cudaMemcpy(t->wb, s->wb, s->n_params * 2, cudaMemcpyDeviceToDevice));
-                CU(cudaMemcpy(t->wtb, s->wtb, s->n_params * 2, cudaMemcpyDeviceToDevice));
+                CU(cudaMemcpy(t->wb, s->wb, s->n_pad * 2, cudaMemcpyDeviceToDevice));
+                CU(cudaMemcpy(t->wtb, s->wtb, s->n_pad * 2, cudaMemcpyDeviceToDevice));
             }
             if (s->wpad && t->wpad && s->n_wpad == t->n_wpad) CU(cudaMemcpy(t->wpad, s->wpad, s->n_wpad * 2, cudaMemcpyDeviceToDevice));
         }
@@ -1056,7 +1139,7 @@ int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_pr
             out->t_f_ms = ms[ui * 4 + 0];
             out->t_b_ms = ms[ui * 4 + 3];
             if (u.kind == U_CONV || u.kind == U_DW) {
-                uint64_t macs = (uint64_t)vout.elems * (u.kind == U_DW ? 9 : (uint64_t)u.g.k * u.g.k * u.g.ci);
+                uint64_t macs = (uint64_t)vout.elems * (u.kind == U_DW ? (uint64_t)u.g.k * u.g.k : (uint64_t)u.g.k * u.g.k * u.g.ci);
                 out->flops = 2 * macs;
                 out->alg_bytes_f = xin + zo + out->w_l_bytes;
                 // bwd-weight reads dy, z, x; bwd-data reads dy, z and writes dx
@@ -1064,6 +1147,12 @@ int asteroid_stage_profile(asteroid_stage* s, int layer, int batch, ast_layer_pr
             } else if (u.kind == U_ADD) {
                 out->alg_bytes_f = 3 * zo;
                 out->alg_bytes_b = u.act == ACT_RELU ? 3 * zo : 0;
+            } else if (u.kind == U_SILU) {
+                out->alg_bytes_f = xin + zo;
+                out->alg_bytes_b = 3 * zo;              // dy, x -> dx
+            } else if (u.kind == U_SE) {
+                out->alg_bytes_f = 2 * xin + zo;        // x for the squeeze, x again for the scaling
+                out->alg_bytes_b = 5 * zo;              // x and dout for the gate gradient, both again for dx
             } else {
                 out->alg_bytes_f = xin + zo;
                 out->alg_bytes_b = xin + zo;

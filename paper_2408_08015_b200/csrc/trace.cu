@@ -36,7 +36,7 @@ cudaEvent_t take_event() {
 const char* const kNames[K_KINDS] = {
     "conv_fwd_simt", "conv_bwd_data_simt", "conv_bwd_weight_simt", "reduce_splits", "dw_fwd", "dw_bwd_data", "dw_bwd_weight",
     "dw_bwd_weight_finish", "bn_stats", "bn_stats_finish", "bn_bwd_reduce", "bn_bwd_finish", "ew_add", "ew_relu_mask", "ew_sum",
-    "gap_fwd", "gap_bwd", "accumulate", "sgd_step", "refresh_derived", "loss_mse", "loss_softmax_xent", "pw_fwd_tcgen05", "pw_bwd_data_tcgen05", "pw_bwd_weight_tcgen05", "conv3x3_fwd_tcgen05", "conv3x3_bwd_data_tcgen05", "conv3x3_bwd_weight_tcgen05", "dw_bwd_fused", "conv_im2col", "conv_pad_unpad"};
+    "gap_fwd", "gap_bwd", "accumulate", "sgd_step", "refresh_derived", "loss_mse", "loss_softmax_xent", "pw_fwd_tcgen05", "pw_bwd_data_tcgen05", "pw_bwd_weight_tcgen05", "conv3x3_fwd_tcgen05", "conv3x3_bwd_data_tcgen05", "conv3x3_bwd_weight_tcgen05", "dw_bwd_fused", "conv_im2col", "conv_pad_unpad", "silu", "squeeze_excite"};
 }  // namespace
 
 int sm_count() {

@@ -100,8 +100,12 @@ def test_unsupported_patterns_are_refused():
     L = si.Layer
     bn_first = [L("bn", 8, 8, 0, 1, 0, -1, -1), L("conv", 8, 8, 1, 1, 0, 0, -1)]
     assert _code(P.asteroid_stage_create, bn_first, 0, 1, 4, 4, 2, 1) == P.AST_ERR_UNSUPPORTED          # BN with no conv to belong to
-    dw5 = [L("dwconv", 8, 8, 5, 1, 2, -1, -1)]
-    assert _code(P.asteroid_stage_create, dw5, 0, 0, 8, 8, 2, 1) == P.AST_ERR_UNSUPPORTED                # depthwise is 3x3 only
+    dw9 = [L("dwconv", 8, 8, 9, 1, 4, -1, -1)]
+    assert _code(P.asteroid_stage_create, dw9, 0, 0, 8, 8, 2, 1) == P.AST_ERR_UNSUPPORTED                # depthwise is 3x3, 5x5 or 7x7
+    dw5_pad = [L("dwconv", 8, 8, 5, 1, 1, -1, -1)]
+    assert _code(P.asteroid_stage_create, dw5_pad, 0, 0, 8, 8, 2, 1) == P.AST_ERR_UNSUPPORTED            # ... with "same" padding
+    se_wide = [L("conv", 8, 8, 1, 1, 0, -1, -1), L("se", 8, 8, 2000, 1, 0, 0, -1)]
+    assert _code(P.asteroid_stage_create, se_wide, 0, 1, 4, 4, 2, 1) == P.AST_ERR_ARG                    # squeeze width out of range
     dw_odd = [L("dwconv", 12, 12, 3, 1, 1, -1, -1)]
     assert _code(P.asteroid_stage_create, dw_odd, 0, 0, 8, 8, 2, 1, dtype=P.AST_BF16) == P.AST_ERR_UNSUPPORTED   # 12 % 8 != 0 in bfloat16
     # a layer that reads the un-normalised conv output from inside a conv-BN-activation chain

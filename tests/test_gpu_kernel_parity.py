@@ -56,6 +56,18 @@ CASES = {
     "dw_144_s2": (si.single_unit_net("dwconv", 144, 144, stride=2), 56, 56, 3, 2, "mse", DW),
     "dw_96_s2_bn_odd": (si.single_unit_net("dwconv", 96, 96, stride=2, bn=True), 31, 29, 3, 1, "mse", DW),
     "dw_960_7": (si.single_unit_net("dwconv", 960, 960, bn=True), 7, 7, 4, 1, "mse", DW),
+    # depthwise 5x5 / 7x7 (EfficientNet), stride 1 and 2, even and odd maps
+    "dw5_144_s1": (si.single_unit_net("dwconv", 144, 144, k=5), 29, 27, 3, 2, "mse", DW),
+    "dw5_240_s2_bn_odd": (si.single_unit_net("dwconv", 240, 240, k=5, stride=2, bn=True), 31, 29, 3, 1, "mse", DW),
+    "dw5_144_s2_even": (si.single_unit_net("dwconv", 144, 144, k=5, stride=2), 56, 56, 2, 1, "mse", DW),
+    "dw7_48_s1_bn": (si.single_unit_net("dwconv", 48, 48, k=7, bn=True), 17, 19, 2, 2, "mse", DW),
+    # SiLU and squeeze-excite are smooth: held to the contract like the activation-free paths
+    "pw_24_144_bn_silu": (si.single_unit_net("conv", 24, 144, bn=True, act="silu"), 29, 27, 3, 2, "mse", PW + ("silu",)),
+    "pw_3_6_silu_narrow": (si.single_unit_net("conv", 3, 6, act="silu"), 9, 7, 3, 1, "mse", ("silu",)),
+    "pw_24_144_bn_se": (si.single_unit_net("conv", 24, 144, bn=True, se=6), 29, 27, 3, 2, "mse", PW + ("squeeze_excite",)),
+    "pw_16_240_se10_odd": (si.single_unit_net("conv", 16, 240, se=10), 7, 5, 5, 1, "mse", PW + ("squeeze_excite",)),
+    "pw_3_6_se_narrow": (si.single_unit_net("conv", 3, 6, se=2), 9, 7, 3, 1, "mse", ("squeeze_excite",)),
+    "dw5_144_bn_silu_se": (si.single_unit_net("dwconv", 144, 144, k=5, bn=True, act="silu", se=6), 28, 28, 3, 1, "mse", DW + ("silu", "squeeze_excite")),
     # classifier head: pool, linear, softmax cross-entropy (with and without a conv + BatchNorm in front)
     "head_1280_1000": (si.head_net(1280, 1000), 7, 7, 16, 2, "xent", ("gap_fwd", "loss_softmax_xent") + PW),
     "head_320_1280_bn_1000": (si.head_net(320, 1000, bn_conv=1280), 7, 7, 16, 1, "xent", ("gap_fwd", "loss_softmax_xent") + PW),

@@ -26,6 +26,11 @@ SMALL = {
     "bottleneck_c128": (si.bottleneck_net(128, [(128, 128, 2, 1)]), 7, 12, 2, 1, "mse"),
     # stride-2 3x3 conv with tensor-core channel counts on an odd-sized map (zero-inserted gradient, subsampled forward)
     "bottleneck_c64_s2_odd": (si.bottleneck_net(64, [(64, 128, 1, 2)]), 9, 7, 2, 2, "mse"),
+    # EfficientNet MBConv: expand, 5x5 depthwise, SiLU, squeeze-excite, project, residual
+    "mbconv_k5_residual": (si.mbconv_net(24, [(24, 1, 6, 5)]), 13, 11, 3, 2, "mse"),
+    "mbconv_k3_s2": (si.mbconv_net(16, [(24, 2, 6, 3)]), 14, 12, 2, 2, "mse"),
+    "mbconv_t1_then_k5": (si.mbconv_net(16, [(16, 1, 1, 3), (24, 2, 6, 5)]), 12, 12, 2, 1, "mse"),
+    "efficientnet_stage_small": (si.efficientnet_b1_stage_net(), 28, 28, 4, 2, "mse"),
 }
 
 
@@ -52,6 +57,7 @@ SHALLOW = ((CONTRACT, MIRROR), ("y", "loss"))
 BF16_RULES = {
     "block_ragged": SHALLOW, "block_c16": SHALLOW, "bnfree_block": SHALLOW, "bottleneck_c64": SHALLOW, "bottleneck_c64_s2_odd": SHALLOW,
     "bottlenecks_small": ((CONTRACT, MIRROR), ("loss",)),
+    "mbconv_k5_residual": SHALLOW, "mbconv_k3_s2": SHALLOW, "mbconv_t1_then_k5": (ALL, ("y", "loss")), "efficientnet_stage_small": (ALL, ("y", "loss")),
     "bottleneck_c128": (ALL, ("y", "loss")), "mbv2_4blocks_small": (ALL, ("y", "loss")), "small_mobilenet_xent": (ALL, ("y", "loss")),
 }
 
@@ -110,6 +116,14 @@ def test_config4_resnet_stage_bf16():
     net = si.resnet50_c2c3_net()
     print(summary(sampled_round_check(net, 0, len(net) - 1, 56, 56, 8, 8, "mse", True, [5], 2e-2, allow=ALL, outlier_frac=5e-4,
                                       case="config4/bf16/B8", contract_kinds=("loss",))))
+
+
+def test_efficientnet_stage_bf16_full_size():
+    """Five MBConv6 blocks (5x5 then 3x3 depthwise, squeeze-excite, SiLU) at 56x56x24, M=4 micro-batches of 16, bfloat16;
+    the oracle evaluates micro-batches 0 and 3."""
+    net = si.efficientnet_b1_stage_net()
+    print(summary(sampled_round_check(net, 0, len(net) - 1, 56, 56, 16, 4, "mse", True, [0, 3], 2e-2, allow=ALL, outlier_frac=5e-4,
+                                      case="efficientnet_stage/bf16")))
 
 
 def test_one_forward_one_backward_order_is_bit_identical():
