@@ -173,12 +173,12 @@ void gap_bwd(int dtype, const void* da, int n, int hw, int c, const void* addend
 void silu_fwd(int dtype, const ValSrc& x, size_t pixels, int c, void* out, void* out2, cudaStream_t st);
 void silu_bwd(int dtype, const void* dy, const ValSrc& x, const void* addend, size_t pixels, int c, void* dx, cudaStream_t st);
 // squeeze-excite over [n][hw][c] with k hidden units; s [n][c], p1 [n][k], gate [n][c] are float vectors kept for the backward pass;
-// work: >= n*(3c+k) floats
+// work: >= n*(2c+k) floats; scratch: partials of the pixel-split reductions (any size >= n*c floats; more allows more splits)
 void se_forward(int dtype, const ValSrc& x, int n, int hw, int c, int k, const float* w1, const float* b1, const float* w2, const float* b2,
-                float* s, float* p1, float* gate, void* out, void* out2, cudaStream_t st);
+                float* s, float* p1, float* gate, float* scratch, size_t scratch_floats, void* out, void* out2, cudaStream_t st);
 void se_backward(int dtype, const void* dout, const ValSrc& x, int n, int hw, int c, int k, const float* w1, const float* w2, const float* s,
-                 const float* p1, const float* gate, float* work, const void* addend, void* dx, float* gw1, float* gb1, float* gw2, float* gb2,
-                 cudaStream_t st);
+                 const float* p1, const float* gate, float* work, float* scratch, size_t scratch_floats, const void* addend, void* dx, float* gw1, float* gb1,
+                 float* gw2, float* gb2, cudaStream_t st);
 // depthwise conv of odd kernel size k <= 7, pad (k-1)/2, stride 1 or 2; weights tap-major wkc[r*k+s][c]; gw[c][k][k]
 void dwk_fwd(int dtype, const ConvGeom& g, const ValSrc& x, const float* wkc, void* z, cudaStream_t st);
 void dwk_bwd_data(int dtype, const ConvGeom& g, const GradSrc& dz, const float* wkc, const void* addend, void* dx, cudaStream_t st);

@@ -560,7 +560,7 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
             const float* wp = s->w + u.w_off;        // w1 [k][c], b1 [k], w2 [c][k], b2 [c]
             float* sev = sv.stats + u.se_off;        // s [B][c], p1 [B][k], gate [B][c]
             se_forward(dt, val_src(s, sv, u.in), s->B, o.h * o.w, c, k, wp, wp + (size_t)k * c, wp + (size_t)k * c + k, wp + 2 * (size_t)k * c + k, sev,
-                       sev + (size_t)s->B * c, sev + (size_t)s->B * (c + k), obuf, is_last ? y : nullptr, st);
+                       sev + (size_t)s->B * c, sev + (size_t)s->B * (c + k), s->scratch, s->scratch_floats, obuf, is_last ? y : nullptr, st);
         } else if (u.kind == U_ADD) {
             ew_add(dt, val_src(s, sv, u.in), val_src(s, sv, u.in2), u.act, o.elems / o.c, o.c, obuf, is_last ? y : nullptr, st);
         } else {
@@ -763,7 +763,7 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
                 float* gp = s->g + u.w_off;
                 const float* sev = sv.stats + u.se_off;
                 se_backward(dt, go.ptr, val_src(s, sv, u.in), s->B, o.h * o.w, c, k, wp, wp + (size_t)k * c + k, sev, sev + (size_t)s->B * c,
-                            sev + (size_t)s->B * (c + k), s->coef + u.se_work_off, addend, want_in ? own(u.in) : nullptr, gp, gp + (size_t)k * c, gp + (size_t)k * c + k,
+                            sev + (size_t)s->B * (c + k), s->coef + u.se_work_off, s->scratch, s->scratch_floats, addend, want_in ? own(u.in) : nullptr, gp, gp + (size_t)k * c, gp + (size_t)k * c + k,
                             gp + 2 * (size_t)k * c + k, st);
             } else if (want_in) {
                 silu_bwd(dt, go.ptr, val_src(s, sv, u.in), addend, o.elems / o.c, o.c, own(u.in), st);

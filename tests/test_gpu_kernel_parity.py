@@ -61,6 +61,9 @@ CASES = {
     "dw5_240_s2_bn_odd": (si.single_unit_net("dwconv", 240, 240, k=5, stride=2, bn=True), 31, 29, 3, 1, "mse", DW),
     "dw5_144_s2_even": (si.single_unit_net("dwconv", 144, 144, k=5, stride=2), 56, 56, 2, 1, "mse", DW),
     "dw7_48_s1_bn": (si.single_unit_net("dwconv", 48, 48, k=7, bn=True), 17, 19, 2, 2, "mse", DW),
+    "dw7_48_s2_odd": (si.single_unit_net("dwconv", 48, 48, k=7, stride=2), 15, 13, 2, 1, "mse", DW),
+    "dw5_16_map_smaller_than_the_kernel": (si.single_unit_net("dwconv", 16, 16, k=5, bn=True), 3, 2, 4, 2, "mse", DW),
+    "dw5_16_s2_map_smaller_than_the_kernel": (si.single_unit_net("dwconv", 16, 16, k=5, stride=2), 2, 3, 4, 1, "mse", DW),
     # SiLU and squeeze-excite are smooth: held to the contract like the activation-free paths
     "pw_24_144_bn_silu": (si.single_unit_net("conv", 24, 144, bn=True, act="silu"), 29, 27, 3, 2, "mse", PW + ("silu",)),
     "pw_3_6_silu_narrow": (si.single_unit_net("conv", 3, 6, act="silu"), 9, 7, 3, 1, "mse", ("silu",)),
