@@ -13,7 +13,8 @@ package.  It shares no code with the CUDA library and never calls it.
 
 Pins (tests/test_oracle_*.py): brute-force direct convolution, central finite
 differences, adjoint identities, BatchNorm closed forms and invariants, loss
-special cases, closed-form SGD steps, the micro-batch accumulation invariant,
+special cases, closed-form SGD steps, the micro-batch accumulation invariant (also across the
+devices of a data-parallel group),
 agreement with torch.autograd in float64 on whole stages, and the K_p values the
 paper prints for a three-stage pipeline; the storage-mirroring mode by tests/test_oracle_mirror.py;
 the planner (oracle/planner.py) by closed forms and exhaustive search on tiny instances

@@ -12,7 +12,7 @@ weight [c_out][c_in], bias; squeeze-excite w1 [k][c], b1 [k], w2 [c][k], b2 [c].
 import numpy as np
 from . import layers as L
 
-__all__ = ["Stage", "layer_profile"]
+__all__ = ["Stage", "layer_profile", "group_step"]
 
 
 def _layer_param_shapes(layer):
@@ -225,6 +225,25 @@ class Stage:
 
     def layer_outputs(self, mb):
         return self.saved[mb][0]
+
+
+def group_step(stages, shares, lr, momentum):
+    """Update of a device group that runs one stage data-parallel (Section 3.2: every device of the group holds the
+    stage model and processes its share y_d of each micro-batch; the gradients are synchronised with AllReduce, Eq. (5),
+    before they are applied).  Each device's micro-batch loss is a mean over its own samples, so the gradient of the
+    whole micro-batch's mean loss is sum_d (y_d / B) G_d with B = sum_d y_d; every device then applies the same
+    SGD-momentum step to its copy of the parameters.  reading: the paper does not say how shares of unequal size are
+    weighted; y_d / B is the weighting under which a BatchNorm-free group reproduces the single-device round."""
+    B = float(sum(shares))
+    if any(st.n_accumulated != st.M for st in stages):
+        raise RuntimeError("step before all micro-batches were accumulated")
+    keys = list(stages[0].p)
+    total = {k: sum((y / B) * st.G[k] for st, y in zip(stages, shares)) for k in keys}
+    for st in stages:
+        for k in keys:
+            st.p[k], st.v[k] = L.sgd_momentum_step(st.p[k], st.v[k], total[k], st.M, lr, momentum)
+            st.G[k] = np.zeros_like(st.G[k])
+        st.n_accumulated = 0
 
 
 def layer_profile(net, first, last, in_h, in_w, layer, batch, elem_bytes):

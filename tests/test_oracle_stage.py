@@ -179,6 +179,42 @@ def test_accumulated_gradient_equals_full_batch_gradient_without_bn(act):
     assert rel(st.flat_params(), full.flat_params()) < 1e-14
 
 
+@pytest.mark.parametrize("shares", [(2, 2), (3, 1), (1, 2, 1)])
+def test_group_of_devices_without_bn_reproduces_the_single_device_round(shares):
+    """Section 3.2: a group runs the stage data-parallel on shares y_d of every micro-batch and synchronises the gradients
+    before the update.  Without BatchNorm the group's update must be the single device's, for equal and unequal shares."""
+    net = si.bnfree_net(4, 2, "relu6")
+    first, last, h, w, M = 0, len(net) - 1, 5, 5, 3
+    B = sum(shares)
+    one, out, xs, tg, params = run_round(net, first, last, h, w, B, M, "mse", seed=8)
+    one.step(0.05, 0.9)
+    group = [O.Stage(net, first, last, y, M, params) for y in shares]
+    lo = 0
+    for st, y in zip(group, shares):
+        for m in range(M):
+            ym = st.forward(m, xs[m][lo:lo + y])
+            _, dy = O.mse_loss(ym, tg[m][lo:lo + y])
+            st.backward(m, dy)
+            st.accumulate(m)
+        lo += y
+    O.group_step(group, shares, 0.05, 0.9)
+    for st in group:
+        assert rel(st.flat_params(), one.flat_params()) < 1e-13
+        assert rel(st.flat_momentum(), one.flat_momentum()) < 1e-13
+        assert not st.flat_grad_accum().any()
+    # a wrong weighting (plain mean over devices) differs as soon as the shares are unequal
+    if len(set(shares)) > 1:
+        wrong = [O.Stage(net, first, last, y, M, params) for y in shares]
+        lo = 0
+        for st, y in zip(wrong, shares):
+            for m in range(M):
+                _, dy = O.mse_loss(st.forward(m, xs[m][lo:lo + y]), tg[m][lo:lo + y])
+                st.backward(m, dy); st.accumulate(m)
+            lo += y
+        O.group_step(wrong, [1] * len(shares), 0.05, 0.9)
+        assert rel(wrong[0].flat_params(), one.flat_params()) > 1e-6
+
+
 def test_with_bn_single_microbatch_round_is_the_plain_minibatch_step():
     net = si.block_net(4, 2)
     st, out, xs, tg, params = run_round(net, 0, len(net) - 1, 5, 5, 4, 1, "mse", seed=2)
