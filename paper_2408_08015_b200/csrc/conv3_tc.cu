@@ -745,7 +745,11 @@ void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, v
     a.x = x; a.w = wb; a.out = (__nv_bfloat16*)z; a.err = err;
     a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.C = g.ci; a.N = g.co; a.flip = 0;
     double px = (double)g.n * g.hi * g.wi;
-    launch_c3<false>(a, K_CONV3_FWD_TC, 2.0 * px * (g.ci + g.co) + 2.0 * 9 * g.ci * g.co, useful_flops, st);
+    const double bytes = 2.0 * px * (g.ci + g.co) + 2.0 * 9 * g.ci * g.co;
+    if (conv3_pipe(false, g.n, g.hi, g.wi, g.ci, g.co, x, GradSrc{}, wb, nullptr, z, err, K_CONV3_FWD_TC, bytes,
+                   useful_flops > 0 ? useful_flops : 2.0 * 9.0 * px * g.ci * g.co, st))
+        return;
+    launch_c3<false>(a, K_CONV3_FWD_TC, bytes, useful_flops, st);
 }
 
 void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st,
@@ -754,8 +758,11 @@ void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16
     a.dz = dz; a.w = wtb; a.addend = addend; a.out = (__nv_bfloat16*)dx; a.err = err;
     a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.C = g.co; a.N = g.ci; a.flip = 1;
     double px = (double)g.n * g.hi * g.wi;
-    launch_c3<true>(a, K_CONV3_BWD_DATA_TC,
-                    2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci * (addend ? 2.0 : 1.0) + 2.0 * 9 * g.ci * g.co, useful_flops, st);
+    const double bytes = 2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci * (addend ? 2.0 : 1.0) + 2.0 * 9 * g.ci * g.co;
+    if (conv3_pipe(true, g.n, g.hi, g.wi, g.co, g.ci, ValSrc{}, dz, wtb, addend, dx, err, K_CONV3_BWD_DATA_TC, bytes,
+                   useful_flops > 0 ? useful_flops : 2.0 * 9.0 * px * g.ci * g.co, st))
+        return;
+    launch_c3<true>(a, K_CONV3_BWD_DATA_TC, bytes, useful_flops, st);
 }
 
 bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g) {

@@ -119,6 +119,10 @@ bool conv3_tc_supported(int dtype, const ConvGeom& g);
 void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st, double useful_flops = 0);
 void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st,
                        double useful_flops = 0);
+// pipelined form (conv3_pipe.cu) for up to 128 reduction channels: forward (bwd == false: x, w = [c_out][9][c_in], C = c_in,
+// N = c_out) or backward-data (bwd == true: dz, w = [c_in][9][c_out], C = c_out, N = c_in); false = layer does not fit, nothing launched
+bool conv3_pipe(bool bwd, int n_img, int H, int W, int C, int N, const ValSrc& x, const GradSrc& dz, const __nv_bfloat16* w, const void* addend,
+                void* out, int* err, int kind, double bytes, double flops, cudaStream_t st);
 bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g);
 void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                          cudaStream_t st, double useful_flops = 0);
