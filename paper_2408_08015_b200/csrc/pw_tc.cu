@@ -15,6 +15,7 @@
 
 #include "kernels.h"
 #include "tc_common.cuh"
+#include "tma.cuh"
 
 namespace ast {
 namespace {
@@ -551,7 +552,10 @@ struct PipeArgs {
     int need_z;                 // backward: the transform also reads z
     uint32_t raw_bytes;         // bytes of one raw stage (both tensors), multiple of 128
     uint32_t a_bytes, b_bytes;  // one operand stage / the resident weights
-    uint32_t o_bytes;           // one output staging tile [128][N] bf16 (multiple of 128)
+    uint32_t o_bytes;           // one output staging tile
+    int panels;                 // staging tile layout: 1 = 64-channel panels of [128 rows][128 bytes], 16-byte chunks XOR-swizzled with the
+                                // row, stored by tiled tensor copies (N a multiple of 64); 0 = [128][N] row-major, stored by one bulk copy
+    uint32_t z_bytes;           // one tile [128][N] bf16 of the producing unit's raw output (backward sums), multiple of 128
     int OS;                     // output staging tiles: 1 or 2
     int AS;                     // operand stages: 2, or 1 where a long reduction leaves no room for two
     int xf_warps;               // of the 12 worker warps, how many transform (4 or 8); the rest run the epilogue: a tile
@@ -567,7 +571,8 @@ struct PipeArgs {
 
 // EXTRA: the epilogue adds the bias (forward) or the residual gradient (backward); a template
 // parameter because even a never-taken branch around those loads slows the epilogue's inner loop.
-template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const PipeArgs a) {
+// PANELS: layout of the output staging tile (see PipeArgs::panels); a template parameter for the same reason.
+template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(PIPE_THREADS, 1) pw_pipe_kernel(const __grid_constant__ CUtensorMap tm_out, const PipeArgs a) {
     // Set-up that reads nothing the previous kernel in the stream writes (barriers, tensor memory, the resident
     // weights: written only by the refresh kernel, which never releases its dependents before it has completed) runs before
     // the dependency wait and so overlaps the previous kernel's tail.
@@ -581,9 +586,9 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = base;                               // operand stages (a.AS of them)
     uint8_t* sB = base + (size_t)a.AS * a.a_bytes;    // resident weights
-    uint8_t* sR = sB + a.b_bytes;                     // raw ring
-    uint8_t* sO = sR + (size_t)a.R * a.raw_bytes;     // output staging tiles
-    uint8_t* sZ = sO + (size_t)a.OS * a.o_bytes;      // backward sums: two tiles of the producing unit's raw output
+    uint8_t* sO = sB + a.b_bytes;                     // output staging tiles (1024-byte aligned: the swizzle is a function of the address)
+    uint8_t* sR = sO + (size_t)a.OS * a.o_bytes;      // raw ring
+    uint8_t* sZ = sR + (size_t)a.R * a.raw_bytes;     // backward sums: two tiles of the producing unit's raw output
     const bool bred = BWD && a.r_partial != nullptr;
     const bool csum = bred || (!BWD && a.stat_partial != nullptr);   // the transform warps take column sums of every output tile
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -683,7 +688,7 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
                 const int valid = min(TM, a.P - tile * TM);
                 const uint32_t bytes = (uint32_t)valid * (uint32_t)a.N * 2u;
                 mbar_expect_tx(zp_full(zb), bytes);
-                bulk_g2s(smem_u32(sZ + (size_t)zb * a.o_bytes), a.rz + (size_t)tile * TM * a.N, bytes, zp_full(zb));
+                bulk_g2s(smem_u32(sZ + (size_t)zb * a.z_bytes), a.rz + (size_t)tile * TM * a.N, bytes, zp_full(zb));
             }
             for (int k = (zissued > 2 ? zissued - 2 : 0); k < zissued; ++k) mbar_wait(zp_full(k & 1), (uint32_t)((k >> 1) & 1));
         }
@@ -750,11 +755,15 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             if (got && ractive) {
                 const uint32_t row_out = (uint32_t)a.N * 2u;
                 const uint8_t* so = sO + (size_t)ob * a.o_bytes;
-                const uint8_t* sz = sZ + (size_t)zb * a.o_bytes;
+                const uint8_t* sz = sZ + (size_t)zb * a.z_bytes;
+                // the thread's four channels inside the staged tile: panel, 16-byte chunk, half of the chunk
+                const uint32_t so_col = (uint32_t)(cu >> 4) * (TM * 128u) + (uint32_t)((cu & 1) << 3);
+                const uint32_t so_chunk = (uint32_t)((cu & 15) >> 1);
                 const int valid = min(TM, a.P - ((int)blockIdx.x + r * (int)gridDim.x) * TM);
 #pragma unroll 4
                 for (int rr = rh; rr < valid; rr += r_split) {
-                    const uint2 dr = *reinterpret_cast<const uint2*>(so + (size_t)rr * row_out + (cu << 3));
+                    const uint2 dr = PANELS ? *reinterpret_cast<const uint2*>(so + so_col + (uint32_t)rr * 128u + ((so_chunk ^ (uint32_t)(rr & 7)) << 4))
+                                              : *reinterpret_cast<const uint2*>(so + (size_t)rr * row_out + (cu << 3));
                     const float d[4] = {__uint_as_float(dr.x << 16), __uint_as_float(dr.x & 0xffff0000u), __uint_as_float(dr.y << 16),
                                         __uint_as_float(dr.y & 0xffff0000u)};
                     if (BWD) {
@@ -855,9 +864,13 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        // The 128 epilogue threads (one accumulator row each) round the tile to bf16 into a
-        // shared-memory staging tile laid out exactly like the output rows in global memory, which
-        // are one contiguous byte range; one thread then stores the tile with a single bulk copy.
+        // The epilogue threads (one accumulator row each) round the tile to bf16 into a shared-memory
+        // staging tile.  With N a multiple of 64 the tile is made of 64-channel panels whose rows are
+        // 128 bytes with the 16-byte chunks XOR-swizzled by the row index: the 32 rows a warp stores at
+        // once then fall into different banks (a row-major tile puts them all into the same four), and
+        // one thread hands the panels to tiled tensor copies that undo the swizzle on the way to global
+        // memory.  Other widths keep the row-major tile, which is the output's own byte range and
+        // leaves with a single bulk copy.
         const int q = warp & 3;                            // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
         const int et = tid - epi_warp0 * 32;
@@ -911,7 +924,9 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) vv[i] += ad[i];
                             }
-                            *reinterpret_cast<uint4*>(so + (size_t)row * row_out + (nn << 1)) = pack8(vv);
+                            const uint32_t so_off = PANELS ? (uint32_t)(nn >> 6) * (TM * 128u) + (uint32_t)row * 128u + ((((uint32_t)(nn & 63) >> 3) ^ (uint32_t)(row & 7)) << 4)
+                                                             : (uint32_t)row * row_out + (uint32_t)(nn << 1);
+                            *reinterpret_cast<uint4*>(so + so_off) = pack8(vv);
                         }
                     }
                 }
@@ -920,9 +935,13 @@ template <bool BWD, bool EXTRA> __global__ void __launch_bounds__(PIPE_THREADS, 
             mbar_arrive(acc_empty(st));
             fence_async_smem();
             named_bar_sync(1, nepi);
-            const int valid = min(TM, a.P - tile * TM);
             if (et == 0) {
-                bulk_s2g(a.out + (size_t)tile * TM * a.N, smem_u32(so), (uint32_t)valid * row_out);
+                if (PANELS) {
+                    // rows past the end of the tensor are clipped by the copy
+                    for (int pn = 0; pn * 64 < a.N; ++pn) tma::store_2d(&tm_out, smem_u32(so) + (uint32_t)pn * (TM * 128u), pn * 64, tile * TM);
+                } else {
+                    bulk_s2g(a.out + (size_t)tile * TM * a.N, smem_u32(so), (uint32_t)min(TM, a.P - tile * TM) * row_out);
+                }
                 bulk_commit();
                 ++issued;
                 if (csum) mbar_arrive(so_full(ob));      // the staged tile is complete (ordered by the named barrier above)
@@ -947,11 +966,12 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
     const int nkb = (a.K + KB - 1) / KB;
     a.a_bytes = (uint32_t)nkb * TM * 128u;
     a.b_bytes = (uint32_t)nkb * (uint32_t)a.NT * 128u;
-    a.o_bytes = ((uint32_t)TM * (uint32_t)a.N * 2u + 127u) / 128u * 128u;
-    if (a.o_bytes < 8192u) a.o_bytes = 8192u;      // also holds the [128 / (N/8)][2][N] floats of the statistics' block sum
+    a.z_bytes = ((uint32_t)TM * (uint32_t)a.N * 2u + 127u) / 128u * 128u;
+    a.panels = a.N % 64 == 0 ? 1 : 0;
+    a.o_bytes = a.panels ? (uint32_t)(a.N / 64) * TM * 128u : (a.z_bytes + 1023u) / 1024u * 1024u;
     const size_t budget = 220 * 1024 - 1024;
     const int tensors = a.need_z ? 2 : 1;
-    const size_t zp = a.r_partial ? 2 * (size_t)a.o_bytes : 0;      // two tiles of the raw output the backward sums read
+    const size_t zp = a.r_partial ? 2 * (size_t)a.z_bytes : 0;      // two tiles of the raw output the backward sums read
     // two operand stages if they fit; one for long reductions (the transform of tile t+1 then waits for the MMAs of t)
     {
         // split of the twelve worker warps: estimated instructions per tile of the two roles, spread over their warps
@@ -994,9 +1014,19 @@ bool plan_pipe(PipeArgs& a, size_t* smem) {
     return false;
 }
 
-template <bool BWD> int launch_pipe(PipeArgs& a, size_t smem, int kind, double bytes, size_t partial_floats, cudaStream_t st) {
-    smem_limit_once<101 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, false>, 222 * 1024);
-    smem_limit_once<102 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, true>, 222 * 1024);
+// tensor map of the output [P][N] for the epilogue's panel stores: boxes of 64 channels x 128 pixels
+bool make_out_map(const void* out, int P, int N, CUtensorMap* m) {
+    const uint64_t dims[2] = {(uint64_t)N, (uint64_t)P};
+    const uint64_t strides[1] = {(uint64_t)N * 2};
+    const uint32_t box[2] = {64, TM};
+    return tma::encode_bf16(m, out, 2, dims, strides, box);
+}
+
+template <bool BWD> int launch_pipe(PipeArgs& a, const CUtensorMap& tm_out, size_t smem, int kind, double bytes, size_t partial_floats, cudaStream_t st) {
+    smem_limit_once<101 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, false, false>, 222 * 1024);
+    smem_limit_once<102 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, true, false>, 222 * 1024);
+    smem_limit_once<103 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, false, true>, 222 * 1024);
+    smem_limit_once<104 + (BWD ? 50 : 0)>(pw_pipe_kernel<BWD, true, true>, 222 * 1024);
     const int n_sm = sm_count();
     int grid = a.tiles < n_sm ? a.tiles : n_sm;
     if (a.stat_partial && (size_t)grid * 2 * a.N > partial_floats) a.stat_partial = nullptr;
@@ -1004,8 +1034,13 @@ template <bool BWD> int launch_pipe(PipeArgs& a, size_t smem, int kind, double b
     const bool fused = BWD ? a.r_partial != nullptr : a.stat_partial != nullptr;
     LaunchScope ls(kind, bytes + (fused ? 8.0 * a.N * grid : 0.0) + (BWD && fused ? 2.0 * a.P * a.N : 0.0), 2.0 * a.P * a.N * a.K, st);
     const bool extra = BWD ? a.addend != nullptr : a.bias != nullptr;
-    if (extra) launch_pdl(pw_pipe_kernel<BWD, true>, grid, PIPE_THREADS, smem, st, a);
-    else launch_pdl(pw_pipe_kernel<BWD, false>, grid, PIPE_THREADS, smem, st, a);
+    if (a.panels) {
+        if (extra) launch_pdl(pw_pipe_kernel<BWD, true, true>, grid, PIPE_THREADS, smem, st, tm_out, a);
+        else launch_pdl(pw_pipe_kernel<BWD, false, true>, grid, PIPE_THREADS, smem, st, tm_out, a);
+    } else {
+        if (extra) launch_pdl(pw_pipe_kernel<BWD, true, false>, grid, PIPE_THREADS, smem, st, tm_out, a);
+        else launch_pdl(pw_pipe_kernel<BWD, false, false>, grid, PIPE_THREADS, smem, st, tm_out, a);
+    }
     return fused ? grid : 0;
 }
 
@@ -1326,7 +1361,8 @@ int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const
             pa.stat_partial = partial;
         }
         size_t smem = 0;
-        if (plan_pipe(pa, &smem)) return launch_pipe<false>(pa, smem, K_PW_FWD_TC, bytes, partial_floats, st);
+        alignas(64) CUtensorMap tm_out;
+        if (plan_pipe(pa, &smem) && make_out_map(z, pa.P, pa.N, &tm_out)) return launch_pipe<false>(pa, tm_out, smem, K_PW_FWD_TC, bytes, partial_floats, st);
     }
     Tiling t = pick_tiling(a.K, a.N);
     launch<false>(a, t, K_PW_FWD_TC, bytes, st);
@@ -1363,7 +1399,9 @@ int pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wt
             pa.r_partial = red->partial;
         }
         size_t smem = 0;
-        if (plan_pipe(pa, &smem)) return launch_pipe<true>(pa, smem, K_PW_BWD_DATA_TC, bytes, with_red ? red->partial_floats : 0, st);
+        alignas(64) CUtensorMap tm_out;
+        if (plan_pipe(pa, &smem) && make_out_map(dx, pa.P, pa.N, &tm_out))
+            return launch_pipe<true>(pa, tm_out, smem, K_PW_BWD_DATA_TC, bytes, with_red ? red->partial_floats : 0, st);
     }
     Tiling t = pick_tiling(a.K, a.N);
     launch<true>(a, t, K_PW_BWD_DATA_TC, bytes, st);
