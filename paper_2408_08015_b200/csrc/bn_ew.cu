@@ -16,44 +16,97 @@ struct StatsOp {
     static constexpr int NACC = 2, NCTX = 1;     // context: the pivot (first pixel's value of each channel)
     const void* z;
     template <typename T, int V> __device__ __forceinline__ void init(int c0, float (*ctx)[V]) const { ld_raw_w<T, V>(z, (size_t)c0, ctx[0]); }
+    static constexpr int NLD = 1;                // tensors read per pixel
+    template <typename T> __device__ __forceinline__ void load(size_t e, Vec<T>* r) const { r[0].load(z, e / Vec<T>::N); }
+    template <typename T, int V> __device__ __forceinline__ void acc_raw(const Vec<T>* r, const float (*ctx)[V], float (*a)[V]) const {
+        float v[V];
+        r[0].unpack(v);
+        acc_vals<V>(v, ctx, a);
+    }
     template <typename T, int V> __device__ __forceinline__ void acc(size_t e, const float (*ctx)[V], float (*a)[V]) const {
         float v[V];
         ld_raw_w<T, V>(z, e, v);
+        acc_vals<V>(v, ctx, a);
+    }
+    template <int V> __device__ __forceinline__ void acc_vals(const float* v, const float (*ctx)[V], float (*a)[V]) const {
+        if (V % 2 == 0) {
+            // two channels per packed fp32 instruction
 #pragma unroll
-        for (int q = 0; q < V; ++q) {
-            float d = v[q] - ctx[0][q];
-            a[0][q] += d;
-            a[1][q] = fmaf(d, d, a[1][q]);
+            for (int q = 0; q < V; q += 2) {
+                const float2 d = __fadd2_rn(make_float2(v[q], v[q + 1]), make_float2(-ctx[0][q], -ctx[0][q + 1]));
+                const float2 s1 = __fadd2_rn(make_float2(a[0][q], a[0][q + 1]), d);
+                const float2 s2 = __ffma2_rn(d, d, make_float2(a[1][q], a[1][q + 1]));
+                a[0][q] = s1.x; a[0][q + 1] = s1.y;
+                a[1][q] = s2.x; a[1][q + 1] = s2.y;
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < V; ++q) {
+                float d = v[q] - ctx[0][q];
+                a[0][q] += d;
+                a[1][q] = fmaf(d, d, a[1][q]);
+            }
         }
     }
 };
 
-// sums of dpre = dy*mask(pre) and of dpre*xhat; the per-channel coefficients live in registers
+// sums of dpre = dy*mask(pre) and of dpre*xhat; the per-channel coefficients live in registers.  The activation is a pair
+// of bounds (ReLU6: 0..6, ReLU: 0..inf, none: -inf..inf) so that every storage type and activation runs one instruction
+// stream; xhat = z*rstd - mean*rstd is one fused multiply-add.
 struct BwdOp {
-    static constexpr int NACC = 2, NCTX = 4;     // context: scale, shift, mean, rstd
+    static constexpr int NACC = 2, NCTX = 4;     // context: scale, shift, -mean*rstd, rstd
     GradSrc g;            // k1 unused here
     const float* mean;
     const float* rstd;
+    float lo, hi;
     template <typename T, int V> __device__ __forceinline__ void init(int c0, float (*ctx)[V]) const {
 #pragma unroll
         for (int q = 0; q < V; ++q) {
             ctx[0][q] = g.scale ? __ldg(g.scale + c0 + q) : 1.f;
             ctx[1][q] = g.scale ? __ldg(g.shift + c0 + q) : 0.f;
-            ctx[2][q] = mean ? __ldg(mean + c0 + q) : 0.f;
             ctx[3][q] = mean ? __ldg(rstd + c0 + q) : 0.f;
+            ctx[2][q] = mean ? -__ldg(mean + c0 + q) * ctx[3][q] : 0.f;
         }
     }
+    static constexpr int NLD = 2;
+    template <typename T> __device__ __forceinline__ void load(size_t e, Vec<T>* r) const {
+        r[0].load(g.dy, e / Vec<T>::N);
+        if (g.act != ACT_NONE || mean) r[1].load(g.z, e / Vec<T>::N);
+    }
+    template <typename T, int V> __device__ __forceinline__ void acc_raw(const Vec<T>* r, const float (*ctx)[V], float (*a)[V]) const {
+        float d[V], z[V];
+        r[0].unpack(d);
+        if (g.act != ACT_NONE || mean) r[1].unpack(z);
+        acc_vals<V>(d, z, ctx, a);
+    }
     template <typename T, int V> __device__ __forceinline__ void acc(size_t e, const float (*ctx)[V], float (*a)[V]) const {
-        float d[V];
+        float d[V], z[V];
         ld_raw_w<T, V>(g.dy, e, d);
+        if (g.act != ACT_NONE || mean) ld_raw_w<T, V>(g.z, e, z);
+        acc_vals<V>(d, z, ctx, a);
+    }
+    template <int V> __device__ __forceinline__ void acc_vals(const float* d, const float* z, const float (*ctx)[V], float (*a)[V]) const {
         if (g.act != ACT_NONE || mean) {
-            float z[V];
-            ld_raw_w<T, V>(g.z, e, z);
+            if (V % 2 == 0) {
 #pragma unroll
-            for (int q = 0; q < V; ++q) {
-                float dm = d[q] * act_mask(fmaf(z[q], ctx[0][q], ctx[1][q]), g.act);
-                a[0][q] += dm;
-                a[1][q] = fmaf(dm, (z[q] - ctx[2][q]) * ctx[3][q], a[1][q]);
+                for (int q = 0; q < V; q += 2) {
+                    const float2 z2 = make_float2(z[q], z[q + 1]);
+                    const float2 pre = __ffma2_rn(z2, make_float2(ctx[0][q], ctx[0][q + 1]), make_float2(ctx[1][q], ctx[1][q + 1]));
+                    const float2 xh = __ffma2_rn(z2, make_float2(ctx[3][q], ctx[3][q + 1]), make_float2(ctx[2][q], ctx[2][q + 1]));
+                    const float2 dm = make_float2((pre.x > lo && pre.x < hi) ? d[q] : 0.f, (pre.y > lo && pre.y < hi) ? d[q + 1] : 0.f);
+                    const float2 s1 = __fadd2_rn(make_float2(a[0][q], a[0][q + 1]), dm);
+                    const float2 s2 = __ffma2_rn(dm, xh, make_float2(a[1][q], a[1][q + 1]));
+                    a[0][q] = s1.x; a[0][q + 1] = s1.y;
+                    a[1][q] = s2.x; a[1][q + 1] = s2.y;
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < V; ++q) {
+                    const float pre = fmaf(z[q], ctx[0][q], ctx[1][q]);
+                    const float dm = (pre > lo && pre < hi) ? d[q] : 0.f;
+                    a[0][q] += dm;
+                    a[1][q] = fmaf(dm, fmaf(z[q], ctx[3][q], ctx[2][q]), a[1][q]);
+                }
             }
         } else {
 #pragma unroll
@@ -82,8 +135,20 @@ __global__ void __launch_bounds__(512) chan_reduce_kernel(OP op, size_t pixels, 
         float ctx[OP::NCTX][V];
         op.template init<T, V>(c0, ctx);
         size_t pbeg = (size_t)blockIdx.y * pix_per_block, pend = min(pixels, pbeg + pix_per_block);
-#pragma unroll 8
-        for (size_t p = pbeg + row; p < pend; p += rows) op.template acc<T, V>(p * c + c0, ctx, a);
+        size_t p = pbeg + row;
+        if (V == Vec<T>::N) {
+            // the loads of a batch of pixels (eight vectors per thread) are issued before any is used: with one block per SM
+            // the bytes in flight come from each thread's own batch
+            constexpr int U = 8 / OP::NLD;
+            for (; p + (size_t)(U - 1) * rows < pend; p += (size_t)U * rows) {
+                Vec<T> r[U][OP::NLD];
+#pragma unroll
+                for (int u = 0; u < U; ++u) op.template load<T>((p + (size_t)u * rows) * c + c0, r[u]);
+#pragma unroll
+                for (int u = 0; u < U; ++u) op.template acc_raw<T, V>(r[u], ctx, a);
+            }
+        }
+        for (; p < pend; p += rows) op.template acc<T, V>(p * c + c0, ctx, a);
     }
     const int width = cw * V;
     for (int t = 0; t < OP::NACC; ++t) {
@@ -523,7 +588,8 @@ void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int 
                    const float* mean, const float* rstd, const float* gamma, float* scratch, size_t scratch_floats, const BnBwdOut& o,
                    cudaStream_t st) {
     ReducePlan p = plan_reduce(dtype, pixels, c, 2, scratch_floats);
-    BwdOp op{GradSrc{dy, z, scale, shift, nullptr, nullptr, nullptr, act}, mean, rstd};
+    BwdOp op{GradSrc{dy, z, scale, shift, nullptr, nullptr, nullptr, act}, mean, rstd, act == ACT_NONE ? -INFINITY : 0.f,
+             act == ACT_RELU6 ? 6.f : INFINITY};
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_BWD_REDUCE, (double)pixels * c * esz(dtype) * ((act != ACT_NONE || mean) ? 2.0 : 1.0), st);
     LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
     launch_pdl(bn_bwd_finish, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);

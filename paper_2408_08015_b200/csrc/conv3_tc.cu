@@ -703,29 +703,38 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
     (void)kbi; (void)kbo;
 }
 
+// out[i] = sum over splits of partial[split][i], n a multiple of 4.  A block finishes 128 consecutive outputs: warp kg adds
+// the splits kg, kg+32, ... (each lane four consecutive outputs: 512 contiguous bytes per split and warp, all of a
+// thread's loads issued before the additions), the 32 sub-sums are combined in index order through shared memory.
 __global__ void __launch_bounds__(1024) reduce_splits_c3(const float* __restrict__ partial, int splits, size_t n, float* __restrict__ out) {
     pdl_wait();
     pdl_launch();
-    __shared__ float sh[32][33];
+    __shared__ float4 sh[32][33];
     const int il = threadIdx.x & 31, kg = threadIdx.x >> 5;
-    const size_t i = (size_t)blockIdx.x * 32 + il;
-    float acc = 0.f;
+    const size_t i = ((size_t)blockIdx.x * 32 + il) * 4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i < n) {
-        for (int k0 = kg; k0 < splits; k0 += 32 * 8) {
-            float v[8];
+        for (int k0 = kg; k0 < splits; k0 += 32 * 4) {
+            float4 v[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = (k0 + 32 * u < splits) ? partial[(size_t)(k0 + 32 * u) * n + i] : 0.f;
+            for (int u = 0; u < 4; ++u)
+                v[u] = (k0 + 32 * u < splits) ? *reinterpret_cast<const float4*>(partial + (size_t)(k0 + 32 * u) * n + i) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) acc += v[u];
+            for (int u = 0; u < 4; ++u) {
+                acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
+            }
         }
     }
     sh[kg][il] = acc;
     __syncthreads();
     if (kg == 0 && i < n) {
-        float s = 0.f;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 32; ++k) s += sh[k][il];
-        out[i] = s;
+        for (int k = 0; k < 32; ++k) {
+            const float4 v = sh[k][il];
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+        *reinterpret_cast<float4*>(out + i) = s;
     }
 }
 
@@ -772,6 +781,19 @@ bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g) {
 
 void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                          cudaStream_t st, double useful_flops) {
+    {
+        // the pipelined kernel fed by tensor copies, where the layer fits it
+        const double px = (double)g.n * g.hi * g.wi;
+        const size_t out_elems = (size_t)g.co * 9 * g.ci;
+        const int ctas = conv3_wgrad_pipe(g.n, g.hi, g.wi, g.ci, g.co, dz, x, scratch, scratch_floats, err,
+                                          2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci,
+                                          useful_flops > 0 ? useful_flops : 2.0 * 9.0 * px * g.ci * g.co, st);
+        if (ctas > 0) {
+            LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);
+            launch_pdl(reduce_splits_c3, (unsigned)((out_elems / 4 + 31) / 32), 1024, 0, st, scratch, ctas, out_elems, gw);
+            return;
+        }
+    }
     W3Args a{};
     a.dz = dz; a.x = x; a.partial = scratch; a.err = err;
     a.n_img = g.n; a.H = g.hi; a.W = g.wi; a.CI = g.ci; a.CO = g.co;
@@ -802,7 +824,7 @@ void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, 
         launch_pdl(conv3_wgrad_tc_kernel, dim3(ctas, groups), C3_THREADS, smem, st, a);
     }
     LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);
-    launch_pdl(reduce_splits_c3, (unsigned)((out_elems + 31) / 32), 1024, 0, st, scratch, ctas, out_elems, gw);
+    launch_pdl(reduce_splits_c3, (unsigned)((out_elems / 4 + 31) / 32), 1024, 0, st, scratch, ctas, out_elems, gw);
 }
 
 }  // namespace ast

@@ -123,6 +123,10 @@ void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16
 // N = c_out) or backward-data (bwd == true: dz, w = [c_in][9][c_out], C = c_out, N = c_in); false = layer does not fit, nothing launched
 bool conv3_pipe(bool bwd, int n_img, int H, int W, int C, int N, const ValSrc& x, const GradSrc& dz, const __nv_bfloat16* w, const void* addend,
                 void* out, int* err, int kind, double bytes, double flops, cudaStream_t st);
+// pipelined weight gradient (conv3_wgrad_pipe.cu): writes per-CTA partials [ctas][c_out][9][c_in] and returns ctas, or 0 if the
+// layer does not fit (nothing launched)
+int conv3_wgrad_pipe(int n_img, int H, int W, int CI, int CO, const GradSrc& dz, const ValSrc& x, float* partial, size_t partial_floats, int* err,
+                     double bytes, double flops, cudaStream_t st);
 bool conv3_wgrad_tc_supported(int dtype, const ConvGeom& g);
 void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                          cudaStream_t st, double useful_flops = 0);

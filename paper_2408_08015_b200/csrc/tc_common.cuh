@@ -184,6 +184,41 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Issue forms for a whole warp in convergent control flow: every lane executes the instruction stream (so that the
+// descriptor arithmetic can stay in the uniform datapath) and the elected lane alone issues.
+__device__ __forceinline__ uint32_t elect_leader() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "elect.sync _|p, 0xffffffff;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(pred));
+    return pred;
+}
+__device__ __forceinline__ void umma_bf16_lead(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate, uint32_t leader) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "setp.ne.b32 q, %5, 0;\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_lead(uint32_t mbar, uint32_t leader) {
+    asm volatile(
+        "{\n"
+        ".reg .pred q;\n"
+        "setp.ne.b32 q, %1, 0;\n"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+        "}\n" ::"r"(mbar),
+        "r"(leader)
+        : "memory");
+}
+
 // Branch-free operand transforms with per-thread register coefficients.  Absent BatchNorm
 // terms take neutral values (scale 1, shift 0, k1 1, k2 = k3 0) and the activation becomes a pair
 // of bounds (ReLU6: 0..6, ReLU: 0..inf, none: -inf..inf), so that every lane runs the same
