@@ -223,29 +223,64 @@ __device__ __forceinline__ void umma_commit_lead(uint32_t mbar, uint32_t leader)
 // terms take neutral values (scale 1, shift 0, k1 1, k2 = k3 0) and the activation becomes a pair
 // of bounds (ReLU6: 0..6, ReLU: 0..inf, none: -inf..inf), so that every lane runs the same
 // instruction stream whatever its operand.
+// These transforms are bound by the integer / min-max / convert pipe (64 lanes per clock and SM, half the fused
+// multiply-add pipe's rate), so they keep that pipe's work to the two unpacks and one pack per pair of elements it cannot
+// avoid: the clamp of an activation is applied AFTER rounding, on packed bfloat16 pairs (rounding is monotonic and the
+// bounds 0 and 6 are bfloat16 numbers, so the result is the same), and the activation mask of the backward transform is
+// formed on the multiply-add pipe as a saturated product instead of a compare and a select.
 struct XfVal {
-    float cs[8], ch[8], lo, hi;
+    float cs[8], ch[8];
+    int act;
     __device__ __forceinline__ void init(const ValSrc& s, int c0) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             cs[q] = s.scale ? __ldg(s.scale + c0 + q) : 1.f;
             ch[q] = s.scale ? __ldg(s.shift + c0 + q) : 0.f;
         }
-        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
-        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
+        act = s.act;
     }
     __device__ __forceinline__ uint4 apply(const uint4& raw) const {
         Vec<__nv_bfloat16> v;
         v.raw = raw;
         float f[8];
         v.unpack(f);
+        uint32_t w[4];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) f[q] = fminf(fmaxf(fmaf(f[q], cs[q], ch[q]), lo), hi);
-        return pack8(f);
+        for (int q = 0; q < 8; q += 2) {
+            const float2 r = __ffma2_rn(make_float2(f[q], f[q + 1]), make_float2(cs[q], cs[q + 1]), make_float2(ch[q], ch[q + 1]));
+            __nv_bfloat162 h = __floats2bfloat162_rn(r.x, r.y);
+            w[q >> 1] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        if (act != ACT_NONE) {                      // uniform branch
+            const __nv_bfloat162 zero = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                __nv_bfloat162 h = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&w[i]), zero);
+                w[i] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            if (act == ACT_RELU6) {
+                const __nv_bfloat162 six = __floats2bfloat162_rn(6.f, 6.f);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    __nv_bfloat162 h = __hmin2(*reinterpret_cast<__nv_bfloat162*>(&w[i]), six);
+                    w[i] = *reinterpret_cast<uint32_t*>(&h);
+                }
+            }
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
     }
 };
+// 1 for v > 0 (denormals included), 0 for v <= 0, formed on the multiply-add pipe: saturate(v * 2^126) is 1 for every
+// normal positive v and at least 2^-23 for a denormal one, which the second product lifts to 1.
+__device__ __forceinline__ float step_pos(float v) {
+    float m;
+    asm("mul.sat.f32 %0, %1, 0f7E800000;" : "=f"(m) : "f"(v));
+    asm("mul.sat.f32 %0, %1, 0f7E800000;" : "=f"(m) : "f"(m));
+    return m;
+}
 struct XfGrad {
-    float cs[8], ch[8], k1[8], k2[8], k3[8], lo, hi;
+    float cs[8], ch[8], k1[8], k2[8], k3[8];
+    int act;
     __device__ __forceinline__ void init(const GradSrc& s, int c0) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -255,8 +290,7 @@ struct XfGrad {
             k2[q] = s.k1 ? __ldg(s.k2 + c0 + q) : 0.f;
             k3[q] = s.k1 ? __ldg(s.k3 + c0 + q) : 0.f;
         }
-        lo = s.act == ACT_NONE ? -INFINITY : 0.f;
-        hi = s.act == ACT_RELU6 ? 6.f : INFINITY;
+        act = s.act;
     }
     __device__ __forceinline__ uint4 apply(const uint4& rawdy, const uint4& rawz) const {
         Vec<__nv_bfloat16> v;
@@ -265,17 +299,24 @@ struct XfGrad {
         v.unpack(f);
         v.raw = rawz;
         v.unpack(z);
+        if (act != ACT_NONE) {                      // uniform branch: dy <- dy * [pre strictly inside the linear region]
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            // lo < pre < hi  <=>  (pre - lo) * (hi - pre) > 0: differences of floats keep their sign
-            // exactly, infinite bounds give +inf, and 0 * inf = NaN compares false (pre == 0 under ReLU);
-            // the test runs on the FMA pipe and guards one predicated fused multiply-add
-            const float pre = fmaf(z[q], cs[q], ch[q]);
-            float o = fmaf(k3[q], z[q], k2[q]);
-            if ((pre - lo) * (hi - pre) > 0.f) o = fmaf(k1[q], f[q], o);
-            f[q] = o;
+            for (int q = 0; q < 8; ++q) {
+                const float pre = fmaf(z[q], cs[q], ch[q]);
+                float m = step_pos(pre);
+                if (act == ACT_RELU6) m *= step_pos(6.f - pre);
+                f[q] *= m;
+            }
         }
-        return pack8(f);
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 8; q += 2) {
+            float2 o = __ffma2_rn(make_float2(k3[q], k3[q + 1]), make_float2(z[q], z[q + 1]), make_float2(k2[q], k2[q + 1]));
+            o = __ffma2_rn(make_float2(k1[q], k1[q + 1]), make_float2(f[q], f[q + 1]), o);
+            __nv_bfloat162 h = __floats2bfloat162_rn(o.x, o.y);
+            w[q >> 1] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
     }
 };
 
