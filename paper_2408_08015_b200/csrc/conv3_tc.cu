@@ -48,7 +48,9 @@ template <bool BWD> __global__ void __launch_bounds__(C3_THREADS) conv3_tc_kerne
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2];
     __shared__ uint32_t tmem_slot;
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Wp = a.W + 2;
     const int kbs = a.C >> 6;                               // 64-channel blocks
@@ -256,7 +258,9 @@ template <bool BWD, int IT, int NTHR> __global__ void __launch_bounds__(NTHR, NT
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2];
     __shared__ uint32_t tmem_slot;
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Wp = a.W + 2;
     const int kbs = a.C >> 6;
@@ -543,7 +547,9 @@ __global__ void __launch_bounds__(C3_THREADS) conv3_wgrad_tc_kernel(const W3Args
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bar_store;
     __shared__ uint32_t tmem_slot;
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Wp = a.W + 2;
     const int kbi = a.CI >> 6, kbo = (a.CO + 63) >> 6;

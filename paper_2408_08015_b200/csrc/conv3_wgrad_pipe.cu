@@ -83,7 +83,9 @@ conv3_wgrad_pipe_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_store;
     volatile int* abort_flag = &abort_store;
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Wp = a.W + 2, kbi = a.CI >> 6, kbo = a.CO >> 6, S = a.S, ZS = a.ZS;
     uint8_t* sSt = base;                                   // stages: [x blocks][dy blocks]

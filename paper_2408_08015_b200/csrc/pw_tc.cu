@@ -47,7 +47,9 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
     __shared__ uint32_t tmem_slot;
     __shared__ int failed;
     // 1024-byte aligned operand area (the swizzle pattern is a function of the address bits)
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int NT = a.NT;
     uint8_t* sA = base;
     uint8_t* sB = base + (size_t)(a.KC / KB) * TM * 128;
@@ -279,7 +281,9 @@ __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArg
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t mbar_store[2];
     __shared__ uint32_t tmem_slot;
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * TM;                    // first output channel of this CTA
     const int n0 = blockIdx.z * a.NT;                  // first input channel
@@ -583,7 +587,9 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_store;
     volatile int* abort_flag = &abort_store;
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t* sA = base;                               // operand stages (a.AS of them)
     uint8_t* sB = base + (size_t)a.AS * a.a_bytes;    // resident weights
     uint8_t* sO = sB + a.b_bytes;                     // output staging tiles (1024-byte aligned: the swizzle is a function of the address)
@@ -609,17 +615,17 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
     if (tid == 0) {
         for (int s = 0; s < R; ++s) {
             mbar_init(raw_full(s), 1);
-            mbar_init(raw_empty(s), nxf);
+            mbar_init(raw_empty(s), a.xf_warps);
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(a_full(s), nxf);
+            mbar_init(a_full(s), a.xf_warps);
             mbar_init(a_empty(s), 1);
             mbar_init(acc_full(s), 1);
-            mbar_init(acc_empty(s), nepi);
+            mbar_init(acc_empty(s), PIPE_WORKERS - a.xf_warps);
             mbar_init(zp_full(s), 1);
-            mbar_init(zp_empty(s), nxf);
+            mbar_init(zp_empty(s), a.xf_warps);
             mbar_init(so_full(s), 1);
-            mbar_init(so_free(s), nxf);
+            mbar_init(so_free(s), a.xf_warps);
         }
         abort_store = 0;
     }
@@ -694,9 +700,13 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // every lane runs the loop (convergent control flow keeps the descriptor arithmetic in the uniform datapath: a
+        // single diverged lane issues at about half the rate), the elected lane issues
+        {
+            const uint32_t leader = elect_leader();
             const uint32_t idesc = make_idesc(NT);
-            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+            const uint64_t dconst = make_desc(0);
+            const uint32_t a0 = smem_u32(sA) >> 4, b0 = smem_u32(sB) >> 4;
             const int steps = vpr_pad >> 1;
             for (int t = 0; t < my_tiles; ++t) {
                 const int st = t & 1, n = t >> 1;                                    // accumulator stage and its use count
@@ -705,13 +715,15 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
                 if (n > 0 && !mbar_wait_abortable(acc_empty(st), (uint32_t)((n - 1) & 1), abort_flag)) break;
                 fence_after_sync();
                 const uint32_t d = tmem + (uint32_t)(st * NT);
+                const uint32_t as0 = a0 + ((uint32_t)as * a.a_bytes >> 4);
                 for (int k = 0; k < steps; ++k) {
-                    const int kb = k >> 2, ks = k & 3;
-                    umma_bf16(d, make_desc(a0 + as * a.a_bytes + (uint32_t)kb * TM * 128u + (uint32_t)ks * 32u),
-                              make_desc(b0 + (uint32_t)kb * (uint32_t)NT * 128u + (uint32_t)ks * 32u), idesc, k > 0 ? 1u : 0u);
+                    const uint32_t kb = (uint32_t)k >> 2, ks = (uint32_t)k & 3u;
+                    umma_bf16_lead(d, dconst + (uint64_t)(as0 + kb * (TM * 8u) + ks * 2u), dconst + (uint64_t)(b0 + kb * ((uint32_t)NT * 8u) + ks * 2u), idesc,
+                                   k > 0 ? 1u : 0u, leader);
                 }
-                umma_commit(a_empty(as));
-                umma_commit(acc_full(st));
+                umma_commit_lead(a_empty(as), leader);
+                umma_commit_lead(acc_full(st), leader);
+                __syncwarp();
             }
         }
     } else if (warp < epi_warp0) {
@@ -787,8 +799,12 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
                     }
                 }
             }
-            mbar_arrive(so_free(ob));
-            if (BWD) mbar_arrive(zp_empty(zb));
+            // one arrival per warp (an arrival is a shared-memory atomic: hundreds of them per hand-off serialise)
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(so_free(ob));
+                if (BWD) mbar_arrive(zp_empty(zb));
+            }
             return got;
         };
         int it = 0, reduced_tiles = 0;
@@ -826,11 +842,13 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
                         *reinterpret_cast<uint4*>(dstA + tile_off(sub * RS + rl, j, TM)) = q4;
                     }
                 }
-                mbar_arrive(raw_empty(s));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(raw_empty(s));
             }
             if (!ok) break;
             fence_async_smem();
-            mbar_arrive(a_full(st));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(a_full(st));
             // as many tiles behind as there are staging tiles: by then that tile's MMA and epilogue have had the time of
             // a whole transform + sum step, and the staging tile it occupies is the next one the epilogue needs back
             if (csum && t >= a.OS) {
@@ -932,7 +950,8 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
                 }
             }
             fence_before_sync();
-            mbar_arrive(acc_empty(st));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(st));
             fence_async_smem();
             named_bar_sync(1, nepi);
             if (et == 0) {
@@ -1079,7 +1098,9 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_store;
     volatile int* abort_flag = &abort_store;
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned start, formed by pointer arithmetic on the shared array: a round trip through an integer would make
+    // every access through it a generic load / store instead of a shared-memory one
+    uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t* sOp = base;                                   // operand stages (a.OPS of them): [A panels][B panels]
     uint8_t* sR = base + (size_t)a.OPS * a.op_bytes;       // raw ring
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1093,10 +1114,10 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
     if (tid == 0) {
         for (int s = 0; s < R; ++s) {
             mbar_init(raw_full(s), 1);
-            mbar_init(raw_empty(s), 256);
+            mbar_init(raw_empty(s), 8);      // one arrival per transform warp
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(op_full(s), 256);
+            mbar_init(op_full(s), 8);
             mbar_init(op_empty(s), 1);
         }
         mbar_init(done_bar, 1);
@@ -1202,9 +1223,13 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
                 if (kr >= valid) q4 = make_uint4(0, 0, 0, 0);
                 *reinterpret_cast<uint4*>(dstB + kr * 128 + (((jb & 7) ^ (kr & 7)) << 4)) = q4;
             }
-            mbar_arrive(raw_empty(s));
+            // one arrival per warp (an arrival is a shared-memory atomic: hundreds of them per hand-off serialise)
             fence_async_smem();
-            mbar_arrive(op_full(st));
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(raw_empty(s));
+                mbar_arrive(op_full(st));
+            }
         }
         if (ok && stages > 0) ok = mbar_wait_abortable(done_bar, 0u, abort_flag);
         if (ok) {
