@@ -178,7 +178,9 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
         }
         fence_async_smem();
         __syncthreads();
-        if (tid == 0) {
+        if (warp == 0) {
+            // the whole warp runs the issue loop in convergent control flow, the elected lane issues
+            const uint32_t leader = elect_leader();
             fence_after_sync();
             const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
             const int steps = vpr_pad >> 1;           // 16 elements per MMA
@@ -186,9 +188,9 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
                 int kb = s >> 2, ks = s & 3;          // 64-element block, 32-byte step inside it
                 uint64_t da = make_desc(a0 + (uint32_t)kb * TM * 128u + (uint32_t)ks * 32u);
                 uint64_t db = make_desc(b0 + (uint32_t)kb * (uint32_t)NT * 128u + (uint32_t)ks * 32u);
-                umma_bf16(tmem, da, db, idesc, (k0 > 0 || s > 0) ? 1u : 0u);
+                umma_bf16_lead(tmem, da, db, idesc, (k0 > 0 || s > 0) ? 1u : 0u, leader);
             }
-            umma_commit(mbar);
+            umma_commit_lead(mbar, leader);
         }
         // all threads wait until the MMAs have consumed shared memory / produced the accumulators
         ok = mbar_wait(mbar, phase);
@@ -458,13 +460,14 @@ __global__ void __launch_bounds__(NTHREADS) pw_bwd_weight_tc_kernel(const PwWArg
         }
         fence_async_smem();
         __syncthreads();
-        if (tid == 0) {
+        if (warp == 0) {
+            const uint32_t leader = elect_leader();
             fence_after_sync();
             const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
 #pragma unroll
             for (int s = 0; s < WSTAGE / 16; ++s)      // 16 pixels = two 8-row groups per MMA
-                umma_bf16(tmem, make_desc_mn(a0 + s * 2048), make_desc_mn(b0 + s * 2048), idesc, (stage > 0 || s > 0) ? 1u : 0u);
-            umma_commit(b ? mbar1 : mbar0);
+                umma_bf16_lead(tmem, make_desc_mn(a0 + s * 2048), make_desc_mn(b0 + s * 2048), idesc, (stage > 0 || s > 0) ? 1u : 0u, leader);
+            umma_commit_lead(b ? mbar1 : mbar0, leader);
         }
         issued[b] = 1;
     }
@@ -1157,7 +1160,9 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
             for (int k = (it > R ? it - R : 0); k < it; ++k) mbar_wait(raw_full(k % R), (uint32_t)((k / R) & 1));
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
+            // every lane runs the loop, the elected lane issues (see the forward / backward-data pipeline)
+            const uint32_t leader = elect_leader();
             const uint32_t idesc = make_idesc(a.NT) | (1u << 15) | (1u << 16);
             bool ok = true;
             for (int it = 0; it < stages && ok; ++it) {
@@ -1173,12 +1178,13 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
                         const uint32_t d = tmem + (uint32_t)((mt * a.ntiles + nt) * a.NT);
 #pragma unroll
                         for (int k = 0; k < WSTAGE / 16; ++k)
-                            umma_bf16(d, make_desc_mn(a0 + (uint32_t)mt * 2u * PANEL + k * 2048), make_desc_mn(b0 + (uint32_t)nt * (uint32_t)(a.NT >> 6) * PANEL + k * 2048),
-                                      idesc, (it > 0 || k > 0) ? 1u : 0u);
+                            umma_bf16_lead(d, make_desc_mn(a0 + (uint32_t)mt * 2u * PANEL + k * 2048),
+                                           make_desc_mn(b0 + (uint32_t)nt * (uint32_t)(a.NT >> 6) * PANEL + k * 2048), idesc, (it > 0 || k > 0) ? 1u : 0u, leader);
                     }
-                umma_commit(op_empty(st));
+                umma_commit_lead(op_empty(st), leader);
+                __syncwarp();
             }
-            if (ok) umma_commit(done_bar);
+            if (ok) umma_commit_lead(done_bar, leader);
         }
     } else {
         // ---------------------------------------------------------------- transformers, then epilogue
