@@ -42,6 +42,13 @@ CASES = {
     "c3_128_128": (si.single_unit_net("conv", 128, 128, k=3), 28, 28, 3, 1, "mse", C3),
     "c3_128_128_bn": (si.single_unit_net("conv", 128, 128, k=3, bn=True), 15, 14, 3, 2, "mse", C3),
     "c3_64_128": (si.single_unit_net("conv", 64, 128, k=3), 15, 14, 3, 1, "mse", C3),
+    # pipelined 3x3 kernels at their edges: a map narrower than one MMA row tile and shorter than a tile of image rows, a
+    # last tile that runs past the bottom row, a single image, more tiles than CTAs (several windows per CTA)
+    "c3_64_64_7x7_bn": (si.single_unit_net("conv", 64, 64, k=3, bn=True), 7, 7, 5, 1, "mse", C3),
+    "c3_128_64_ragged_rows": (si.single_unit_net("conv", 128, 64, k=3, bn=True), 9, 61, 1, 2, "mse", C3),
+    "c3_64_64_many_tiles_bn": (si.single_unit_net("conv", 64, 64, k=3, bn=True), 60, 33, 11, 1, "mse", C3),
+    # 256 channels do not fit the pipelined kernels' resident weights: other kernels take the layer
+    "c3_256_64_fallback": (si.single_unit_net("conv", 256, 64, k=3), 9, 8, 2, 1, "mse", ()),
     # dense 3x3, stride 2, even and odd maps
     "c3_s2_128_128": (si.single_unit_net("conv", 128, 128, k=3, stride=2), 28, 28, 3, 1, "mse", C3[:2]),
     "c3_s2_128_128_bn_odd": (si.single_unit_net("conv", 128, 128, k=3, stride=2, bn=True), 15, 13, 3, 2, "mse", C3[:2]),
