@@ -108,6 +108,10 @@ int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const
 // of the unit that produced this conv's input.  Returns the number of CTAs (for bn_bwd_finish_partials); 0 = none written.
 int pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, const BnRed* red, int* err,
                    cudaStream_t st);
+// streaming form (pw_stream.cu) for stride-1 layers with more than 256 channels on a side (channel counts multiples of 64): forward
+// (bwd == false: x [P][K], w = [N][K]) or backward-data (bwd == true: dz [P][K], w = transposed weights [N][K]); false = does not fit
+bool pw_stream(bool bwd, int P, int K, int N, const ValSrc& x, const GradSrc& dz, const __nv_bfloat16* w, const void* addend, void* out, int* err,
+               int kind, double bytes, cudaStream_t st);
 // gw[co][ci]; per-CTA partial sums in scratch, summed in fixed order by a second kernel
 void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                       cudaStream_t st);

@@ -1395,6 +1395,8 @@ int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const
         alignas(64) CUtensorMap tm_out;
         if (plan_pipe(pa, &smem) && make_out_map(z, pa.P, pa.N, &tm_out)) return launch_pipe<false>(pa, tm_out, smem, K_PW_FWD_TC, bytes, partial_floats, st);
     }
+    // more than 256 channels on a side: the streaming kernel, where the layer fits it
+    if (g.stride == 1 && !bias && pw_stream(false, a.P, a.K, a.N, x, GradSrc{}, wb, nullptr, z, err, K_PW_FWD_TC, bytes, st)) return 0;
     Tiling t = pick_tiling(a.K, a.N);
     launch<false>(a, t, K_PW_FWD_TC, bytes, st);
     return 0;
@@ -1434,6 +1436,9 @@ int pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wt
         if (plan_pipe(pa, &smem) && make_out_map(dx, pa.P, pa.N, &tm_out))
             return launch_pipe<true>(pa, tm_out, smem, K_PW_BWD_DATA_TC, bytes, with_red ? red->partial_floats : 0, st);
     }
+    // the streaming kernel where the gradient needs no transform: with one, its 64-channel blocks are too small a unit of
+    // work for the transform warps' hand-offs and the one-tile kernel below is as fast
+    if (!grad_needs_z(dz) && pw_stream(true, a.P, a.K, a.N, ValSrc{}, dz, wtb, addend, dx, err, K_PW_BWD_DATA_TC, bytes, st)) return 0;
     Tiling t = pick_tiling(a.K, a.N);
     launch<true>(a, t, K_PW_BWD_DATA_TC, bytes, st);
     return 0;
