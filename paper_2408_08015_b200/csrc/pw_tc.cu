@@ -775,7 +775,7 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
                 const uint32_t so_col = (uint32_t)(cu >> 4) * (TM * 128u) + (uint32_t)((cu & 1) << 3);
                 const uint32_t so_chunk = (uint32_t)((cu & 15) >> 1);
                 const int valid = min(TM, a.P - ((int)blockIdx.x + r * (int)gridDim.x) * TM);
-#pragma unroll 4
+#pragma unroll 2
                 for (int rr = rh; rr < valid; rr += r_split) {
                     const uint2 dr = PANELS ? *reinterpret_cast<const uint2*>(so + so_col + (uint32_t)rr * 128u + ((so_chunk ^ (uint32_t)(rr & 7)) << 4))
                                               : *reinterpret_cast<const uint2*>(so + (size_t)rr * row_out + (cu << 3));
@@ -830,7 +830,9 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
                     // loads and arithmetic interleave
                     const int jl = data ? j : 0;
                     const int rows_left = a.P - tile * TM - sub * RS;
-#pragma unroll 4
+                    // not unrolled: the kernel's roles share a small instruction cache, and this loop gains nothing from a
+                    // longer body (a load cannot move above a store that might alias it)
+#pragma unroll 1
                     for (int rl = grp; rl < RS; rl += groups) {
                         const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)rl * row_bytes + (jl << 4));
                         uint4 q4;
@@ -1216,14 +1218,14 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
             const int valid = min(WSTAGE, pend - (pbeg + it * WSTAGE));
             // straight-line bodies: rows past the end of the CTA's range are transformed like any
             // other (stale but in-bounds shared memory) and zeroed afterwards
-#pragma unroll 4
+#pragma unroll 1
             for (int kr = ga; kr < rowsA; kr += groupsA) {
                 const uint4 r0 = *reinterpret_cast<const uint4*>(raw + (size_t)kr * rowA + (ja << 4));
                 uint4 q4 = a.need_z ? xg.apply(r0, *reinterpret_cast<const uint4*>(raw + offZ + (size_t)kr * rowA + (ja << 4))) : r0;
                 if (kr >= valid) q4 = make_uint4(0, 0, 0, 0);
                 *reinterpret_cast<uint4*>(dstA + kr * 128 + (((ja & 7) ^ (kr & 7)) << 4)) = q4;
             }
-#pragma unroll 2
+#pragma unroll 1
             for (int kr = gb; kr < rowsB; kr += groupsB) {
                 uint4 q4 = xv.apply(*reinterpret_cast<const uint4*>(raw + offX + (size_t)kr * rowB + (jb << 4)));
                 if (kr >= valid) q4 = make_uint4(0, 0, 0, 0);
