@@ -19,9 +19,9 @@
 //   warps 1-2     MMA issuers: each owns a share of the CTA's taps (disjoint accumulator columns) and
 //                 issues, for every 16 positions, one tcgen05.mma (M = 128 output channels, N = c_in)
 //                 per tap; every lane runs the loop, the elected lane issues
-//   warps 3-10    transform x in place (BatchNorm + activation), padding positions stay zero
-//   warps 11-18   transform dy in place into dz (BatchNorm-backward transform with z)
-//   warps 19-22   after the last tile: tcgen05.ld of the accumulators, float stores of the partial
+//   warps 3-6     transform x in place (BatchNorm + activation), padding positions stay zero
+//   warps 7-14    transform dy in place into dz (BatchNorm-backward transform with z)
+//   warps 15-18   after the last tile: tcgen05.ld of the accumulators, float stores of the partial
 //
 // Shared memory is zeroed once: rows of a slot that no copy ever writes (the tail up to a whole
 // number of 16-position steps, the rows the last taps read past the window) are multiplied by
@@ -37,7 +37,9 @@ namespace ast {
 namespace {
 
 using namespace tc;
-constexpr int WP_X_WARPS = 8, WP_D_WARPS = 8, WP_EPI_WARPS = 4, WP_MMA_WARPS = 2;
+// 19 warps: with more, the register allocation per thread drops below what the backward transform's coefficients need and
+// they spill into the hot loop
+constexpr int WP_X_WARPS = 4, WP_D_WARPS = 8, WP_EPI_WARPS = 4, WP_MMA_WARPS = 2;
 constexpr int WP_FIRST_X = 1 + WP_MMA_WARPS, WP_FIRST_D = WP_FIRST_X + WP_X_WARPS, WP_FIRST_EPI = WP_FIRST_D + WP_D_WARPS;
 constexpr int WP_THREADS = (WP_FIRST_EPI + WP_EPI_WARPS) * 32;
 constexpr int WP_MAX_S = 3;
@@ -171,6 +173,7 @@ conv3_wgrad_pipe_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
         const uint32_t leader = elect_leader();
         // D = f32, A = B = bf16, both MN-major (bits 15, 16); M = 128, N = c_in
         const uint32_t idesc = make_idesc(a.CI) | (1u << 15) | (1u << 16);
+        const uint32_t idesc2 = make_idesc(2 * a.CI) | (1u << 15) | (1u << 16);      // a pair of taps (64 input channels)
         // this warp's taps of the group: the first ceil(n/2) or the rest
         const int h = (t_count + 1) >> 1;
         const int tt0 = iss == 0 ? 0 : h, tt1 = iss == 0 ? h : t_count;
@@ -187,12 +190,25 @@ conv3_wgrad_pipe_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
             fence_after_sync();
             const uint32_t x0 = smem_u32(sSt + (size_t)s * a.stage_bytes);
             const uint32_t d0 = x0 + (uint32_t)kbi * a.x_block;
-            for (int tt = tt0; tt < tt1; ++tt) {
+            for (int tt = tt0; tt < tt1;) {
                 const int tp = t_first + tt, r = tp / 3, sx = tp - r * 3;
                 const uint32_t xs = x0 + (uint32_t)(r * Wp + sx) * 128u;
                 const uint32_t d = tmem + (uint32_t)(tt * a.CI);
-                for (int k = 0; k < a.ksteps; ++k)
-                    umma_bf16_lead(d, desc_mn(d0 + (uint32_t)k * 2048u, lbo_a), desc_mn(xs + (uint32_t)k * 2048u, lbo_b), idesc, (t > 0 || k > 0) ? 1u : 0u, leader);
+                if (kbi == 1 && tt + 1 < tt1) {
+                    // 64 input channels: two consecutive taps in one instruction of N = 128.  The second 64-column panel of the B
+                    // operand is the same x window moved by the distance between the two taps' row offsets (the
+                    // leading-dimension offset), its accumulator columns are the next tap's: half the instructions, and the A
+                    // operand is fetched from shared memory once for both taps.
+                    const uint32_t lbo_pair = (uint32_t)(sx < 2 ? 1 : Wp - 2) * 128u;
+                    for (int k = 0; k < a.ksteps; ++k)
+                        umma_bf16_lead(d, desc_mn(d0 + (uint32_t)k * 2048u, lbo_a), desc_mn(xs + (uint32_t)k * 2048u, lbo_pair), idesc2, (t > 0 || k > 0) ? 1u : 0u,
+                                       leader);
+                    tt += 2;
+                } else {
+                    for (int k = 0; k < a.ksteps; ++k)
+                        umma_bf16_lead(d, desc_mn(d0 + (uint32_t)k * 2048u, lbo_a), desc_mn(xs + (uint32_t)k * 2048u, lbo_b), idesc, (t > 0 || k > 0) ? 1u : 0u, leader);
+                    tt += 1;
+                }
             }
             umma_commit_lead(st_empty(s), leader);
             __syncwarp();
