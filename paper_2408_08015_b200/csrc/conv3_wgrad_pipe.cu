@@ -20,7 +20,8 @@
 //                 issues, for every 16 positions, one tcgen05.mma (M = 128 output channels, N = c_in)
 //                 per tap; every lane runs the loop, the elected lane issues
 //   warps 3-6     transform x in place (BatchNorm + activation), padding positions stay zero
-//   warps 7-14    transform dy in place into dz (BatchNorm-backward transform with z)
+//   warps 7-14    transform dy in place into dz (BatchNorm-backward transform with z); where only one operand needs a
+//                 transform all twelve warps work on it
 //   warps 15-18   after the last tile: tcgen05.ld of the accumulators, float stores of the partial
 //
 // Shared memory is zeroed once: rows of a slot that no copy ever writes (the tail up to a whole
@@ -113,7 +114,7 @@ conv3_wgrad_pipe_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(z_full(s), 1);
-            mbar_init(z_empty(s), WP_D_WARPS);
+            mbar_init(z_empty(s), a.xf_x ? WP_D_WARPS : WP_X_WARPS + WP_D_WARPS);
         }
         mbar_init(done, WP_MMA_WARPS);
         abort_store = 0;
@@ -216,10 +217,15 @@ conv3_wgrad_pipe_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_c
         if (ok) umma_commit_lead(done, leader);
     } else if (warp < WP_FIRST_EPI) {
         // ------------------------------------------------------------ transforms, in place
-        const bool is_x = warp < WP_FIRST_D;
+        // Split of the twelve transform warps: four on x and eight on dy when both operands need a transform, all twelve on
+        // the one that does when only one does (a stride-2 layer's zero-inserted gradient arrives already transformed)
+        const int wt = warp - WP_FIRST_X;
+        const bool both = a.xf_x && a.xf_d;
+        const bool is_x = both ? wt < WP_X_WARPS : a.xf_x != 0;
+        const int nrole = both ? (is_x ? WP_X_WARPS : WP_D_WARPS) : WP_X_WARPS + WP_D_WARPS;
         const int nblk = is_x ? kbi : kbo;                       // channel blocks of this operand
-        const int nw = (is_x ? WP_X_WARPS : WP_D_WARPS) / nblk;  // warps per block
-        const int wi = warp - (is_x ? WP_FIRST_X : WP_FIRST_D);
+        const int nw = nrole / nblk;                             // warps per block
+        const int wi = both && !is_x ? wt - WP_X_WARPS : wt;
         const int kb = wi / nw, wl = wi - kb * nw;               // this warp's block; its index among the block's warps
         const int j = lane & 7, pos0 = wl * 4 + (lane >> 3), npos = nw * 4;
         const bool need = is_x ? a.xf_x != 0 : a.xf_d != 0;
