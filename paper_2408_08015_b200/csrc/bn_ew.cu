@@ -18,7 +18,7 @@ struct StatsOp {
     template <typename T, int V> __device__ __forceinline__ void init(int c0, float (*ctx)[V]) const { ld_raw_w<T, V>(z, (size_t)c0, ctx[0]); }
     static constexpr int NLD = 1;                // tensors read per pixel
     template <typename T> __device__ __forceinline__ void load(size_t e, Vec<T>* r) const { r[0].load(z, e / Vec<T>::N); }
-    template <typename T, int V> __device__ __forceinline__ void acc_raw(const Vec<T>* r, const float (*ctx)[V], float (*a)[V]) const {
+    template <typename T, int V> __device__ __forceinline__ void acc_raw(size_t, const Vec<T>* r, const float (*ctx)[V], float (*a)[V]) const {
         float v[V];
         r[0].unpack(v);
         acc_vals<V>(v, ctx, a);
@@ -73,7 +73,7 @@ struct BwdOp {
         r[0].load(g.dy, e / Vec<T>::N);
         if (g.act != ACT_NONE || mean) r[1].load(g.z, e / Vec<T>::N);
     }
-    template <typename T, int V> __device__ __forceinline__ void acc_raw(const Vec<T>* r, const float (*ctx)[V], float (*a)[V]) const {
+    template <typename T, int V> __device__ __forceinline__ void acc_raw(size_t, const Vec<T>* r, const float (*ctx)[V], float (*a)[V]) const {
         float d[V], z[V];
         r[0].unpack(d);
         if (g.act != ACT_NONE || mean) r[1].unpack(z);
@@ -115,6 +115,54 @@ struct BwdOp {
     }
 };
 
+// Backward of a residual add followed by ReLU, fused with the BatchNorm-backward sums of the one operand branch that ends in
+// a BatchNorm without activation: dst = d * [out > 0] is stored, and its sums (of dst and of dst * xhat, xhat from the
+// branch's raw conv output z) are taken from the same registers.
+struct MaskBwdOp {
+    static constexpr int NACC = 2, NCTX = 2, NLD = 3;     // context: -mean*rstd, rstd
+    const void* d;        // gradient w.r.t. the ReLU's output
+    const void* out;      // the ReLU's output (its sign is the mask)
+    const void* z;        // raw conv output of the BatchNorm branch
+    void* dst;            // gradient w.r.t. the sum (and, by alias, w.r.t. both operands)
+    const float* mean;
+    const float* rstd;
+    template <typename T, int V> __device__ __forceinline__ void init(int c0, float (*ctx)[V]) const {
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            ctx[1][q] = __ldg(rstd + c0 + q);
+            ctx[0][q] = -__ldg(mean + c0 + q) * ctx[1][q];
+        }
+    }
+    template <typename T> __device__ __forceinline__ void load(size_t e, Vec<T>* r) const {
+        r[0].load(d, e / Vec<T>::N);
+        r[1].load(out, e / Vec<T>::N);
+        r[2].load(z, e / Vec<T>::N);
+    }
+    template <typename T, int V> __device__ __forceinline__ void acc_raw(size_t e, const Vec<T>* r, const float (*ctx)[V], float (*a)[V]) const {
+        float g[V], y[V], zz[V];
+        r[0].unpack(g);
+        r[1].unpack(y);
+        r[2].unpack(zz);
+#pragma unroll
+        for (int q = 0; q < V; ++q) g[q] = y[q] > 0.f ? g[q] : 0.f;
+        Vec<T> o;
+        o.pack(g);
+        o.store(dst, e / Vec<T>::N);
+        // the sums are of the gradient as stored (after rounding), like every other producer's
+        o.unpack(g);
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            a[0][q] += g[q];
+            a[1][q] = fmaf(g[q], fmaf(zz[q], ctx[1][q], ctx[0][q]), a[1][q]);
+        }
+    }
+    template <typename T, int V> __device__ __forceinline__ void acc(size_t e, const float (*ctx)[V], float (*a)[V]) const {
+        Vec<T> r[3];
+        load<T>(e, r);
+        acc_raw<T, V>(e, r, ctx, a);
+    }
+};
+
 template <typename T, int V, typename OP>
 __global__ void __launch_bounds__(512) chan_reduce_kernel(OP op, size_t pixels, int c, int cw, int rows, size_t pix_per_block,
                                                           float* __restrict__ partial) {
@@ -145,7 +193,7 @@ __global__ void __launch_bounds__(512) chan_reduce_kernel(OP op, size_t pixels, 
 #pragma unroll
                 for (int u = 0; u < U; ++u) op.template load<T>((p + (size_t)u * rows) * c + c0, r[u]);
 #pragma unroll
-                for (int u = 0; u < U; ++u) op.template acc_raw<T, V>(r[u], ctx, a);
+                for (int u = 0; u < U; ++u) op.template acc_raw<T, V>((p + (size_t)u * rows) * c + c0, r[u], ctx, a);
             }
         }
         for (; p < pend; p += rows) op.template acc<T, V>(p * c + c0, ctx, a);
@@ -593,6 +641,17 @@ void bn_bwd_reduce(int dtype, const void* dy, const void* z, size_t pixels, int 
     launch_reduce(dtype, p, op, pixels, c, scratch, K_BN_BWD_REDUCE, (double)pixels * c * esz(dtype) * ((act != ACT_NONE || mean) ? 2.0 : 1.0), st);
     LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
     launch_pdl(bn_bwd_finish, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
+}
+
+bool ew_relu_mask_bn_sums(int dtype, const void* d, const void* out_val, const void* z, size_t pixels, int c, const float* mean, const float* rstd,
+                          const float* gamma, void* dst, float* scratch, size_t scratch_floats, const BnBwdOut& o, cudaStream_t st) {
+    if (c % (dtype == 0 ? 4 : 8)) return false;          // whole vectors per thread (the op stores what it loads)
+    ReducePlan p = plan_reduce(dtype, pixels, c, 2, scratch_floats);
+    MaskBwdOp op{d, out_val, z, dst, mean, rstd};
+    launch_reduce(dtype, p, op, pixels, c, scratch, K_EW_MASK, (double)pixels * c * esz(dtype) * 4.0, st);
+    LaunchScope ls(K_BN_BWD_FINISH, 8.0 * c * (p.by + 4), 10.0 * c, st);
+    launch_pdl(bn_bwd_finish, (c + 31) / 32, 1024, 0, st, scratch, (int)p.by, c, (double)pixels, mean, rstd, gamma, o);
+    return true;
 }
 
 void bn_bwd_finish_partials(const float* partial, int blocks, size_t pixels, int c, const float* mean, const float* rstd, const float* gamma,

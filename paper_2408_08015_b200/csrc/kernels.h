@@ -173,6 +173,10 @@ void bn_bwd_finish_partials(const float* partial, int blocks, size_t pixels, int
 void ew_add(int dtype, const ValSrc& a, const ValSrc& b, int act, size_t pixels, int c, void* out, void* out2, cudaStream_t st);
 void ew_apply(int dtype, const ValSrc& a, size_t pixels, int c, void* out, cudaStream_t st);
 void ew_relu_mask(int dtype, const void* d, const void* out_val, size_t n, void* dst, cudaStream_t st);
+// the same, fused with the BatchNorm-backward sums (and finishing step) of the operand branch whose raw conv output is z and whose
+// BatchNorm has no activation: dst's sums are that BatchNorm's; false = channel count not a whole number of vectors, nothing launched
+bool ew_relu_mask_bn_sums(int dtype, const void* d, const void* out_val, const void* z, size_t pixels, int c, const float* mean, const float* rstd,
+                          const float* gamma, void* dst, float* scratch, size_t scratch_floats, const BnBwdOut& o, cudaStream_t st);
 void ew_sum(int dtype, const void* a, const void* b, size_t n, void* dst, cudaStream_t st);
 // bfloat16, channel counts multiples of 8: zero-inserted gradient / subsampled output of a stride-2 3x3 conv (see conv3_s2_tc_supported)
 void ew_upsample2_grad(const GradSrc& d, int n, int hi, int wi, int ho, int wo, int c, void* up, cudaStream_t st);

@@ -746,7 +746,31 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
         } else if (u.kind == U_ADD) {
             tick(s, ui, 4, st);
             if (u.act == ACT_RELU) {
-                ew_relu_mask(dt, go.ptr, sv.base + o.buf_off, o.elems, own(u.out), st);
+                // The masked gradient is the complete gradient of every operand used nowhere else.  If such an operand is
+                // the output of a conv -> BatchNorm unit without activation, the mask kernel also takes that BatchNorm's
+                // backward sums (one such operand: a second one keeps its own pass).
+                int tgt = -1;
+                for (int v : {u.in, u.in2}) {
+                    const Val& ov = s->vals[v];
+                    if (tgt >= 0 || ov.consumers != 1 || ov.unit < 0) continue;
+                    const Unit& q = s->units[ov.unit];
+                    if ((q.kind == U_CONV || q.kind == U_DW) && q.l_bn >= 0 && q.act == ACT_NONE && !reduced[ov.unit]) tgt = ov.unit;
+                }
+                bool fused = false;
+                if (tgt >= 0) {
+                    const Unit& tu = s->units[tgt];
+                    const Val& tv = s->vals[tu.out];
+                    float* ts = sv.stats + tv.stat_off;
+                    float* tk = s->coef + tu.k_off;
+                    BnBwdOut tbo{s->g + tu.gamma_off, s->g + tu.beta_off, tk, tk + tv.c, tk + 2 * (size_t)tv.c};
+                    fused = ew_relu_mask_bn_sums(dt, go.ptr, sv.base + o.buf_off, sv.base + tv.buf_off, o.elems / o.c, o.c, ts, ts + tv.c, s->w + tu.gamma_off,
+                                                 own(u.out), s->scratch, s->scratch_floats, tbo, st);
+                    if (fused) {
+                        reduced[tgt] = 1;
+                        s->bwd_sums_by[tgt] = ui;
+                    }
+                }
+                if (!fused) ew_relu_mask(dt, go.ptr, sv.base + o.buf_off, o.elems, own(u.out), st);
                 go.state = G_OWNED;
                 go.ptr = own(u.out);
             }
