@@ -133,6 +133,16 @@ int asteroid_stage_backward(asteroid_stage* s, int mb, const void* dy, void* dx,
 /* G += g_mb: accumulate the gradients of the micro-batch whose BP ran last (Section 3.2: each device
  * accumulates gradients for all micro-batches of the mini-batch).  AST_ERR_ORDER if mb is not that one. */
 int asteroid_stage_accumulate(asteroid_stage* s, int mb, void* stream);
+/* Accumulated-gradient arena of the stage, for the gradient synchronisation of a data-parallel device group
+ * (Section 3.2: the devices of a group hold replicas of the stage, each runs its share of every micro-batch and
+ * the gradients are synchronised with an AllReduce before the update; Eq. (5) counts its volume).  *G receives a
+ * DEVICE pointer to the float32 arena that asteroid_stage_accumulate adds into and asteroid_stage_step consumes,
+ * *n its length in floats (parameters in layer order, every layer starting at a multiple of 8 floats, the
+ * padding is zero).  The stage owns the memory; the pointer stays valid until asteroid_stage_destroy.  Between the
+ * last accumulate of a round and asteroid_stage_step a group member may scale the arena by its share of the
+ * micro-batch (y_d / B) and sum it over the group on the stream its stage calls use; the library itself does no
+ * communication.  AST_ERR_ARG for a null argument. */
+int asteroid_stage_grad_buffer(asteroid_stage* s, float** G, size_t* n);
 /* End of the HPP-Round (Section 3.2: accumulated gradients are applied to the stage parameters):
  * g = G/M; v = momentum*v + g; w = w - lr*v; G = 0; derived weight copies refreshed.
  * AST_ERR_ORDER unless exactly M micro-batches were accumulated since the last step. */

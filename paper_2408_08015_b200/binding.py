@@ -12,7 +12,7 @@ OP_CODES = {"conv": 0, "dwconv": 1, "bn": 2, "relu6": 3, "relu": 4, "add": 5, "g
 EXPORTS = ["asteroid_stage_create", "asteroid_stage_destroy", "asteroid_stage_param_count",
            "asteroid_stage_output_elems", "asteroid_stage_import_state", "asteroid_stage_export_state",
            "asteroid_stage_export_bn_running", "asteroid_stage_forward", "asteroid_stage_backward",
-           "asteroid_stage_accumulate", "asteroid_stage_step", "asteroid_stage_profile",
+           "asteroid_stage_accumulate", "asteroid_stage_step", "asteroid_stage_grad_buffer", "asteroid_stage_profile",
            "asteroid_loss_mse", "asteroid_loss_mse_noalloc", "asteroid_loss_softmax_xent", "asteroid_trace_start", "asteroid_trace_stop",
            "asteroid_selftest_bounded_wait", "asteroid_plan", "asteroid_launch_count", "asteroid_last_error"]
 
@@ -88,6 +88,7 @@ def lib():
         L.asteroid_stage_backward.argtypes = [vp, i, vp, vp, vp]
         L.asteroid_stage_accumulate.argtypes = [vp, i, vp]
         L.asteroid_stage_step.argtypes = [vp, f, f, vp]
+        L.asteroid_stage_grad_buffer.argtypes = [vp, C.POINTER(vp), C.POINTER(sz)]
         L.asteroid_stage_profile.argtypes = [vp, i, i, C.POINTER(ast_layer_profile)]
         L.asteroid_loss_mse.argtypes = [vp, vp, sz, i, vp, vp, vp]
         L.asteroid_loss_mse_noalloc.argtypes = [vp, vp, sz, i, vp, vp, vp]
@@ -143,6 +144,13 @@ def asteroid_stage_output_elems(h):
     a, b, c = C.c_int(), C.c_int(), C.c_int()
     n = lib().asteroid_stage_output_elems(h, C.byref(a), C.byref(b), C.byref(c))
     return n, (a.value, b.value, c.value)
+
+
+def asteroid_stage_grad_buffer(h):
+    """(device address, length in floats) of the stage's accumulated-gradient arena."""
+    g, n = C.c_void_p(), C.c_size_t()
+    _check(lib().asteroid_stage_grad_buffer(h, C.byref(g), C.byref(n)))
+    return g.value, n.value
 
 
 def asteroid_stage_import_state(h, params, momentum=None):

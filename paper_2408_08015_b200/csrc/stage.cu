@@ -928,6 +928,13 @@ size_t asteroid_stage_output_elems(const asteroid_stage* s, int* h, int* w, int*
     return o.elems;
 }
 
+int asteroid_stage_grad_buffer(asteroid_stage* s, float** G, size_t* n) {
+    if (!s || !G || !n) return fail(AST_ERR_ARG, "null argument");
+    *G = s->G;
+    *n = s->n_pad;
+    return AST_OK;
+}
+
 int asteroid_stage_import_state(asteroid_stage* s, const float* params, const float* momentum, size_t n) {
     if (!s || !params) return fail(AST_ERR_ARG, "null argument");
     if (n != s->n_params) return fail(AST_ERR_ARG, "state has %zu values, the stage has %zu parameters", n, s->n_params);
