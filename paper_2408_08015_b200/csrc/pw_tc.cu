@@ -12,6 +12,7 @@
 // (K and N are small), so a CTA holds one 128-pixel tile and several CTAs per SM overlap
 // their load, MMA and store phases.  Every wait is bounded and reports through an error word.
 #include <cuda_bf16.h>
+#include <string.h>
 
 #include "kernels.h"
 #include "tc_common.cuh"
@@ -1087,7 +1088,9 @@ struct WgArgs {
     float* partial;       // [ctas][CO][CI]
     float* gw;            // [CO][CI] (written by the split-sum kernel that follows)
     int* err;
-    int P, CO, CI;
+    int P, CO, CI;        // CO, CI: channels one CTA works on (a sub-range of a side that is split over blockIdx.y)
+    int COf, CIf;         // the layer's channel counts = row pitches of dy / z and of x, in elements
+    int nsa, nsb;         // channel sub-ranges per side; with more than one, the raw rows come by tiled tensor copies
     int pix_per_cta;      // multiple of WSTAGE
     int mtiles, ntiles, NT, tmem_cols;
     int pa, pb;           // 64-channel panels of the two operands per stage (pa even)
@@ -1096,7 +1099,8 @@ struct WgArgs {
     uint32_t raw_bytes, op_bytes;
 };
 
-__global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgArgs a) {
+__global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_z,
+                                                                      const __grid_constant__ CUtensorMap tm_x, const WgArgs a) {
     pdl_launch();             // barrier and tensor-memory set-up overlaps the previous kernel; the wait follows it
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * MAX_RAW + 5];    // raw_full[R], raw_empty[R], op_full[2], op_empty[2], done
@@ -1141,6 +1145,8 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
     const int stages = (pend - pbeg + WSTAGE - 1) / WSTAGE;
     const uint32_t rowA = (uint32_t)a.CO * 2u, rowB = (uint32_t)a.CI * 2u;
     const uint32_t offZ = WSTAGE * rowA, offX = offZ * (a.need_z ? 2u : 1u);
+    const bool split = a.nsa * a.nsb > 1;
+    const int coA = ((int)blockIdx.y % a.nsa) * a.CO, coB = ((int)blockIdx.y / a.nsa) * a.CI;     // first channel of this CTA's sub-ranges
 
     if (warp == 0) {
         if (lane == 0) {
@@ -1154,6 +1160,15 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
                 const int p0 = pbeg + it * WSTAGE;
                 const uint32_t valid = (uint32_t)min(WSTAGE, pend - p0);
                 uint8_t* dst = sR + (size_t)s * a.raw_bytes;
+                if (split) {
+                    // a channel sub-range of 64 pixel rows is not contiguous: one tiled copy per operand lands it as the same
+                    // dense rows (a box counts its full size; rows past the last pixel arrive as zeros)
+                    mbar_expect_tx(raw_full(s), (uint32_t)WSTAGE * (rowA * (a.need_z ? 2u : 1u) + rowB));
+                    tma::load_2d(smem_u32(dst), &tm_dy, coA, p0, raw_full(s));
+                    if (a.need_z) tma::load_2d(smem_u32(dst + offZ), &tm_z, coA, p0, raw_full(s));
+                    tma::load_2d(smem_u32(dst + offX), &tm_x, coB, p0, raw_full(s));
+                    continue;
+                }
                 mbar_expect_tx(raw_full(s), valid * (rowA * (a.need_z ? 2u : 1u) + rowB));
                 bulk_g2s(smem_u32(dst), gdy + (size_t)p0 * rowA, valid * rowA, raw_full(s));
                 if (a.need_z) bulk_g2s(smem_u32(dst + offZ), gz + (size_t)p0 * rowA, valid * rowA, raw_full(s));
@@ -1199,8 +1214,8 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
         const int rowsA = ga < groupsA ? WSTAGE : 0, rowsB = gb < groupsB ? WSTAGE : 0;
         XfGrad xg;
         XfVal xv;
-        xg.init(a.dz, ja << 3);
-        xv.init(a.x, jb << 3);
+        xg.init(a.dz, coA + (ja << 3));
+        xv.init(a.x, coB + (jb << 3));
         bool ok = true;
         for (int it = 0; it < stages; ++it) {
             const int st = a.OPS == 2 ? (it & 1) : 0, n = a.OPS == 2 ? (it >> 1) : it, s = it % R;
@@ -1243,7 +1258,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
         if (ok) {
             fence_after_sync();
             const int q = warp & 3, half = (warp - 2) >> 2;    // two warps share each lane quarter
-            float* pbase = a.partial + (size_t)blockIdx.x * a.CO * a.CI;
+            float* pbase = a.partial + (size_t)blockIdx.x * a.COf * a.CIf + (size_t)coA * a.CIf + coB;
             for (int mt = 0; mt < a.mtiles; ++mt) {
                 const int k = mt * TM + q * 32 + lane;
                 for (int nt = 0; nt < a.ntiles; ++nt)
@@ -1260,7 +1275,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) pw_wgrad_pipe_kernel(const WgAr
 #pragma unroll
                             for (int hh = 0; hh < 4; ++hh)
                                 if (c + hh * 4 < a.CI)
-                                    *reinterpret_cast<float4*>(pbase + (size_t)k * a.CI + c + hh * 4) = make_float4(v[hh * 4], v[hh * 4 + 1], v[hh * 4 + 2], v[hh * 4 + 3]);
+                                    *reinterpret_cast<float4*>(pbase + (size_t)k * a.CIf + c + hh * 4) = make_float4(v[hh * 4], v[hh * 4 + 1], v[hh * 4 + 2], v[hh * 4 + 3]);
                         }
                     }
             }
@@ -1302,7 +1317,13 @@ __global__ void __launch_bounds__(1024) reduce_splits_2d(const float* __restrict
     }
 }
 
+// Plans the kernel for a.nsa x a.nsb channel sub-ranges of the layer's a.COf x a.CIf weight gradient.
 bool plan_wgrad(WgArgs& a, size_t* smem, size_t scratch_floats, int n_sm) {
+    if (a.COf % a.nsa || a.CIf % a.nsb) return false;
+    a.CO = a.COf / a.nsa;
+    a.CI = a.CIf / a.nsb;
+    const int ns = a.nsa * a.nsb;
+    if (ns > 1 && (a.CO % 64 || a.CI % 64 || a.CO > 256 || a.CI > 256)) return false;     // box of a tiled copy: at most 256 elements wide
     if (a.CO > 512 || a.CI > 512 || (a.CO + a.CI) / 8 > 256) return false;
     a.ntiles = (a.CI + 255) / 256;
     a.NT = ((a.CI + a.ntiles - 1) / a.ntiles + 63) / 64 * 64;      // whole panels per N tile
@@ -1318,7 +1339,7 @@ bool plan_wgrad(WgArgs& a, size_t* smem, size_t scratch_floats, int n_sm) {
     size_t rb = (size_t)WSTAGE * (a.CO * 2 * (a.need_z ? 2 : 1) + a.CI * 2);
     rb = (rb + 127) / 128 * 128;
     a.raw_bytes = (uint32_t)rb;
-    const size_t budget = 220 * 1024 - 1024;
+    const size_t budget = 226 * 1024 - 1024;
     a.OPS = 2 * (size_t)a.op_bytes + 2 * rb <= budget ? 2 : 1;
     const size_t fixed = (size_t)a.OPS * a.op_bytes;
     if (fixed + 2 * rb > budget) return false;
@@ -1326,8 +1347,8 @@ bool plan_wgrad(WgArgs& a, size_t* smem, size_t scratch_floats, int n_sm) {
     if (r > 4) r = 4;
     a.R = (int)r;
     *smem = fixed + r * rb + 1024;
-    size_t out_elems = (size_t)a.CO * a.CI;
-    int ctas = n_sm;
+    size_t out_elems = (size_t)a.COf * a.CIf;
+    int ctas = n_sm / ns;                       // pixel ranges; every range is worked on by one CTA per pair of sub-ranges
     int max_by_pix = (a.P + 2 * WSTAGE - 1) / (2 * WSTAGE);
     if (ctas > max_by_pix) ctas = max_by_pix;
     size_t cap = scratch_floats / out_elems;
@@ -1398,7 +1419,10 @@ int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const
         if (plan_pipe(pa, &smem) && make_out_map(z, pa.P, pa.N, &tm_out)) return launch_pipe<false>(pa, tm_out, smem, K_PW_FWD_TC, bytes, partial_floats, st);
     }
     // more than 256 channels on a side: the streaming kernel, where the layer fits it
-    if (g.stride == 1 && !bias && pw_stream(false, a.P, a.K, a.N, x, GradSrc{}, wb, nullptr, z, err, K_PW_FWD_TC, bytes, st)) return 0;
+    int stat_blocks = 0;
+    if (g.stride == 1 && !bias &&
+        pw_stream(false, a.P, a.K, a.N, x, GradSrc{}, wb, nullptr, z, err, K_PW_FWD_TC, bytes, st, pivot, partial, partial_floats, &stat_blocks))
+        return stat_blocks;
     Tiling t = pick_tiling(a.K, a.N);
     launch<false>(a, t, K_PW_FWD_TC, bytes, st);
     return 0;
@@ -1449,23 +1473,44 @@ int pw_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wt
 void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, float* scratch, size_t scratch_floats, float* gw, int* err,
                       cudaStream_t st) {
     if (g.stride == 1) {
-        smem_limit_once<104>(pw_wgrad_pipe_kernel, 222 * 1024);
+        smem_limit_once<104>(pw_wgrad_pipe_kernel, 226 * 1024);
         const int n_sm = sm_count();
         WgArgs wa{};
         wa.dz = dz; wa.x = x; wa.partial = scratch; wa.gw = gw; wa.err = err;
-        wa.P = g.n * g.ho * g.wo; wa.CO = g.co; wa.CI = g.ci;
+        wa.P = g.n * g.ho * g.wo; wa.COf = g.co; wa.CIf = g.ci;
         wa.need_z = (dz.act != ACT_NONE || dz.k1) ? 1 : 0;
         size_t smem = 0;
-        if (plan_wgrad(wa, &smem, scratch_floats, n_sm)) {
+        // the whole gradient in one CTA's tensor memory where its stages fit; else the wider side in 2 or 4 channel sub-ranges
+        // (the other side's rows are then read once per sub-range, by CTAs that run side by side: a re-read from L2)
+        static const int kSplits[3][2] = {{1, 1}, {4, 1}, {2, 1}};
+        bool planned = false;
+        for (int i = 0; i < 3 && !planned; ++i) {
+            wa.nsa = g.co >= g.ci ? kSplits[i][0] : kSplits[i][1];
+            wa.nsb = g.co >= g.ci ? kSplits[i][1] : kSplits[i][0];
+            planned = plan_wgrad(wa, &smem, scratch_floats, n_sm);
+        }
+        alignas(64) CUtensorMap tm_dy, tm_z, tm_x;
+        memset(&tm_dy, 0, sizeof(tm_dy)); memset(&tm_z, 0, sizeof(tm_z)); memset(&tm_x, 0, sizeof(tm_x));
+        if (planned && wa.nsa * wa.nsb > 1) {
+            const uint64_t da[2] = {(uint64_t)wa.COf, (uint64_t)wa.P}, db[2] = {(uint64_t)wa.CIf, (uint64_t)wa.P};
+            const uint64_t sa[1] = {(uint64_t)wa.COf * 2}, sb[1] = {(uint64_t)wa.CIf * 2};
+            const uint32_t ba[2] = {(uint32_t)wa.CO, (uint32_t)WSTAGE}, bb[2] = {(uint32_t)wa.CI, (uint32_t)WSTAGE};
+            planned = tma::encode_bf16(&tm_dy, dz.dy, 2, da, sa, ba, false) && (!wa.need_z || tma::encode_bf16(&tm_z, dz.z, 2, da, sa, ba, false)) &&
+                      tma::encode_bf16(&tm_x, x.p, 2, db, sb, bb, false);
+        }
+        if (planned) {
             int ctas = (wa.P + wa.pix_per_cta - 1) / wa.pix_per_cta;
-            double bytes = 2.0 * (double)wa.P * wa.CO * (wa.need_z ? 2.0 : 1.0) + 2.0 * (double)wa.P * wa.CI + 4.0 * wa.CO * wa.CI * (2.0 * ctas + 1);
+            double bytes = 2.0 * (double)wa.P * wa.COf * (wa.need_z ? 2.0 : 1.0) + 2.0 * (double)wa.P * wa.CIf + 4.0 * wa.COf * wa.CIf * (2.0 * ctas + 1);
             {
-                LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * wa.P * wa.CO * wa.CI, st);
-                launch_pdl(pw_wgrad_pipe_kernel, ctas, WG_THREADS, smem, st, wa);
+                LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * wa.P * wa.COf * wa.CIf, st);
+                launch_pdl(pw_wgrad_pipe_kernel, dim3(ctas, wa.nsa * wa.nsb), WG_THREADS, smem, st, tm_dy, tm_z, tm_x, wa);
             }
-            size_t out_elems = (size_t)wa.CO * wa.CI;
+            size_t out_elems = (size_t)wa.COf * wa.CIf;
             LaunchScope ls(K_REDUCE_SPLITS, 4.0 * out_elems * (ctas + 1), (double)out_elems * ctas, st);
-            launch_pdl(reduce_splits_2d, (unsigned)((out_elems + 31) / 32), 1024, 0, st, scratch, ctas, out_elems, gw);
+            if (out_elems % 4 == 0 && (reinterpret_cast<uintptr_t>(scratch) | reinterpret_cast<uintptr_t>(gw)) % 16 == 0)
+                reduce_splits_f4(scratch, ctas, out_elems, gw, st);
+            else
+                launch_pdl(reduce_splits_2d, (unsigned)((out_elems + 31) / 32), 1024, 0, st, scratch, ctas, out_elems, gw);
             return;
         }
     }

@@ -1,9 +1,10 @@
 // Tiled bulk tensor copies (cp.async.bulk.tensor): host-side tensor-map encoding through the
 // driver entry point (no link-time dependency on the driver library) and the device-side copy
-// instructions.  Every map uses the 128-byte swizzle, so that a box whose innermost extent is
+// instructions.  Maps use the 128-byte swizzle unless asked otherwise, so that a box whose innermost extent is
 // 64 bf16 elements lands in shared memory as rows of 128 bytes in exactly the layout the tcgen05
 // shared-memory descriptors of tc_common.cuh read (16-byte chunk j of row r at chunk position
-// j ^ (r & 7), groups of 8 rows 1024 bytes apart).  Coordinates outside the tensor read zeros.
+// j ^ (r & 7), groups of 8 rows 1024 bytes apart).  A map without swizzle lands its box as dense
+// rows (innermost extent up to 256 elements).  Coordinates outside the tensor read zeros.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -27,8 +28,9 @@ inline EncodeTiledFn encode_fn() {
 
 // bf16 tensor of `rank` dimensions, innermost first: dims[i] elements, strides[i] bytes between
 // consecutive indices of dimension i+1 (rank-1 entries, multiples of 16), box[i] elements copied
-// per dimension (box[0] * 2 bytes = 128).  Returns false if the driver refuses the description.
-inline bool encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides, const uint32_t* box) {
+// per dimension (box[0] * 2 bytes = 128 with the swizzle).  Returns false if the driver refuses the description.
+inline bool encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides, const uint32_t* box,
+                        bool swizzle = true) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t gd[5], gs[4];
@@ -40,7 +42,7 @@ inline bool encode_bf16(CUtensorMap* map, const void* base, int rank, const uint
     }
     for (int i = 0; i + 1 < rank; ++i) gs[i] = strides[i];
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 #ifdef __CUDACC__
