@@ -746,6 +746,10 @@ __global__ void __launch_bounds__(1024) reduce_splits_c3(const float* __restrict
 
 }  // namespace
 
+void reduce_splits_f4(const float* partial, int splits, size_t n, float* out, cudaStream_t st) {
+    launch_pdl(reduce_splits_c3, (unsigned)((n / 4 + 31) / 32), 1024, 0, st, partial, splits, n, out);
+}
+
 bool conv3_tc_supported(int dtype, const ConvGeom& g) {
     if (!(dtype == 1 && g.k == 3 && g.stride == 1 && g.pad == 1)) return false;
     if (g.ci % 64 || g.co % 64 || g.ci > 256 || g.co > 256) return false;

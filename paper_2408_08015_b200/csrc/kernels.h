@@ -123,6 +123,8 @@ bool conv3_tc_supported(int dtype, const ConvGeom& g);
 void conv3_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, void* z, int* err, cudaStream_t st, double useful_flops = 0);
 void conv3_bwd_data_tc(const ConvGeom& g, const GradSrc& dz, const __nv_bfloat16* wtb, const void* addend, void* dx, int* err, cudaStream_t st,
                        double useful_flops = 0);
+// out[i] = sum over k < splits of partial[k][i] in a fixed order; n a multiple of 4, both pointers 16-byte aligned (conv3_tc.cu)
+void reduce_splits_f4(const float* partial, int splits, size_t n, float* out, cudaStream_t st);
 // pipelined form (conv3_pipe.cu) for up to 128 reduction channels: forward (bwd == false: x, w = [c_out][9][c_in], C = c_in,
 // N = c_out) or backward-data (bwd == true: dz, w = [c_in][9][c_out], C = c_out, N = c_in); false = layer does not fit, nothing launched
 bool conv3_pipe(bool bwd, int n_img, int H, int W, int C, int N, const ValSrc& x, const GradSrc& dz, const __nv_bfloat16* w, const void* addend,

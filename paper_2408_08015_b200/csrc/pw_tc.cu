@@ -1419,10 +1419,7 @@ int pw_fwd_tc(const ConvGeom& g, const ValSrc& x, const __nv_bfloat16* wb, const
         if (plan_pipe(pa, &smem) && make_out_map(z, pa.P, pa.N, &tm_out)) return launch_pipe<false>(pa, tm_out, smem, K_PW_FWD_TC, bytes, partial_floats, st);
     }
     // more than 256 channels on a side: the streaming kernel, where the layer fits it
-    int stat_blocks = 0;
-    if (g.stride == 1 && !bias &&
-        pw_stream(false, a.P, a.K, a.N, x, GradSrc{}, wb, nullptr, z, err, K_PW_FWD_TC, bytes, st, pivot, partial, partial_floats, &stat_blocks))
-        return stat_blocks;
+    if (g.stride == 1 && !bias && pw_stream(false, a.P, a.K, a.N, x, GradSrc{}, wb, nullptr, z, err, K_PW_FWD_TC, bytes, st)) return 0;
     Tiling t = pick_tiling(a.K, a.N);
     launch<false>(a, t, K_PW_FWD_TC, bytes, st);
     return 0;
