@@ -829,7 +829,7 @@ void conv3_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, 
     size_t smem = 2 * (size_t)TM * 128 + (size_t)(a.CI / 64) * a.rows_pad * 128 + 1024;
     double px = (double)g.n * g.hi * g.wi;
     {
-        LaunchScope ls(K_CONV3_BWD_WEIGHT_TC, 2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci + 4.0 * out_elems * ctas,
+        LaunchScope ls(K_CONV3_BWD_WEIGHT_TC, 2.0 * px * g.co * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * px * g.ci + 4.0 * out_elems,
                        useful_flops > 0 ? useful_flops : 2.0 * 9.0 * px * g.ci * g.co, st);
         launch_pdl(conv3_wgrad_tc_kernel, dim3(ctas, groups), C3_THREADS, smem, st, a);
     }

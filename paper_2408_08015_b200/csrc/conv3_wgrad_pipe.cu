@@ -370,7 +370,8 @@ int conv3_wgrad_pipe(int n_img, int H, int W, int CI, int CO, const GradSrc& dz,
         if (!tma::encode_bf16(&mz, p.xf_d ? dz.z : dz.dy, 4, dd, sd, bd)) return 0;
     }
     smem_limit_once<122>(conv3_wgrad_pipe_kernel, 226 * 1024);
-    LaunchScope ls(K_CONV3_BWD_WEIGHT_TC, bytes + 4.0 * out_elems * ctas, flops, st);
+    // recorded bytes: the operands once and the gradient once; the per-CTA partials are the split-sum kernel's traffic
+    LaunchScope ls(K_CONV3_BWD_WEIGHT_TC, bytes + 4.0 * out_elems, flops, st);
     launch_pdl(conv3_wgrad_pipe_kernel, dim3(ctas, groups), WP_THREADS, (size_t)p.smem_bytes + 1024, st, mx, md, mz, p);
     return ctas;
 }

@@ -1113,7 +1113,7 @@ void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc
         const size_t ipb = (n_items + by - 1) / by;
         by = (n_items + ipb - 1) / ipb;
         dim3 grid(gx, (unsigned)by);
-        LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
+        LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci, 18.0 * out_e, st);
         constexpr int NL = TWR + 2 + 2 * TWR;
         if (dtype == 0) {
             constexpr int D = 2;
@@ -1135,7 +1135,7 @@ void dw_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc
         by = (n_items + ipb - 1) / ipb;
         const size_t smem = (size_t)rows * cw * V * sizeof(float);
         dim3 grid(gx, (unsigned)by);
-        LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci * by, 18.0 * out_e, st);
+        LaunchScope ls(K_DW_BWD_WEIGHT, grad_src_bytes(dz, out_e, dtype) + in_e * esz(dtype) + 36.0 * g.ci, 18.0 * out_e, st);
         if (dtype == 0) launch_pdl(dw_wgrad_s2_kernel<float, 4, TWR>, grid, 128, smem, st, g, dz, x, cw, rows, th, ipb, scratch);
         else launch_pdl(dw_wgrad_s2_kernel<__nv_bfloat16, 4, TWR>, grid, 128, smem, st, g, dz, x, cw, rows, th, ipb, scratch);
     }
@@ -1169,7 +1169,7 @@ bool dw_bwd_fused(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSrc&
     smem_limit_once<202 + V * 10000 + TWR * 1000 + D * 100>(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, false>, 96 * 1024);
     double e = (double)g.n * g.hi * g.wi * g.ci;
     {
-        LaunchScope ls(K_DW_BWD_FUSED, grad_src_bytes(dz, e, dtype) + e * 2.0 * (addend ? 3.0 : 2.0) + 36.0 * g.ci * (by + 1), 36.0 * e, st);
+        LaunchScope ls(K_DW_BWD_FUSED, grad_src_bytes(dz, e, dtype) + e * 2.0 * (addend ? 3.0 : 2.0) + 36.0 * g.ci, 36.0 * e, st);
         dim3 grid(gx, (unsigned)by);
         if (addend) launch_pdl(dw_bwd_fused_kernel<__nv_bfloat16, V, TWR, D, true>, grid, 128, smem, st, g, dz, x, w9c, (const __nv_bfloat16*)addend, (__nv_bfloat16*)dx, cw,
                                                                             rows, ipb, scratch);

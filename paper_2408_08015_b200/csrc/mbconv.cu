@@ -735,7 +735,7 @@ void dwk_bwd_weight(int dtype, const ConvGeom& g, const GradSrc& dz, const ValSr
         if (want < 1) want = 1;
         const size_t spb = (total + want - 1) / want;
         by = (int)((total + spb - 1) / spb);
-        LaunchScope ls(K_DW_BWD_WEIGHT, ((double)out_e * (grad_needs_z(dz) ? 2 : 1) + in_e) * esz_(dtype) + 4.0 * taps * g.ci * by, 2.0 * taps * out_e, st);
+        LaunchScope ls(K_DW_BWD_WEIGHT, ((double)out_e * (grad_needs_z(dz) ? 2 : 1) + in_e) * esz_(dtype) + 4.0 * taps * g.ci, 2.0 * taps * out_e, st);
         if (g.stride == 1) launch_pdl(dwk_bwd_weight_kernel<T, V, K, 1, TW>, dim3(gx, by), 128, 0, st, g, dz, x, strips, spb, scratch);
         else launch_pdl(dwk_bwd_weight_kernel<T, V, K, 2, TW>, dim3(gx, by), 128, 0, st, g, dz, x, strips, spb, scratch);
     }););

@@ -1497,7 +1497,7 @@ void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, flo
         }
         if (planned) {
             int ctas = (wa.P + wa.pix_per_cta - 1) / wa.pix_per_cta;
-            double bytes = 2.0 * (double)wa.P * wa.COf * (wa.need_z ? 2.0 : 1.0) + 2.0 * (double)wa.P * wa.CIf + 4.0 * wa.COf * wa.CIf * (2.0 * ctas + 1);
+            double bytes = 2.0 * (double)wa.P * wa.COf * (wa.need_z ? 2.0 : 1.0) + 2.0 * (double)wa.P * wa.CIf + 4.0 * wa.COf * wa.CIf;   // operands and gradient once: partials belong to the split sum
             {
                 LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * wa.P * wa.COf * wa.CIf, st);
                 launch_pdl(pw_wgrad_pipe_kernel, dim3(ctas, wa.nsa * wa.nsb), WG_THREADS, smem, st, tm_dy, tm_z, tm_x, wa);
@@ -1535,7 +1535,7 @@ void pw_bwd_weight_tc(const ConvGeom& g, const GradSrc& dz, const ValSrc& x, flo
     size_t smem = (size_t)2 * (2 + (a.NT + 63) / 64) * PANEL + 1024;
     smem_limit_once<105>(pw_bwd_weight_tc_kernel, 200 * 1024);
     double bytes = 2.0 * (double)a.P * a.CO * ((dz.act != ACT_NONE || dz.k1) ? 2.0 : 1.0) + 2.0 * (double)g.n * g.hi * g.wi * a.CI +
-                   4.0 * out_elems * splits;
+                   4.0 * out_elems;
     {
         LaunchScope ls(K_PW_BWD_WEIGHT_TC, bytes, 2.0 * a.P * a.CO * a.CI, st);
         launch_pdl(pw_bwd_weight_tc_kernel, dim3(mtiles, splits, ntiles), NTHREADS, smem, st, a);
