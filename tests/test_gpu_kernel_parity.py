@@ -32,6 +32,10 @@ CASES = {
     "pw_512_128": (si.single_unit_net("conv", 512, 128), 29, 27, 3, 1, "mse", PW),
     "pw_512_128_bn": (si.single_unit_net("conv", 512, 128, bn=True), 29, 27, 3, 1, "mse", PW),
     "pw_320_1280_bn": (si.single_unit_net("conv", 320, 1280, bn=True), 7, 7, 5, 1, "mse", PW),
+    # weight gradient on channel sub-ranges with the BatchNorm-backward transform on the wide side: four sub-ranges of 128
+    # (512 channels), two of 192 (384 channels, where a quarter is no multiple of 64)
+    "pw_128_512_bn": (si.single_unit_net("conv", 128, 512, bn=True), 29, 27, 3, 1, "mse", PW),
+    "pw_128_384_bn": (si.single_unit_net("conv", 128, 384, bn=True), 23, 21, 3, 1, "mse", PW),
     # strided 1x1 (projection shortcut) on an odd-sized map
     "pw_s2_64_128": (si.single_unit_net("conv", 64, 128, stride=2), 13, 11, 3, 2, "mse", PW),
     "pw_s2_256_512_bn": (si.single_unit_net("conv", 256, 512, stride=2, bn=True), 13, 11, 3, 1, "mse", PW),
