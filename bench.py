@@ -264,7 +264,7 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
 
-    def one_round(s):
+    def one_round(s, sp=sp):
         for m in range(Mn):
             P.asteroid_stage_forward(hdl, m, s["x"][m].data_ptr(), s["y"][m].data_ptr(), sp)
             lp = s["loss"].data_ptr() + 4 * m
@@ -323,8 +323,32 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
     warm = max(args.warmup, 3)
     for _ in range(warm):
         one_round(sets[0])
+    # The device-timed steps replay one captured CUDA graph of the round (the stage calls only enqueue: the same kernels, in
+    # the same order, on the same two streams, without the per-launch submission cost).  If the capture is refused the steps
+    # are issued call by call, on a fresh stage (a capture that stopped half-way leaves the stage's bookkeeping mid-round).
+    run_round, launch_mode, launches_per_round = (lambda: one_round(sets[0])), "call by call", None
+    if not args.no_graph:
+        torch.cuda.synchronize()
+        try:
+            n_cap = P.asteroid_launch_count()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, capture_error_mode="thread_local"):
+                one_round(sets[0], torch.cuda.current_stream().cuda_stream)
+            launches_per_round = P.asteroid_launch_count() - n_cap
+            for _ in range(2):
+                graph.replay()
+            torch.cuda.synchronize()
+            run_round, launch_mode = graph.replay, "one captured CUDA graph of the round, replayed"
+        except Exception as exc:                                     # noqa: BLE001 (any refusal means: no graph)
+            sys.stderr.write("graph capture refused (%s): steps issued call by call\n" % (str(exc).splitlines() or [""])[0])
+            torch.cuda.synchronize()
+            P.asteroid_stage_destroy(hdl)
+            hdl = P.asteroid_stage_create(wl.net, wl.first, wl.last, wl.H, wl.W, Bn, Mn, dtype=adt, need_input_grad=wl.need_dx)
+            P.asteroid_stage_import_state(hdl, np.ascontiguousarray(params))
+            for _ in range(warm):
+                one_round(sets[0])
     # repeats: the timed region lasts about MIN_TIMED_S (every rank takes the same count: it comes from rank 0's probe)
-    probe = timed(lambda: one_round(sets[0]), 2) / 2
+    probe = timed(run_round, 2) / 2
     rep = max(1, int(np.ceil(args.min_seconds * 1e3 / max(probe * args.steps, 1e-3))))
     if dist is not None:
         t = torch.tensor([rep], device=dev)
@@ -337,8 +361,8 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
         gpu_id = str(dev.index)
     sampler = ClockSampler(gpu_id)
     n0 = P.asteroid_launch_count()
-    ms = timed(lambda: one_round(sets[0]), steps_timed)
-    launches = P.asteroid_launch_count() - n0
+    ms = timed(run_round, steps_timed)
+    launches = P.asteroid_launch_count() - n0 if launches_per_round is None else launches_per_round * steps_timed
     clocks = sampler.stop()
 
     def e2e_timed(steps):
@@ -401,7 +425,7 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
             "warmup": warm, "ms_per_step": ms / steps_timed, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
             "config": {"workload": wl.name, "samples_per_step_per_gpu": Bn * Mn, "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "steps_timed": steps_timed,
+                       "steps_timed": steps_timed, "launch": launch_mode,
                        "timed_region": "%d x %d steps so that it lasts about %.0f s; ms_per_step is their mean" % (rep, args.steps, args.min_seconds),
                        "l2": ("no flush: each step streams its activation slots and gradients, far beyond the 126 MB L2" if wl.cfg != 1 else
                               "no flush and smaller than L2: a step touches about 30 MB, so this workload is launch- and latency-bound by construction")},
@@ -454,6 +478,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="all", choices=["1", "2", "3", "4", "6", "all"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="issue the device-timed steps call by call instead of replaying a captured graph")
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
                     help="the K timed steps are repeated until the timed region lasts about this long (0: exactly K steps)")
     args = ap.parse_args()
