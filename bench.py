@@ -298,7 +298,10 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
                 s["t"][m].copy_(ht[m], non_blocking=True)
             copied[b].record(h2d)
         stream.wait_event(copied[b])
-        one_round(s)
+        if graphs[b] is not None:
+            graphs[b].replay()                   # the same round, captured once per buffer set
+        else:
+            one_round(s)
         computed[b].record(stream)
         d2h.wait_event(computed[b])
         with torch.cuda.stream(d2h):
@@ -327,19 +330,25 @@ def bench_config(wl, args, torch, P, dist, dev, rank, world):
     # the same order, on the same two streams, without the per-launch submission cost).  If the capture is refused the steps
     # are issued call by call, on a fresh stage (a capture that stopped half-way leaves the stage's bookkeeping mid-round).
     run_round, launch_mode, launches_per_round = (lambda: one_round(sets[0])), "call by call", None
+    graphs = [None, None]                         # one per device buffer set (the end-to-end leg alternates between the two)
     if not args.no_graph:
         torch.cuda.synchronize()
         try:
-            n_cap = P.asteroid_launch_count()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, capture_error_mode="thread_local"):
-                one_round(sets[0], torch.cuda.current_stream().cuda_stream)
-            launches_per_round = P.asteroid_launch_count() - n_cap
+            made = []
+            for b in range(2):
+                n_cap = P.asteroid_launch_count()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, capture_error_mode="thread_local"):
+                    one_round(sets[b], torch.cuda.current_stream().cuda_stream)
+                launches_per_round = P.asteroid_launch_count() - n_cap
+                made.append(graph)
             for _ in range(2):
-                graph.replay()
+                made[0].replay()
             torch.cuda.synchronize()
-            run_round, launch_mode = graph.replay, "one captured CUDA graph of the round, replayed"
+            graphs = made
+            run_round, launch_mode = graphs[0].replay, "one captured CUDA graph of the round, replayed"
         except Exception as exc:                                     # noqa: BLE001 (any refusal means: no graph)
+            launches_per_round = None
             sys.stderr.write("graph capture refused (%s): steps issued call by call\n" % (str(exc).splitlines() or [""])[0])
             torch.cuda.synchronize()
             P.asteroid_stage_destroy(hdl)
