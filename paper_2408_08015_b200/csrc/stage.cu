@@ -65,6 +65,7 @@ struct Unit {
     // over an explicit im2col tensor kept in the slot (col_kp = padded reduction length, 0 = not such a unit)
     int col_kp = 0;
     size_t col_off = 0;     // bytes into a slot
+    long sub_off = -1;      // bytes into a slot: the input of a stride-2 1x1 conv sampled at the positions the conv reads
     size_t wpad_off = 0;    // elements into the padded bf16 weight arena
     // stride-2 3x3 conv on the stride-1 tensor-core kernels: bytes into the arena of zero-inserted output gradients (one
     // buffer per such unit: the weight-gradient kernel reads it on the second stream while the pass goes on), -1 = none
@@ -344,6 +345,15 @@ static int build_plan(asteroid_stage* s) {
             s->n_gpad = std::max(s->n_gpad, (size_t)u.g.co * u.col_kp);
         }
     }
+    // A 1x1 conv with stride 2 reads one input position in four: the forward copies those positions into a dense tensor kept
+    // in the slot, and the forward and the weight gradient then run the stride-1 pointwise pipelines on it.
+    for (auto& u : s->units) {
+        if (u.kind == U_CONV && s->dtype == AST_BF16 && u.g.k == 1 && u.g.stride == 2 && u.g.pad == 0 && u.g.ci % 8 == 0 && u.g.co % 8 == 0 &&
+            u.b_off < 0 && !u.col_kp) {
+            u.sub_off = (long)sb;
+            sb += align_up((size_t)u.g.n * u.g.ho * u.g.wo * u.g.ci * 2, 256);
+        }
+    }
     s->slot_stat_off = sb;
     for (auto& u : s->units) {
         if (u.l_bn >= 0) {
@@ -482,6 +492,12 @@ static bool conv3_s2_tc_supported(const asteroid_stage* s, const Unit& u) {
 static double conv_flops(const ConvGeom& g) { return 2.0 * g.n * g.ho * g.wo * (double)g.co * g.k * g.k * g.ci; }
 
 // geometry of the pointwise GEMM that stands for an im2col unit
+// stride-2 1x1 conv on its subsampled input: a stride-1 conv over the output grid
+static ConvGeom sub_geom(const Unit& u) {
+    ConvGeom g = u.g;
+    g.hi = u.g.ho; g.wi = u.g.wo; g.stride = 1;
+    return g;
+}
 static ConvGeom col_geom(const Unit& u) {
     ConvGeom g = u.g;
     g.hi = u.g.ho; g.wi = u.g.wo; g.ci = u.col_kp; g.k = 1; g.stride = 1; g.pad = 0;
@@ -538,6 +554,13 @@ static int forward_impl(asteroid_stage* s, int slot, const void* x, void* y, cud
                 conv_im2col(u.g, val_src(s, sv, u.in), u.col_kp, col, st);
                 fused_stats = pw_fwd_tc(col_geom(u), ValSrc{col, nullptr, nullptr, ACT_NONE}, s->wpad + u.wpad_off, nullptr, obuf,
                                         bn ? s->run + u.run_off : nullptr, bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
+            } else if (u.sub_off >= 0) {
+                ValSrc xs = val_src(s, sv, u.in);
+                void* sub = sv.base + u.sub_off;
+                ew_subsample2(xs.p, u.g.n, u.g.hi, u.g.wi, u.g.ho, u.g.wo, u.g.ci, sub, st);
+                xs.p = sub;                                  // the producer's BatchNorm / activation is per channel: applied on load as before
+                fused_stats = pw_fwd_tc(sub_geom(u), xs, s->wb + u.w_off, bias, obuf, bn ? s->run + u.run_off : nullptr,
+                                        bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
             } else if (pw_tc_supported(dt, u.g, false))
                 fused_stats = pw_fwd_tc(u.g, val_src(s, sv, u.in), s->wb + u.w_off, bias, obuf, bn ? s->run + u.run_off : nullptr,
                                         bn ? s->scratch : nullptr, s->scratch_floats, s->err, st);
@@ -703,6 +726,10 @@ static int backward_impl(asteroid_stage* s, int slot, const void* dy, void* dx, 
             else if (u.kind == U_CONV && u.col_kp) {
                 pw_bwd_weight_tc(col_geom(u), d, ValSrc{sv.base + u.col_off, nullptr, nullptr, ACT_NONE}, wscratch, s->scratch_floats, s->gpad, s->err, wst);
                 conv_unpad_grad(s->gpad, u.g.co, u.g.k * u.g.k * u.g.ci, u.col_kp, s->g + u.w_off, wst);
+            } else if (u.kind == U_CONV && u.sub_off >= 0) {
+                ValSrc xs = xin;
+                xs.p = sv.base + u.sub_off;                  // written by the forward of this micro-batch
+                pw_bwd_weight_tc(sub_geom(u), d, xs, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst);
             } else if (u.kind == U_CONV && pw_tc_supported(dt, u.g, false))
                 pw_bwd_weight_tc(u.g, d, xin, wscratch, s->scratch_floats, s->g + u.w_off, s->err, wst);
             else if (u.kind == U_CONV && conv3_wgrad_tc_supported(dt, u.g))
