@@ -44,11 +44,16 @@ def _state(P, hdl):
     return wv, vv
 
 
-@pytest.mark.parametrize("bf16", [False, True])
-def test_captured_round_replays_to_the_same_state(bf16):
+@pytest.mark.parametrize("case", ["block_f32", "block_bf16", "bottlenecks_bf16"])
+def test_captured_round_replays_to_the_same_state(case):
     import paper_2408_08015_b200 as P
-    net = si.block_net(16, 6)
-    h, w, B, M, replays = 12, 10, 4, 3, 2
+    bf16 = case.endswith("bf16")
+    if case.startswith("block"):
+        net, h, w, B, M, replays = si.block_net(16, 6), 12, 10, 4, 3, 2
+    else:
+        # bottleneck blocks with a strided projection shortcut: tensor-core 3x3 kernels, the weight-gradient stream, a
+        # device-to-device copy inside the round
+        net, h, w, B, M, replays = si.resnet50_c2c3_net(), 16, 16, 2, 2, 2
     # call by call: one round, then `replays` more
     hdl, dt, n_out, x, t, buf = _setup(P, net, h, w, B, M, bf16, seed=5)
     try:
