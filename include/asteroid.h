@@ -15,7 +15,10 @@
  *    HOST pointers to float.  The stage owns its arenas and frees them in destroy.
  *  - `stream` is a cudaStream_t passed as void*.  forward/backward/accumulate/step and the loss
  *    heads only enqueue work on it; they never synchronise.  create, destroy, import, export
- *    and profile synchronise the device.
+ *    and profile synchronise the device.  backward also enqueues the weight-gradient kernels on a
+ *    stream of the stage that forks from `stream` and joins it before backward returns, so a whole
+ *    round of these calls (after one plain round, in which first-use set-up happens) may be
+ *    captured into a CUDA graph on `stream` and replayed.
  *  - The library has no CPU fallback: without a CUDA device every compute call fails.
  *
  * Flat parameter order (import/export): layers in list order; per layer
