@@ -922,6 +922,19 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
             // before the one wait, so their latencies overlap
             for (int g0 = half * 4; g0 < (NT >> 4); g0 += 4 * nhalf) {
                 uint32_t rr[4][16];
+                // the residual gradient of the batch's 64 columns is requested before the accumulators are read: eight loads in
+                // flight beside the tcgen05.ld instead of one dependent load per 8 columns
+                Vec<__nv_bfloat16> adv[4][2];
+                if (BWD && EXTRA) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const int nn = ((g0 + u) << 4) + (hh << 3);
+                            adv[u][hh].raw = make_uint4(0, 0, 0, 0);
+                            if (p < a.P && nn < a.N) adv[u][hh].load(a.addend, ((size_t)p * a.N + nn) >> 3);
+                        }
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     if (g0 + u < (NT >> 4)) tmem_ld16_issue(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(st * NT + ((g0 + u) << 4)), rr[u]);
@@ -942,9 +955,7 @@ template <bool BWD, bool EXTRA, bool PANELS> __global__ void __launch_bounds__(P
                             }
                             if (BWD && EXTRA && p < a.P) {
                                 float ad[8];
-                                Vec<__nv_bfloat16> av;
-                                av.load(a.addend, ((size_t)p * a.N + nn) >> 3);
-                                av.unpack(ad);
+                                adv[u][hh].unpack(ad);
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) vv[i] += ad[i];
                             }
