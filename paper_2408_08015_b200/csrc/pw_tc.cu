@@ -215,25 +215,39 @@ template <bool BWD> __global__ void __launch_bounds__(NTHREADS) pw_tc_kernel(con
             int ho = t % a.ho, n = t / a.ho;
             pout = ((size_t)n * a.hi + (size_t)ho * a.stride) * a.wi + (size_t)wo * a.stride;
         }
-        for (int g = half; g < (NT >> 3); g += 2) {
-            float v[8];
-            tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g << 3), v);
-            int n = n0 + (g << 3);
-            if (p < a.P && n < a.N) {
-                size_t e = pout * a.N + n;
-                if (!BWD && a.bias) {
+        // column groups in batches of four: the batch's residual-gradient loads are requested before its accumulators are read,
+        // so that four loads are in flight instead of one dependent load per group
+        for (int gb = half; gb < (NT >> 3); gb += 8) {
+            Vec<__nv_bfloat16> av[4];
+            if (BWD && a.addend) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) v[i] += __ldg(a.bias + n + i);
+                for (int u = 0; u < 4; ++u) {
+                    const int n = n0 + ((gb + 2 * u) << 3);
+                    av[u].raw = make_uint4(0, 0, 0, 0);
+                    if (gb + 2 * u < (NT >> 3) && p < a.P && n < a.N) av[u].load(a.addend, (pout * a.N + n) >> 3);
                 }
-                if (BWD && a.addend) {
-                    float ad[8];
-                    Vec<__nv_bfloat16> av;
-                    av.load(a.addend, e >> 3);
-                    av.unpack(ad);
+            }
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) v[i] += ad[i];
+            for (int u = 0; u < 4; ++u) {
+                const int g = gb + 2 * u;
+                if (g >= (NT >> 3)) break;
+                float v[8];
+                tmem_ld8(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g << 3), v);
+                int n = n0 + (g << 3);
+                if (p < a.P && n < a.N) {
+                    size_t e = pout * a.N + n;
+                    if (!BWD && a.bias) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[i] += __ldg(a.bias + n + i);
+                    }
+                    if (BWD && a.addend) {
+                        float ad[8];
+                        av[u].unpack(ad);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[i] += ad[i];
+                    }
+                    *reinterpret_cast<uint4*>(a.out + e) = pack8(v);
                 }
-                *reinterpret_cast<uint4*>(a.out + e) = pack8(v);
             }
         }
     }
