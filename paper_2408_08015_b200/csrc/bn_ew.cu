@@ -581,6 +581,59 @@ __global__ void __launch_bounds__(256) mse_kernel(const T* __restrict__ y, const
     finish_loss(part, scratch, ticket, gridDim.x, 1.f / (float)n, loss, sh);
 }
 
+// Vector form (16-byte loads and stores, two vectors of each operand requested before either is used); elements past the
+// last whole vector are taken by block 0.  The order of additions is fixed by the launch shape.
+template <typename T>
+__global__ void __launch_bounds__(256) mse_vec_kernel(const T* __restrict__ y, const T* __restrict__ t, size_t n, T* __restrict__ dy, float* loss,
+                                                      float* scratch, unsigned* ticket) {
+    pdl_wait();
+    pdl_launch();
+    __shared__ float sh[32];
+    constexpr int V = Vec<T>::N;
+    const size_t nv = n / V, stride = (size_t)gridDim.x * blockDim.x;
+    const float k = 2.f / (float)n;
+    float acc = 0.f;
+    auto one = [&](const Vec<T>& a, const Vec<T>& b, size_t i) {
+        float fa[V], fb[V];
+        a.unpack(fa);
+        b.unpack(fb);
+#pragma unroll
+        for (int q = 0; q < V; ++q) {
+            const float d = fa[q] - fb[q];
+            acc = fmaf(d, d, acc);
+            fa[q] = d * k;
+        }
+        Vec<T> o;
+        o.pack(fa);
+        o.store(dy, i);
+    };
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + stride < nv; i += 2 * stride) {
+        Vec<T> a0, b0, a1, b1;
+        a0.load(y, i);
+        b0.load(t, i);
+        a1.load(y, i + stride);
+        b1.load(t, i + stride);
+        one(a0, b0, i);
+        one(a1, b1, i + stride);
+    }
+    for (; i < nv; i += stride) {
+        Vec<T> a0, b0;
+        a0.load(y, i);
+        b0.load(t, i);
+        one(a0, b0, i);
+    }
+    if (blockIdx.x == 0) {
+        for (size_t e = nv * V + threadIdx.x; e < n; e += blockDim.x) {
+            const float d = to_f<T>(y[e]) - to_f<T>(t[e]);
+            acc = fmaf(d, d, acc);
+            dy[e] = from_f<T>(d * k);
+        }
+    }
+    float part = block_sum(acc, sh);
+    finish_loss(part, scratch, ticket, gridDim.x, 1.f / (float)n, loss, sh);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) xent_kernel(const T* __restrict__ logits, const int32_t* __restrict__ labels, int rows, int classes,
                                                    T* __restrict__ dl, float* loss, float* scratch, unsigned* ticket) {
@@ -820,13 +873,24 @@ void refresh_derived(const float* w, const int32_t* perm, float* derived, __nv_b
     launch_pdl(refresh_kernel, (unsigned)((n + 255) / 256), 256, 0, st, w, perm, derived, wb, wtb, n);
 }
 
-void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, cudaStream_t st) {
-    size_t want = (n + 256 * 8 - 1) / (256 * 8);
+// The MSE head's kernel for both entry points: the vector form where the three tensors are 16-byte aligned, else the scalar form.
+static void launch_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, unsigned* ticket, cudaStream_t st) {
+    const bool vec = ((reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(t) | reinterpret_cast<uintptr_t>(dy)) & 15) == 0;
+    const size_t per_block = vec ? (size_t)256 * 2 * (dtype == 0 ? 4 : 8) : (size_t)256 * 8;
+    size_t want = (n + per_block - 1) / per_block;
     int blocks = (int)(want < 1 ? 1 : (want > LOSS_MAX_BLOCKS ? LOSS_MAX_BLOCKS : want));
-    unsigned* ticket = reinterpret_cast<unsigned*>(scratch + 65536);
     LaunchScope ls(K_LOSS_MSE, 3.0 * n * esz(dtype), 4.0 * n, st);
-    if (dtype == 0) launch_pdl(mse_kernel<float>, blocks, 256, 0, st, (const float*)y, (const float*)t, n, (float*)dy, loss, scratch, ticket);
-    else launch_pdl(mse_kernel<__nv_bfloat16>, blocks, 256, 0, st, (const __nv_bfloat16*)y, (const __nv_bfloat16*)t, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
+    if (dtype == 0) {
+        if (vec) launch_pdl(mse_vec_kernel<float>, blocks, 256, 0, st, (const float*)y, (const float*)t, n, (float*)dy, loss, scratch, ticket);
+        else launch_pdl(mse_kernel<float>, blocks, 256, 0, st, (const float*)y, (const float*)t, n, (float*)dy, loss, scratch, ticket);
+    } else {
+        if (vec) launch_pdl(mse_vec_kernel<__nv_bfloat16>, blocks, 256, 0, st, (const __nv_bfloat16*)y, (const __nv_bfloat16*)t, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
+        else launch_pdl(mse_kernel<__nv_bfloat16>, blocks, 256, 0, st, (const __nv_bfloat16*)y, (const __nv_bfloat16*)t, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
+    }
+}
+
+void loss_mse(int dtype, const void* y, const void* t, size_t n, void* dy, float* loss, float* scratch, cudaStream_t st) {
+    launch_mse(dtype, y, t, n, dy, loss, scratch, reinterpret_cast<unsigned*>(scratch + 65536), st);
 }
 
 void loss_xent(int dtype, const void* logits, const int32_t* labels, int rows, int classes, void* dlogits, float* loss, float* scratch,
@@ -873,13 +937,7 @@ extern "C" int asteroid_loss_mse_noalloc(const void* y, const void* target, size
     cudaStream_t st = (cudaStream_t)stream;
     // the array keeps whatever the previous call left: the ticket must start at zero
     if (cudaMemsetAsync(ticket, 0, sizeof(unsigned), st) != cudaSuccess) return report_error(-5, "asteroid_loss_mse_noalloc: cudaMemsetAsync failed");
-    size_t want = (n + 256 * 8 - 1) / (256 * 8);
-    int blocks = (int)(want < 1 ? 1 : (want > LOSS_MAX_BLOCKS ? LOSS_MAX_BLOCKS : want));
-    {
-        LaunchScope ls(K_LOSS_MSE, 3.0 * n * (dtype == 0 ? 4.0 : 2.0), 4.0 * n, st);
-        if (dtype == 0) launch_pdl(mse_kernel<float>, blocks, 256, 0, st, (const float*)y, (const float*)target, n, (float*)dy, loss, scratch, ticket);
-        else launch_pdl(mse_kernel<__nv_bfloat16>, blocks, 256, 0, st, (const __nv_bfloat16*)y, (const __nv_bfloat16*)target, n, (__nv_bfloat16*)dy, loss, scratch, ticket);
-    }
+    launch_mse(dtype, y, target, n, dy, loss, scratch, ticket, st);
     if (cudaGetLastError() != cudaSuccess) return report_error(-5, "asteroid_loss_mse_noalloc: kernel launch failed");
     return 0;
 }
